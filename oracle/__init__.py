@@ -1,0 +1,142 @@
+"""ctypes loader for the fp64 CPU oracle (``lords_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's
+CPU-baseline leg import this; the product package never does.  The oracle is
+compiled with gcc on first use into ``oracle/liblords_oracle.so``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "lords_oracle.c"
+_LIB = _HERE / "liblords_oracle.so"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    """Compile the oracle (gcc -O2 -fopenmp; no fast-math, so fp64 sums stay in index order)."""
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _LIB.with_suffix(f".tmp{os.getpid()}.so")
+        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-Wall", "-Wextra",
+               str(_SRC), "-o", str(tmp), "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(str(_LIB))
+        i64, p, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
+        lib.lords_oracle_packed_bytes.restype = i64
+        lib.lords_oracle_packed_bytes.argtypes = [i64, i64, ci]
+        lib.lords_oracle_pack_codes.restype = ci
+        lib.lords_oracle_pack_codes.argtypes = [p, i64, i64, ci, p]
+        lib.lords_oracle_unpack_codes.restype = ci
+        lib.lords_oracle_unpack_codes.argtypes = [p, i64, i64, ci, p]
+        lib.lords_oracle_dequant_rows.restype = ci
+        lib.lords_oracle_dequant_rows.argtypes = [p, p, p, p, ci, i64, i64, i64, p, i64, p]
+        lib.lords_oracle_forward.restype = ci
+        lib.lords_oracle_forward.argtypes = [p, p, p, p, p, ci, i64, i64, i64, i64, p, i64, p, ci]
+        lib.lords_oracle_round_bf16.restype = None
+        lib.lords_oracle_round_bf16.argtypes = [p, i64, p]
+        lib.lords_oracle_equivalent_rank.restype = i64
+        lib.lords_oracle_equivalent_rank.argtypes = [i64, i64, i64]
+        _lib = lib
+    return _lib
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def packed_bytes(m: int, n: int, bits: int) -> int:
+    v = _load().lords_oracle_packed_bytes(m, n, bits)
+    if v < 0:
+        raise ValueError(f"oracle: bad shape for packing (m={m}, n={n}, bits={bits})")
+    return int(v)
+
+
+def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
+    """codes uint8 [m, n] -> packed uint8 [m, n*bits/8] in the written layout."""
+    codes = _c(codes, np.uint8)
+    m, n = codes.shape
+    out = np.empty((m, packed_bytes(m, n, bits) // max(m, 1)), dtype=np.uint8)
+    rc = _load().lords_oracle_pack_codes(_ptr(codes), m, n, bits, _ptr(out))
+    if rc != 0:
+        raise ValueError(f"oracle pack failed: {rc}")
+    return out
+
+
+def unpack_codes(packed: np.ndarray, m: int, n: int, bits: int) -> np.ndarray:
+    packed = _c(packed, np.uint8)
+    if packed.size != packed_bytes(m, n, bits):
+        raise ValueError("oracle unpack: wrong packed size")
+    out = np.empty((m, n), dtype=np.uint8)
+    rc = _load().lords_oracle_unpack_codes(_ptr(packed), m, n, bits, _ptr(out))
+    if rc != 0:
+        raise ValueError(f"oracle unpack failed: {rc}")
+    return out
+
+
+def dequant_rows(qpacked, B, A, codebook, bits: int, rows=None) -> np.ndarray:
+    """Rows of W^ = L[Q] (.) (B A) as fp64 [nrows, n]."""
+    B = _c(B, np.uint16); A = _c(A, np.uint16)
+    qpacked = _c(qpacked, np.uint8); codebook = _c(codebook, np.float32)
+    m, r = B.shape
+    n = A.shape[1]
+    assert A.shape[0] == r and codebook.size == 2**bits and qpacked.size == packed_bytes(m, n, bits)
+    if rows is None:
+        rows_p, nrows = None, m
+    else:
+        rows = _c(rows, np.int64); rows_p, nrows = _ptr(rows), rows.size
+    W = np.empty((nrows, n), dtype=np.float64)
+    rc = _load().lords_oracle_dequant_rows(_ptr(qpacked), _ptr(B), _ptr(A), _ptr(codebook), bits,
+                                           m, n, r, rows_p, nrows, _ptr(W))
+    if rc != 0:
+        raise ValueError(f"oracle dequant failed: {rc}")
+    return W
+
+
+def forward(x, qpacked, B, A, codebook, bits: int, rows=None, threads: int = 0, return_threads=False):
+    """y64[t, q] = sum_j x[t, j] * W^[rows[q], j]  (fp64 [M, nrows]); rows=None -> all m rows."""
+    x = _c(x, np.uint16); B = _c(B, np.uint16); A = _c(A, np.uint16)
+    qpacked = _c(qpacked, np.uint8); codebook = _c(codebook, np.float32)
+    M, n = x.shape
+    m, r = B.shape
+    assert A.shape == (r, n) and codebook.size == 2**bits and qpacked.size == packed_bytes(m, n, bits)
+    if rows is None:
+        rows_p, nrows = None, m
+    else:
+        rows = _c(rows, np.int64); rows_p, nrows = _ptr(rows), rows.size
+    y = np.empty((M, nrows), dtype=np.float64)
+    rc = _load().lords_oracle_forward(_ptr(x), _ptr(qpacked), _ptr(B), _ptr(A), _ptr(codebook), bits,
+                                      M, m, n, r, rows_p, nrows, _ptr(y), threads)
+    if rc < 0:
+        raise ValueError(f"oracle forward failed: {rc}")
+    return (y, rc) if return_threads else y
+
+
+def round_bf16(v: np.ndarray) -> np.ndarray:
+    """fp64 array -> bf16 bit patterns (uint16), one round-to-nearest-even step."""
+    v = _c(v, np.float64)
+    out = np.empty(v.shape, dtype=np.uint16)
+    _load().lords_oracle_round_bf16(_ptr(v), v.size, _ptr(out))
+    return out
+
+
+def equivalent_rank(rows: int, cols: int, blk: int) -> int:
+    return int(_load().lords_oracle_equivalent_rank(rows, cols, blk))

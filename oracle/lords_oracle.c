@@ -1,0 +1,236 @@
+/*
+ * lords_oracle.c -- CPU oracle for the LoRDS fused dequantize-and-multiply.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+ * path computes.  It shares no code, header, table or helper with the CUDA
+ * library and must never be linked, imported or called by the product path.
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * What it computes (paper letters in brackets; here m = out-features, n =
+ * in-features, M = tokens, r = rank):
+ *
+ *   S   = B * A                       Eq. 3  (S = BA, B: m x r, A: r x n)
+ *   W^  = L[Q] (.) S                  Eq. 2 and Sec. 3.2/3.3: W^ = Q (.) (BA),
+ *                                     Q_ij a level of the table L (Alg. 1, step 2.1)
+ *   y   = x * W^T                     the linear layer; W is stored out x in (Table 7)
+ *
+ * All arithmetic is fp64, summed sequentially in index order.  Inputs are the
+ * exact bytes the GPU path receives: bf16 bit patterns for x, B, A (widened
+ * exactly), an fp32 level table, and the packed code bytes, which this file
+ * decodes with its OWN reader of the written layout:
+ *
+ *   rows are packed independently, row i starts at byte i * n * bits / 8;
+ *   bits = 4: byte b of a row holds code[2b] in its low nibble, code[2b+1] in its high nibble;
+ *   bits = 3: every 32 consecutive codes form a 96-bit little-endian integer
+ *             sum_j code[j] << (3 j), stored as 12 bytes, least significant first;
+ *   bits = 2: byte b holds code[4b + q] in bits [2q, 2q+2).
+ *
+ * Pins (see tests/test_oracle_pins.py): block-wise equivalence against an
+ * independent Eq. 2 block dequantiser, brute force on tiny inputs, rank-1
+ * reduction to a library matmul, linearity in x, an exact-integer case with a
+ * closed-form answer, pack known-answer bytes, and the rank rule of Table 7.
+ * Not pinned: a forward output on real model weights -- the paper prints no
+ * worked numeric example of the forward path ("parity unpinned" for that only).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_ARG (-1)
+#define ORACLE_ERR_CODE_RANGE (-2)
+#define ORACLE_ERR_NOMEM (-3)
+
+static double bf16_to_f64(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+static int group_ok(int64_t n, int bits)
+{
+    if (bits == 4) return n % 2 == 0;
+    if (bits == 3) return n % 32 == 0;
+    if (bits == 2) return n % 4 == 0;
+    return 0;
+}
+
+/* Read code j of a packed row (bit offset j*bits in the row's little-endian bit stream). */
+static unsigned read_code(const uint8_t *row, int64_t j, int bits)
+{
+    int64_t bit = j * bits;
+    unsigned v = 0;
+    for (int b = 0; b < bits; ++b) {
+        int64_t p = bit + b;
+        v |= (unsigned)((row[p >> 3] >> (p & 7)) & 1u) << b;
+    }
+    return v;
+}
+
+int64_t lords_oracle_packed_bytes(int64_t m, int64_t n, int bits)
+{
+    if (m < 0 || n < 0 || !group_ok(n, bits)) return ORACLE_ERR_ARG;
+    return m * (n * bits / 8);
+}
+
+/* Layout writer, bit by bit from the written spec (used to build oracle inputs). */
+int lords_oracle_pack_codes(const uint8_t *codes, int64_t m, int64_t n, int bits, uint8_t *packed)
+{
+    if (!codes || !packed || m < 0 || n < 0 || !group_ok(n, bits)) return ORACLE_ERR_ARG;
+    int64_t row_bytes = n * bits / 8;
+    memset(packed, 0, (size_t)(m * row_bytes));
+    for (int64_t i = 0; i < m; ++i) {
+        uint8_t *row = packed + i * row_bytes;
+        for (int64_t j = 0; j < n; ++j) {
+            unsigned c = codes[i * n + j];
+            if (c >> bits) return ORACLE_ERR_CODE_RANGE;
+            for (int b = 0; b < bits; ++b) {
+                int64_t p = j * bits + b;
+                row[p >> 3] |= (uint8_t)(((c >> b) & 1u) << (p & 7));
+            }
+        }
+    }
+    return ORACLE_OK;
+}
+
+int lords_oracle_unpack_codes(const uint8_t *packed, int64_t m, int64_t n, int bits, uint8_t *codes)
+{
+    if (!codes || !packed || m < 0 || n < 0 || !group_ok(n, bits)) return ORACLE_ERR_ARG;
+    int64_t row_bytes = n * bits / 8;
+    for (int64_t i = 0; i < m; ++i)
+        for (int64_t j = 0; j < n; ++j)
+            codes[i * n + j] = (uint8_t)read_code(packed + i * row_bytes, j, bits);
+    return ORACLE_OK;
+}
+
+/* Row i of S = B A (Eq. 3), n doubles. */
+static void scale_row(const uint16_t *B, const uint16_t *A, int64_t n, int64_t r, int64_t i, double *S_row)
+{
+    for (int64_t j = 0; j < n; ++j) {
+        double s = 0.0;
+        for (int64_t k = 0; k < r; ++k) s += bf16_to_f64(B[i * r + k]) * bf16_to_f64(A[k * n + j]);
+        S_row[j] = s;
+    }
+}
+
+/*
+ * Rows of the dequantised weight W^ = L[Q] (.) (B A).  rows == NULL means rows 0..nrows-1.
+ * W_out is nrows x n doubles.
+ */
+int lords_oracle_dequant_rows(const uint8_t *qpacked, const uint16_t *B, const uint16_t *A,
+                              const float *codebook, int bits, int64_t m, int64_t n, int64_t r,
+                              const int64_t *rows, int64_t nrows, double *W_out)
+{
+    if (!qpacked || !B || !A || !codebook || !W_out || m < 1 || n < 1 || r < 1 || !group_ok(n, bits))
+        return ORACLE_ERR_ARG;
+    int64_t row_bytes = n * bits / 8;
+    for (int64_t q = 0; q < nrows; ++q) {
+        int64_t i = rows ? rows[q] : q;
+        if (i < 0 || i >= m) return ORACLE_ERR_ARG;
+        double *W_row = W_out + q * n;
+        scale_row(B, A, n, r, i, W_row);
+        for (int64_t j = 0; j < n; ++j)
+            W_row[j] = (double)codebook[read_code(qpacked + i * row_bytes, j, bits)] * W_row[j];
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * y[t][q] = sum_j x[t][j] * W^[rows[q]][j] for t < M, q < nrows, fp64.
+ * rows == NULL means rows 0..nrows-1 (pass nrows = m for the full output).
+ * y64 is M x nrows row-major.  Rows are independent and are spread over `threads`
+ * OpenMP threads (<= 0: all available); the arithmetic of one output does not
+ * depend on the thread count.  Returns the thread count used (> 0) or an error (< 0).
+ */
+int lords_oracle_forward(const uint16_t *x, const uint8_t *qpacked, const uint16_t *B, const uint16_t *A,
+                         const float *codebook, int bits, int64_t M, int64_t m, int64_t n, int64_t r,
+                         const int64_t *rows, int64_t nrows, double *y64, int threads)
+{
+    if (!x || !qpacked || !B || !A || !codebook || !y64 || M < 1 || m < 1 || n < 1 || r < 1 ||
+        nrows < 0 || !group_ok(n, bits))
+        return ORACLE_ERR_ARG;
+    for (int64_t q = 0; q < nrows; ++q) {
+        int64_t i = rows ? rows[q] : q;
+        if (i < 0 || i >= m) return ORACLE_ERR_ARG;
+    }
+    int64_t row_bytes = n * bits / 8;
+    int used = 1;
+    int fail = 0;
+#ifdef _OPENMP
+    if (threads <= 0) threads = omp_get_max_threads();
+    used = threads;
+#else
+    (void)threads;
+#endif
+    /* x widened once: M x n doubles */
+    double *xd = (double *)malloc(sizeof(double) * (size_t)(M * n));
+    if (!xd) return ORACLE_ERR_NOMEM;
+    for (int64_t e = 0; e < M * n; ++e) xd[e] = bf16_to_f64(x[e]);
+
+#pragma omp parallel num_threads(used)
+    {
+        double *W_row = (double *)malloc(sizeof(double) * (size_t)n);
+        if (!W_row) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t q = 0; q < nrows; ++q) {
+            if (!W_row) continue;
+            int64_t i = rows ? rows[q] : q;
+            scale_row(B, A, n, r, i, W_row);                                   /* S_i = (BA)_i      */
+            for (int64_t j = 0; j < n; ++j)                                    /* W^_ij = L[Q_ij] S_ij */
+                W_row[j] = (double)codebook[read_code(qpacked + i * row_bytes, j, bits)] * W_row[j];
+            for (int64_t t = 0; t < M; ++t) {                                  /* y_ti = sum_j x_tj W^_ij */
+                double acc = 0.0;
+                const double *xt = xd + t * n;
+                for (int64_t j = 0; j < n; ++j) acc += xt[j] * W_row[j];
+                y64[t * nrows + q] = acc;
+            }
+        }
+        free(W_row);
+    }
+    free(xd);
+    return fail ? ORACLE_ERR_NOMEM : used;
+}
+
+/*
+ * Round fp64 values to bf16 with one round-to-nearest-even step (no intermediate
+ * fp32 rounding) and return the bit patterns.  Values beyond the bf16 range become
+ * infinities; NaN maps to a quiet NaN.
+ */
+void lords_oracle_round_bf16(const double *v, int64_t count, uint16_t *out)
+{
+    for (int64_t e = 0; e < count; ++e) {
+        double d = v[e];
+        uint16_t sign = (uint16_t)(signbit(d) ? 0x8000u : 0u);
+        double a = fabs(d);
+        if (isnan(d)) { out[e] = 0x7FC0u; continue; }
+        if (a == 0.0) { out[e] = sign; continue; }
+        int ex;
+        (void)frexp(a, &ex);                 /* a = f * 2^ex, f in [0.5, 1) */
+        int e2 = ex - 1;                     /* a = g * 2^e2, g in [1, 2)   */
+        if (e2 < -126) e2 = -126;            /* subnormal range: fixed quantum 2^-133 */
+        double quantum = ldexp(1.0, e2 - 7); /* 8-bit significand */
+        double qv = nearbyint(a / quantum) * quantum; /* default rounding mode: nearest even */
+        float f = (float)qv;                 /* exact: qv is a bf16 value or overflows to inf */
+        if (qv > 3.3895313892515355e38) f = INFINITY;
+        uint32_t u;
+        memcpy(&u, &f, sizeof u);
+        out[e] = (uint16_t)(sign | (uint16_t)(u >> 16));
+    }
+}
+
+/* Equivalent-rank rule of Sec. 3.2 / App. A: r = floor(n m / (blk (n + m))). */
+int64_t lords_oracle_equivalent_rank(int64_t rows, int64_t cols, int64_t blk)
+{
+    if (rows < 1 || cols < 1 || blk < 1) return ORACLE_ERR_ARG;
+    return (rows * cols) / (blk * (rows + cols));
+}

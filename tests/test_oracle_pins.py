@@ -1,0 +1,238 @@
+"""Pins for the fp64 oracle: everything here checks the oracle against something
+other than itself -- paper-printed values, the block-wise special case written as an
+independent Eq. 2 dequantiser, brute force, closed forms and invariants."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2601_22716_b200 import inputs as gen
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _f64(bits16):
+    return gen.bf16_to_f32(bits16).astype(np.float64)
+
+
+def _oracle_forward(lay, rows=None):
+    qp = oracle.pack_codes(lay.codes, lay.bits)
+    return oracle.forward(lay.x, qp, lay.B, lay.A, lay.codebook, lay.bits, rows=rows)
+
+
+# ---------------------------------------------------------------- packing (P7)
+
+def _numpy_pack(codes, bits):
+    """Independent packer: Python big integers, one per row."""
+    m, n = codes.shape
+    out = np.zeros((m, n * bits // 8), dtype=np.uint8)
+    for i in range(m):
+        v = 0
+        for j in range(n):
+            v |= int(codes[i, j]) << (bits * j)
+        out[i] = np.frombuffer(v.to_bytes(n * bits // 8, "little"), dtype=np.uint8)
+    return out
+
+
+def test_pack_known_answers():
+    with open(os.path.join(GOLDEN, "pack_known_answers.txt")) as fh:
+        rows = [ln for ln in fh if ln.strip() and not ln.startswith("#")]
+    assert len(rows) >= 4
+    for ln in rows:
+        bits_s, codes_s, bytes_s = [p.strip() for p in ln.split("|")]
+        bits = int(bits_s)
+        codes = np.array([int(c) for c in codes_s.split()], dtype=np.uint8)[None, :]
+        want = np.array([int(b, 16) for b in bytes_s.split()], dtype=np.uint8)[None, :]
+        got = oracle.pack_codes(codes, bits)
+        assert np.array_equal(got, want), (bits, got, want)
+        assert np.array_equal(oracle.unpack_codes(want, 1, codes.shape[1], bits), codes)
+
+
+@pytest.mark.parametrize("bits,n", [(4, 64), (4, 2), (3, 32), (3, 96), (2, 8)])
+def test_pack_matches_bigint_and_roundtrips(bits, n):
+    rng = np.random.default_rng(bits * 100 + n)
+    codes = rng.integers(0, 2**bits, size=(5, n), dtype=np.uint8)
+    packed = oracle.pack_codes(codes, bits)
+    assert np.array_equal(packed, _numpy_pack(codes, bits))
+    assert np.array_equal(oracle.unpack_codes(packed, 5, n, bits), codes)
+
+
+def test_pack_rejects_bad_input():
+    with pytest.raises(ValueError):
+        oracle.pack_codes(np.full((1, 32), 8, dtype=np.uint8), 3)      # code out of range
+    with pytest.raises(ValueError):
+        oracle.pack_codes(np.zeros((1, 31), dtype=np.uint8), 3)        # n not a multiple of 32
+    with pytest.raises(ValueError):
+        oracle.pack_codes(np.zeros((1, 3), dtype=np.uint8), 4)
+
+
+# ------------------------------------------------- block-wise equivalence (P1)
+
+def _block_dequant(codes, s_bits, codebook, blk):
+    """Eq. 2 written directly: W_b = Q_b * s_b, blocks of blk consecutive in-features per row."""
+    s = _f64(s_bits)
+    levels = codebook.astype(np.float64)[codes]
+    return levels * np.repeat(s, blk, axis=1)
+
+
+@pytest.mark.parametrize("m,n,blk,M,bits", [(256, 256, 64, 4, 4), (48, 128, 32, 3, 3), (24, 96, 32, 2, 3)])
+def test_blockwise_special_case_is_reproduced_exactly(m, n, blk, M, bits):
+    lay, s = gen.make_blockwise_layer(m, n, blk, M, bits=bits, seed=0)
+    W_blk = _block_dequant(lay.codes, s, lay.codebook, blk)
+    qp = oracle.pack_codes(lay.codes, bits)
+    W = oracle.dequant_rows(qp, lay.B, lay.A, lay.codebook, bits)
+    # products with 0/1 and sums of zeros are exact, so equality is bit-for-bit
+    assert np.array_equal(W, W_blk)
+    y = oracle.forward(lay.x, qp, lay.B, lay.A, lay.codebook, bits)
+    y_lib = _f64(lay.x) @ W_blk.T
+    np.testing.assert_allclose(y, y_lib, rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------------------------------ brute force (P2)
+
+@pytest.mark.parametrize("m,n,r,M,bits", [(5, 32, 1, 1, 3), (7, 64, 3, 2, 4), (16, 32, 8, 4, 3), (3, 8, 5, 3, 2)])
+def test_brute_force_elementwise(m, n, r, M, bits):
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=m + n + r, mixed_sign=True)
+    Bf, Af, xf = _f64(lay.B), _f64(lay.A), _f64(lay.x)
+    L = lay.codebook.astype(np.float64)
+    want = np.zeros((M, m))
+    for t in range(M):
+        for i in range(m):
+            acc = 0.0
+            for j in range(n):
+                s = 0.0
+                for k in range(r):
+                    s += Bf[i, k] * Af[k, j]
+                acc += xf[t, j] * (L[lay.codes[i, j]] * s)
+            want[t, i] = acc
+    got = _oracle_forward(lay)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-14)
+
+
+def test_row_subset_matches_full():
+    lay = gen.make_layer(40, 64, 6, 3, bits=4, seed=3)
+    full = _oracle_forward(lay)
+    rows = np.array([39, 0, 17, 17, 5], dtype=np.int64)
+    sub = _oracle_forward(lay, rows=rows)
+    assert np.array_equal(sub, full[:, rows])
+
+
+def test_thread_count_does_not_change_results():
+    lay = gen.make_layer(64, 64, 4, 2, bits=4, seed=9)
+    qp = oracle.pack_codes(lay.codes, 4)
+    y1 = oracle.forward(lay.x, qp, lay.B, lay.A, lay.codebook, 4, threads=1)
+    y4 = oracle.forward(lay.x, qp, lay.B, lay.A, lay.codebook, 4, threads=4)
+    assert np.array_equal(y1, y4)
+
+
+# --------------------------------------------------------------- linearity (P3)
+
+def test_linearity_in_x():
+    m, n, r = 33, 128, 7
+    lay = gen.make_layer(m, n, r, 2, bits=4, seed=11, mixed_sign=True)
+    x = gen.bf16_to_f32(lay.x).copy()
+    x[0, n // 2:] = 0.0       # disjoint supports: the combination below is bf16-exact
+    x[1, :n // 2] = 0.0
+    combo = 4.0 * x[0] - 0.5 * x[1]
+    import torch
+    xs = gen.bf16_bits(torch.from_numpy(np.stack([x[0], x[1], combo])))
+    assert np.array_equal(gen.bf16_to_f32(xs)[2], combo)
+    qp = oracle.pack_codes(lay.codes, 4)
+    y = oracle.forward(xs, qp, lay.B, lay.A, lay.codebook, 4)
+    np.testing.assert_allclose(y[2], 4.0 * y[0] - 0.5 * y[1], rtol=1e-12, atol=1e-13)
+    assert np.abs(y[2]).max() > 0
+
+
+# ------------------------------------------------------ rank-1 reduction (P4)
+
+def test_rank_one_reduces_to_scaled_matmul():
+    m, n, M = 29, 96, 3
+    lay = gen.make_layer(m, n, 1, M, bits=3, seed=5, mixed_sign=True)
+    b = _f64(lay.B)[:, 0]
+    a = _f64(lay.A)[0]
+    Lq = lay.codebook.astype(np.float64)[lay.codes]
+    want = ((_f64(lay.x) * a[None, :]) @ Lq.T) * b[None, :]
+    np.testing.assert_allclose(_oracle_forward(lay), want, rtol=1e-12, atol=1e-14)
+
+
+# ------------------------------------------------------- exact integers (P5)
+
+@pytest.mark.parametrize("bits,n", [(4, 128), (3, 96)])
+def test_integer_case_closed_form(bits, n):
+    m, r, M = 37, 5, 4
+    lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=2)
+    Bi = _f64(lay.B).astype(np.int64)
+    Ai = _f64(lay.A).astype(np.int64)
+    xi = _f64(lay.x).astype(np.int64)
+    Li = lay.codebook.astype(np.int64)[lay.codes]
+    want = xi @ (Li * (Bi @ Ai)).T                       # int64, exact
+    got = _oracle_forward(lay)
+    assert np.array_equal(got, want.astype(np.float64))
+    assert np.abs(want).max() <= 256 and np.abs(want).max() > 0
+    # exactly representable in bf16, so the rounded output carries the same integers
+    assert np.array_equal(gen.bf16_to_f32(oracle.round_bf16(got)).astype(np.int64), want)
+
+
+# ------------------------------------------- reassociated form identity (P6)
+
+def test_reassociated_form_equals_definition():
+    m, n, r, M = 21, 64, 6, 3
+    lay = gen.make_layer(m, n, r, M, bits=4, seed=8, mixed_sign=True)
+    Bf, Af, xf = _f64(lay.B), _f64(lay.A), _f64(lay.x)
+    Lq = lay.codebook.astype(np.float64)[lay.codes]
+    # z[t,i,k] = sum_j L[Q_ij] A_kj x_tj ; y[t,i] = sum_k B_ik z[t,i,k]
+    z = np.einsum("ij,kj,tj->tik", Lq, Af, xf)
+    want = np.einsum("ik,tik->ti", Bf, z)
+    np.testing.assert_allclose(_oracle_forward(lay), want, rtol=1e-11, atol=1e-13)
+
+
+# ------------------------------------------------------ Table 7 rank rule (P8)
+
+def test_equivalent_rank_reproduces_table7():
+    n_rows = 0
+    with open(os.path.join(GOLDEN, "table7_ranks.txt")) as fh:
+        for ln in fh:
+            if not ln.strip() or ln.startswith("#"):
+                continue
+            parts = ln.split()
+            rows, cols, r128, r256 = (int(v) for v in parts[-4:])
+            assert oracle.equivalent_rank(rows, cols, 128) == r128, ln
+            assert oracle.equivalent_rank(rows, cols, 256) == r256, ln
+            n_rows += 1
+    assert n_rows == 13
+    # parameter parity at block size 64 for the 4096 x 4096 projection: 32*(4096+4096) = 4096*4096/64
+    assert oracle.equivalent_rank(4096, 4096, 64) == 32
+
+
+# --------------------------------------------------------- bf16 rounding helper
+
+def test_round_bf16_is_single_rne_step():
+    v = np.array([
+        1.0, -2.5, 0.0, 3.140625,             # exactly representable
+        1.0 + 2.0**-8,                         # tie -> even (1.0)
+        1.0 + 3 * 2.0**-8,                     # tie -> even (1 + 2^-6)
+        1.0 + 2.0**-8 + 2.0**-40,              # just above the tie: must go up (double rounding via fp32 would not)
+        -(1.0 + 2.0**-8 + 2.0**-40),
+        255.5, 1e-3,
+    ])
+    got = gen.bf16_to_f32(oracle.round_bf16(v)).astype(np.float64)
+    want = np.array([1.0, -2.5, 0.0, 3.140625, 1.0, 1.0 + 2.0**-6, 1.0 + 2.0**-7, -(1.0 + 2.0**-7), 256.0,
+                     0.00099945068359375])
+    assert np.array_equal(got, want)
+    # agrees with the torch fp32->bf16 cast wherever the input is an fp32 value
+    import torch
+    f = torch.randn(4096, dtype=torch.float32)
+    assert np.array_equal(oracle.round_bf16(f.double().numpy()), gen.bf16_bits(f))
+
+
+# --------------------------------------------------------------- level tables
+
+@pytest.mark.parametrize("bits", [2, 3, 4])
+def test_nf_codebook_properties(bits):
+    cb = gen.nf_codebook(bits)
+    assert cb.dtype == np.float32 and cb.shape == (2**bits,)
+    assert np.all(np.diff(cb) > 0)
+    assert cb[0] == -1.0 and cb[-1] == 1.0
+    assert np.count_nonzero(cb == 0.0) == 1
+    assert np.count_nonzero(cb < 0) == 2 ** (bits - 1) - 1 and np.count_nonzero(cb > 0) == 2 ** (bits - 1)
