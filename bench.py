@@ -1,0 +1,427 @@
+#!/usr/bin/env python
+"""Benchmark of the LoRDS dequantize-and-multiply hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--case NAME]
+
+A *step* is one pass of the whole hot path (unpack, level lookup, scale reconstruction,
+Hadamard product, contraction, epilogue) over one batch of synthetic layers: `copies`
+distinct weight sets of the case's shape, one forward call each, so that a step touches
+more than twice the L2 capacity and every launch reads its weights from HBM.
+
+The headline case is the Llama-3-8B q_proj decode (m = n = 4096, NF4, r = 32, M = 1) and
+the headline metric is algorithmic HBM bytes per second (packed Q + B + A + x + y).  The
+other cases (M = 8, the 3-bit MLP shapes, the M = 2048 prefill) are reported under "cases".
+
+With N > 1 (torchrun) every rank runs the same workload on its own GPU: the path has no
+exchange step, so the ranks are independent replicas ("weak" scaling, no collective on the
+data path); the time is the max over ranks and the value the sum of all ranks' bytes.
+
+`--impl reference` times the fp64 CPU oracle (the only reference implementation there is)
+on the host cores, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+L2_BYTES = 126 * 1024 * 1024
+
+# name -> (m, n, bits, r, M, outlier_frac, bound)
+CASES = {
+    "decode_q_m1":    dict(m=4096, n=4096, bits=4, r=32, M=1, outliers=0.0, bound="hbm"),
+    "decode_q_m8":    dict(m=4096, n=4096, bits=4, r=32, M=8, outliers=0.0, bound="hbm"),
+    "mlp3_gate_m1":   dict(m=14336, n=4096, bits=3, r=48, M=1, outliers=0.0, bound="hbm"),
+    "mlp3_down_m1":   dict(m=4096, n=14336, bits=3, r=48, M=1, outliers=0.0, bound="hbm"),
+    "mlp3_down_m16":  dict(m=4096, n=14336, bits=3, r=48, M=16, outliers=0.0, bound="hbm"),
+    "prefill_m2048":  dict(m=4096, n=14336, bits=4, r=32, M=2048, outliers=0.01, bound="tensor"),
+}
+HEADLINE = "decode_q_m1"
+METRIC = "LoRDS dequant-GEMM: HBM GB/s at M=1, TFLOP/s at M=2048, % of roofline"
+
+
+def algorithmic_bytes(c):
+    """Packed Q + B + A + x + y, each moved once."""
+    return c["m"] * c["n"] * c["bits"] // 8 + 2 * c["r"] * (c["m"] + c["n"]) + 2 * c["M"] * (c["n"] + c["m"])
+
+
+def useful_flops(c):
+    return 2 * c["M"] * c["m"] * c["n"]
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised
+# under profiles/ (None until a capture of that case exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.splitlines():
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def make_case_layers(case, copies, device):
+    """One host-seeded layer per case; the other weight copies are row-rotations of it
+    (distinct HBM addresses, same statistics), built on the device."""
+    import numpy as np
+    import torch
+    from paper_2601_22716_b200 import binding as lords
+    from paper_2601_22716_b200 import inputs as gen
+
+    c = CASES[case]
+    lay = gen.make_layer(c["m"], c["n"], c["r"], c["M"], bits=c["bits"], seed=0, outlier_frac=c["outliers"])
+    packed = lords.lords_pack_codes(lay.codes, c["bits"])
+    q0 = torch.from_numpy(packed).to(device)
+    B0 = torch.from_numpy(lay.B.view(np.int16)).to(device)
+    A0 = torch.from_numpy(lay.A.view(np.int16)).to(device)
+    x0 = torch.from_numpy(lay.x.view(np.int16)).to(device)
+    sets = []
+    for l in range(copies):
+        if l == 0:
+            sets.append((q0, B0, A0, x0))
+        else:
+            sets.append((torch.roll(q0, l, 0).contiguous(), torch.roll(B0, l, 0).contiguous(),
+                         A0.clone(), x0.clone()))
+    return lay, packed, sets
+
+
+def copies_for(case):
+    c = CASES[case]
+    per = algorithmic_bytes(c)
+    return max(2, -(-2 * L2_BYTES // per) + 1)
+
+
+def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=True):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2601_22716_b200 import binding as lords
+
+    c = CASES[case]
+    copies = copies_for(case)
+    lay, packed, sets = make_case_layers(case, copies, device)
+    M, m, n, r, bits = c["M"], c["m"], c["n"], c["r"], c["bits"]
+    ys = [torch.zeros((M, m), dtype=torch.int16, device=device) for _ in range(copies)]
+
+    def one_step():
+        for (q, B, A, x), y in zip(sets, ys):
+            lords.lords_linear_forward_bits(x, q, B, A, lay.codebook, bits, M, m, n, r, y)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    one_step()
+    torch.cuda.synchronize()
+    launches_per_call = lords.lords_last_launch_count()
+    path = lords.lords_last_path()
+
+    # capture one step in a CUDA graph (launch-bound inner loop); warm up on a side stream first
+    graph = None
+    try:
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            one_step()
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            one_step()
+        graph = g
+    except Exception as e:  # capture is an optimisation, not a requirement
+        print(f"[bench] CUDA graph capture unavailable ({type(e).__name__}: {e}); launching directly",
+              file=sys.stderr)
+        torch.cuda.synchronize()
+
+    run = (graph.replay if graph is not None else one_step)
+    for _ in range(max(warmup, 3)):
+        run()
+    barrier()
+    if sampler is not None:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(steps):
+        run()
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if sampler is not None else None
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / steps
+    assert lords.lords_poll_status() == 0
+
+    # end to end through the host-buffer entry point: H2D of x and D2H of y inside the timed region
+    e2e = None
+    if do_e2e:
+        xh = [torch.from_numpy(lay.x.view(np.int16)).clone().pin_memory() for _ in range(copies)]
+        yh = [torch.zeros((M, m), dtype=torch.int16).pin_memory() for _ in range(copies)]
+
+        def e2e_step():
+            for (q, B, A, _x), xx, yy in zip(sets, xh, yh):
+                lords.lords_linear_forward_host(xx, q, B, A, lay.codebook, bits, M, m, n, r, yy)
+
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        e0.record()
+        e2e_steps = max(1, min(steps, 20))
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        ems = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ems], dtype=torch.float64, device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        e2e = {"ms_per_step": ems / e2e_steps, "h2d_bytes_per_step": copies * M * n * 2,
+               "d2h_bytes_per_step": copies * M * m * 2}
+
+    peaks = measured_peaks()
+    calls = copies
+    us_per_launch = ms_per_step * 1e3 / calls
+    byt, flo = algorithmic_bytes(c), useful_flops(c)
+    gbs = byt / (us_per_launch * 1e-6) / 1e9
+    tfs = flo / (us_per_launch * 1e-6) / 1e12
+    if c["bound"] == "hbm":
+        roof = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0}
+    else:
+        roof = {"bound": "tensor", "achieved": tfs, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": tfs / peaks["bf16_tflops"], "frac_of_sustained": tfs / peaks["bf16_tflops_sustained"],
+                "frac_of_nominal_2.25PF": tfs / 2250.0}
+    roof["peak_source"] = peaks["source"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(case)
+    roof["algorithmic_bytes_per_launch"] = byt
+    roof["us_per_launch"] = us_per_launch
+    res = {
+        "case": case, "path": path, "copies": copies, "ms_per_step": ms_per_step, "us_per_call": us_per_launch,
+        "gbs": gbs * world, "tflops": tfs * world, "roofline": roof, "clocks": clocks,
+        "launches_per_call": launches_per_call, "gpu_launches": steps * calls * launches_per_call,
+        "graph": graph is not None,
+    }
+    if e2e is not None:
+        eus = e2e["ms_per_step"] * 1e3 / calls
+        e2e["gbs"] = byt / (eus * 1e-6) / 1e9 * world
+        e2e["tflops"] = flo / (eus * 1e-6) / 1e12 * world
+        res["e2e"] = e2e
+    res["_lay"] = (lay, packed)
+    return res
+
+
+def cpu_baseline(case, lay, packed, budget_s=12.0):
+    """The oracle as it stands, on the host cores, on a bounded sample of the case."""
+    import numpy as np
+    import oracle
+
+    c = CASES[case]
+    # sample = a subset of output rows sized from a quick probe so the run takes about budget_s
+    probe_rows = np.arange(min(c["m"], 64), dtype=np.int64)
+    t0 = time.perf_counter()
+    _, threads = oracle.forward(lay.x, packed, lay.B, lay.A, lay.codebook, lay.bits, rows=probe_rows,
+                                return_threads=True)
+    dt = max(time.perf_counter() - t0, 1e-4)
+    nrows = int(min(c["m"], max(64, probe_rows.size * budget_s / dt)))
+    rows = np.arange(nrows, dtype=np.int64)
+    t0 = time.perf_counter()
+    oracle.forward(lay.x, packed, lay.B, lay.A, lay.codebook, lay.bits, rows=rows)
+    dt = time.perf_counter() - t0
+    frac = nrows / c["m"]
+    sec_full = dt / frac
+    byt, flo = algorithmic_bytes(c), useful_flops(c)
+    if c["bound"] == "hbm":
+        value, unit = byt / sec_full / 1e9, "GB/s"
+    else:
+        value, unit = flo / sec_full / 1e12, "TFLOP/s"
+    return {"value": value, "unit": unit, "cores": int(threads), "kind": "oracle",
+            "sample": f"{nrows} of {c['m']} output rows of one {case} layer, all {c['M']} tokens, "
+                      f"{dt:.2f} s measured, scaled to the full layer"}
+
+
+def run_reference(args):
+    """--impl reference: the fp64 oracle on the host cores (there is no other reference)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import numpy as np
+    import oracle
+    from paper_2601_22716_b200 import inputs as gen
+
+    case = args.case or HEADLINE
+    c = CASES[case]
+    lay = gen.make_layer(c["m"], c["n"], c["r"], c["M"], bits=c["bits"], seed=0, outlier_frac=c["outliers"])
+    packed = oracle.pack_codes(lay.codes, c["bits"])
+    # each step = the oracle over a fixed sample of output rows of one layer
+    probe = np.arange(min(64, c["m"]), dtype=np.int64)
+    t0 = time.perf_counter()
+    _, threads = oracle.forward(lay.x, packed, lay.B, lay.A, lay.codebook, lay.bits, rows=probe, return_threads=True)
+    dt = max(time.perf_counter() - t0, 1e-4)
+    total = max(1, args.steps + args.warmup)
+    nrows = int(min(c["m"], max(64, 64 * (60.0 / total) / dt)))
+    rows = np.arange(nrows, dtype=np.int64)
+    for _ in range(args.warmup):
+        oracle.forward(lay.x, packed, lay.B, lay.A, lay.codebook, lay.bits, rows=rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.forward(lay.x, packed, lay.B, lay.A, lay.codebook, lay.bits, rows=rows)
+    dt = (time.perf_counter() - t0) / args.steps
+    sec_full = dt * c["m"] / nrows
+    byt, flo = algorithmic_bytes(c), useful_flops(c)
+    value, unit = (byt / sec_full / 1e9, "GB/s") if c["bound"] == "hbm" else (flo / sec_full / 1e12, "TFLOP/s")
+    sample = f"{nrows} of {c['m']} output rows of one {case} layer per step, scaled to the full layer"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": unit, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": case, **{k: c[k] for k in ("m", "n", "bits", "r", "M")}},
+        "cpu_baseline": {"value": value, "unit": unit, "cores": int(threads), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--case", default=None, help="time only this case (default: headline plus the others)")
+    ap.add_argument("--no-extras", action="store_true", help="headline case only")
+    ap.add_argument("--path", default="auto", help="force a kernel path (auto|simt|decode|prefill)")
+    args = ap.parse_args()
+
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2601_22716_b200 import binding as lords   # raises if liblords.so is missing: no fallback
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the hot path has no CPU fallback)")
+    torch.cuda.set_device(local)
+    device = torch.device(f"cuda:{local}")
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    lords.lords_init(local, 0)
+    lords.lords_set_option("path", args.path)
+
+    head = args.case or HEADLINE
+    sampler = ClockSampler(local) if rank == 0 else None
+    res = time_case(head, args.steps, args.warmup, device, rank, world, sampler)
+    lay, packed = res.pop("_lay")
+    c = CASES[head]
+    cases = []
+    if not args.case and not args.no_extras:
+        for name in CASES:
+            if name == head:
+                continue
+            k = max(3, min(args.steps, 20 if CASES[name]["M"] <= 16 else 5))
+            r2 = time_case(name, k, 3, device, rank, world, None, do_e2e=False)
+            r2.pop("_lay")
+            cases.append({"case": name, "path": r2["path"], "us_per_call": r2["us_per_call"],
+                          "gbs": r2["gbs"], "tflops": r2["tflops"], "roofline": r2["roofline"],
+                          "copies": r2["copies"], "steps": k})
+
+    if rank == 0:
+        hbm = c["bound"] == "hbm"
+        value = res["gbs"] if hbm else res["tflops"]
+        unit = "GB/s" if hbm else "TFLOP/s"
+        base = cpu_baseline(head, lay, packed) if world == 1 else None
+        e2e = res.get("e2e")
+        line = {
+            "metric": METRIC, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": res["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16 operands, f32 accumulate, bf16 in/out",
+            "data": "synthetic",
+            "config": {"workload": head, **{k: c[k] for k in ("m", "n", "bits", "r", "M")},
+                       "copies_per_step": res["copies"], "path": res["path"], "cuda_graph": res["graph"],
+                       "l2": f"step rotates over {res['copies']} distinct weight sets "
+                             f"({res['copies'] * algorithmic_bytes(c) / 1e6:.0f} MB > 2 x L2), no explicit flush",
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "us_per_call": res["us_per_call"],
+            "roofline": res["roofline"], "clocks": res["clocks"], "gpu_launches": res["gpu_launches"],
+            "e2e": None if e2e is None else {
+                "value": e2e["gbs"] if hbm else e2e["tflops"], "unit": unit,
+                "h2d_bytes_per_step": e2e["h2d_bytes_per_step"], "d2h_bytes_per_step": e2e["d2h_bytes_per_step"],
+                "ms_per_step": e2e["ms_per_step"]},
+            "cpu_baseline": base, "cases": cases,
+        }
+        print(json.dumps(line))
+    lords.lords_shutdown()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,176 @@
+/*
+ * lords.h -- C ABI of the B200 (sm_100a) LoRDS dequantize-and-multiply library.
+ *
+ * The library computes one quantised linear layer of LoRDS inference:
+ *
+ *     y = x * ( L[Q] (.) (B A) )^T
+ *
+ *   x : M x n activations (tokens x in-features)
+ *   Q : m x n codes, bits per code 2, 3 or 4, packed (layout below)
+ *   L : level table with 2^bits entries (the target data type's discrete levels,
+ *       e.g. NF4; Sec. 3.1 "Round(.) ... nearest discrete levels of a target data type")
+ *   B : m x r, A : r x n -- the low-rank factors of the element-wise scale matrix
+ *       S = B A (Sec. 3.2, Eq. 3); S is rebuilt on chip and never stored in full
+ *   y : M x m outputs (tokens x out-features)
+ *
+ * The dequantised weight is W^ = Q (.) (BA) with Q_ij a level of L (Sec. 3.2-3.3,
+ * Alg. 1 step 2.1; Eq. 2 is its block-wise special case), and the layer is
+ * y = x W^T with W stored out-features x in-features (Table 7 lists shapes that way).
+ * Note the paper writes W in R^{n x m}; this interface uses m for out-features and
+ * n for in-features (the reduction axis).
+ *
+ * Conventions
+ *   - every function returns an int status: LORDS_OK (0) or a negative LORDS_ERR_*;
+ *     nothing throws, exits or traps.  Size-returning calls return a negative
+ *     LORDS_ERR_* on error.
+ *   - "device" pointers are CUDA global-memory pointers on the device given to
+ *     lords_init; "host" pointers are ordinary CPU memory.
+ *   - all matrices are dense row-major without padding.  x, B, A, y hold bf16
+ *     (IEEE bfloat16 bit patterns, 2 bytes); device pointers must be 16-byte aligned.
+ *   - the caller owns every buffer it passes for the whole asynchronous lifetime of
+ *     the call; the library neither retains nor frees them.  x/y aliasing is undefined.
+ *   - forward calls validate on the host, enqueue work on `stream` and return
+ *     without synchronising.  They use library-owned scratch memory, so two forward
+ *     calls may only overlap on the GPU if they are ordered on the same stream.
+ *
+ * Packed code layout (the paper does not fix one; this is the library's definition)
+ *   rows are packed independently; row i starts at byte i * n * bits / 8 and is a
+ *   little-endian bit stream with code j at bit offset j * bits:
+ *     bits = 4 : byte b = code[2b] | code[2b+1] << 4            (n % 2  == 0)
+ *     bits = 3 : 32 codes -> 96-bit little-endian integer, 12 B  (n % 32 == 0)
+ *     bits = 2 : byte b = code[4b+q] << 2q, q = 0..3             (n % 4  == 0)
+ *   Code c selects level L[c].
+ */
+#ifndef LORDS_H_
+#define LORDS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LORDS_VERSION 100 /* major*10000 + minor*100 + patch */
+
+/* status codes */
+#define LORDS_OK 0
+#define LORDS_ERR_NULL (-1)        /* a required pointer is NULL */
+#define LORDS_ERR_SHAPE (-2)       /* M, m, n or r out of range, or n not a multiple of the pack group */
+#define LORDS_ERR_ALIGN (-3)       /* a device pointer is not 16-byte aligned */
+#define LORDS_ERR_BITS (-4)        /* bits is not 2, 3 or 4 */
+#define LORDS_ERR_CODE_RANGE (-5)  /* a code is >= 2^bits */
+#define LORDS_ERR_NOT_INIT (-6)    /* lords_init has not been called (or failed) */
+#define LORDS_ERR_CUDA (-7)        /* a CUDA runtime/driver call failed; see lords_last_cuda_error */
+#define LORDS_ERR_TIMEOUT (-8)     /* a bounded device-side wait gave up (reported by lords_poll_status) */
+#define LORDS_ERR_WORKSPACE (-9)   /* the problem needs more scratch memory than lords_init reserved */
+#define LORDS_ERR_OPTION (-10)     /* unknown option key or bad value */
+#define LORDS_ERR_UNSUPPORTED (-11)/* the forced path cannot run this shape */
+
+#define LORDS_R_MAX 128            /* largest supported rank r */
+#define LORDS_M_MAX 65536          /* largest supported token count M */
+
+/* Library version (LORDS_VERSION of the built library). */
+int lords_version(void);
+
+/* Static, human-readable text for a status code.  Never NULL. */
+const char *lords_strerror(int status);
+
+/*
+ * Equivalent-rank rule of Sec. 3.2 / App. A: r = floor(rows*cols / (blk*(rows+cols))), the rank
+ * whose factor parameters r*(rows+cols) fit the block-wise scale budget rows*cols/blk.
+ * Returns the rank (>= 0) or LORDS_ERR_SHAPE.
+ */
+int64_t lords_equivalent_rank(int64_t rows, int64_t cols, int64_t blk);
+
+/* Bytes of the packed form of an m x n code matrix: m * n * bits / 8, or a negative status. */
+int64_t lords_packed_bytes(int64_t m, int64_t n, int bits);
+
+/*
+ * Pack codes (offline, once per layer; the storage implied by the paper's "4-bit" accounting).
+ *   codes  : host, m*n bytes, one code per byte, row-major
+ *   packed : host, lords_packed_bytes(m, n, bits) bytes, fully overwritten
+ * Pure CPU, deterministic.  Fails with LORDS_ERR_CODE_RANGE (packed contents then unspecified)
+ * if any code >= 2^bits.
+ */
+int lords_pack_codes(const uint8_t *codes, int64_t m, int64_t n, int bits, uint8_t *packed);
+
+/* Inverse of lords_pack_codes: packed (host) -> codes (host, m*n bytes). */
+int lords_unpack_codes(const uint8_t *packed, int64_t m, int64_t n, int bits, uint8_t *codes);
+
+/*
+ * Bind the library to CUDA device `device` and allocate its scratch memory (split-K
+ * partial sums, converted activations, a device status word).  workspace_bytes = 0 selects
+ * the default (256 MiB).  Calling it again re-initialises.  Must precede any forward call.
+ */
+int lords_init(int device, size_t workspace_bytes);
+
+/* Free everything lords_init allocated.  Safe to call when not initialised. */
+int lords_shutdown(void);
+
+/*
+ * The fused dequantize-and-multiply y = x (L[Q] (.) (BA))^T for 4-bit codes (Sec. 3.2-3.4;
+ * the operator timed in Sec. 4.4).
+ *   x        : device, bf16 [M][n]
+ *   Qpacked  : device, packed 4-bit codes, m * n / 2 bytes
+ *   B        : device, bf16 [m][r]
+ *   A        : device, bf16 [r][n]
+ *   codebook : HOST, 16 floats, level table L (copied into the launch; may be freed on return)
+ *   y        : device, bf16 [M][m]; accumulation is fp32, the store rounds to nearest even
+ *   stream   : a cudaStream_t passed as void* (NULL = the default stream)
+ * Ranges: 1 <= M <= LORDS_M_MAX, 1 <= r <= LORDS_R_MAX, m >= 1, n >= 2 and even.
+ */
+int lords_linear_forward(const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                         const float *codebook, int M, int m, int n, int r, void *y, void *stream);
+
+/* Same with an explicit code width: bits in {2, 3, 4}; codebook holds 2^bits floats. */
+int lords_linear_forward_bits(const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                              const float *codebook, int bits, int M, int m, int n, int r, void *y,
+                              void *stream);
+
+/*
+ * Verification entry: identical kernels, but the epilogue stores the fp32 accumulator.
+ *   y32 : device, float [M][m]
+ */
+int lords_linear_forward_f32(const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                             const float *codebook, int bits, int M, int m, int n, int r, float *y32,
+                             void *stream);
+
+/*
+ * End-to-end variant for callers whose activations live in host memory: x_host (bf16 [M][n])
+ * and y_host (bf16 [M][m]) are HOST pointers (pinned memory recommended, otherwise the copies
+ * are synchronous); the weights Qpacked, B, A stay device-resident as above.  Enqueues, on
+ * `stream`, the host-to-device copy of x, the same kernels as lords_linear_forward_bits and
+ * the device-to-host copy of y, and returns without synchronising.  The device staging
+ * buffers are library-owned and grow (cudaMalloc) the first time a larger M*n or M*m is seen,
+ * so the first call of a given size must not be made during stream capture.
+ */
+int lords_linear_forward_host(const void *x_host, const uint8_t *Qpacked, const void *B, const void *A,
+                              const float *codebook, int bits, int M, int m, int n, int r, void *y_host,
+                              void *stream);
+
+/*
+ * Read and clear the device status word.  Synchronises `stream` first.  Returns LORDS_OK, or
+ * the error a kernel recorded (LORDS_ERR_TIMEOUT when a bounded wait ran out).
+ */
+int lords_poll_status(void *stream);
+
+/* The cudaError_t (as int) of the most recent failed CUDA call, 0 if none. */
+int lords_last_cuda_error(void);
+
+/*
+ * Measurement switches.  Keys: "path" = "auto" | "simt" | "decode" | "prefill";
+ * "splitk" = "0" (auto) or a positive integer.  Unknown keys: LORDS_ERR_OPTION.
+ */
+int lords_set_option(const char *key, const char *value);
+
+/* Name of the path the most recent forward call dispatched to ("simt", "decode", "prefill"). */
+const char *lords_last_path(void);
+
+/* Number of kernels the most recent forward call launched. */
+int lords_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LORDS_H_ */

@@ -1,0 +1,308 @@
+// Host side of liblords.so: the C ABI of include/lords.h -- argument validation, the
+// code packer, library state and the per-shape dispatch to the kernels.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+
+#include "lords_internal.h"
+
+namespace lords {
+
+State &state()
+{
+    static State s;
+    return s;
+}
+
+int cuda_fail(cudaError_t e)
+{
+    state().last_cuda_error = (int)e;
+    (void)cudaGetLastError();  // clear the sticky-free error so later calls start clean
+    return LORDS_ERR_CUDA;
+}
+
+static int pack_group(int bits)
+{
+    switch (bits) {
+        case 4: return 2;
+        case 3: return 32;
+        case 2: return 4;
+        default: return 0;
+    }
+}
+
+static int check_pack_shape(int64_t m, int64_t n, int bits)
+{
+    int g = pack_group(bits);
+    if (g == 0) return LORDS_ERR_BITS;
+    if (m < 0 || n < 0 || n % g != 0) return LORDS_ERR_SHAPE;
+    return LORDS_OK;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int validate(const void *x, const uint8_t *q, const void *B, const void *A, const float *cb,
+                    int bits, int M, int m, int n, int r, const void *y)
+{
+    if (!x || !q || !B || !A || !cb || !y) return LORDS_ERR_NULL;
+    int g = pack_group(bits);
+    if (g == 0) return LORDS_ERR_BITS;
+    if (M < 1 || M > LORDS_M_MAX || m < 1 || n < 1 || r < 1 || r > LORDS_R_MAX) return LORDS_ERR_SHAPE;
+    if (n % g != 0) return LORDS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(q) || !aligned16(B) || !aligned16(A) || !aligned16(y)) return LORDS_ERR_ALIGN;
+    if (!state().initialised) return LORDS_ERR_NOT_INIT;
+    return LORDS_OK;
+}
+
+static int forward_common(const void *x, const uint8_t *q, const void *B, const void *A, const float *cb,
+                          int bits, int M, int m, int n, int r, void *y, int y_f32, void *stream)
+{
+    int rc = validate(x, q, B, A, cb, bits, M, m, n, r, y);
+    if (rc != LORDS_OK) return rc;
+    State &st = state();
+    Problem p;
+    p.x = static_cast<const uint16_t *>(x);
+    p.q = q;
+    p.B = static_cast<const uint16_t *>(B);
+    p.A = static_cast<const uint16_t *>(A);
+    for (int c = 0; c < 16; ++c) p.levels[c] = c < (1 << bits) ? cb[c] : 0.0f;
+    p.bits = bits; p.M = M; p.m = m; p.n = n; p.r = r;
+    p.y = y; p.y_f32 = y_f32;
+    st.last_launches = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    // Dispatch.  The tensor-core paths decline (LORDS_ERR_UNSUPPORTED) shapes outside their
+    // tiling rules; "auto" then falls back to the generic CUDA-core path.
+    if (st.forced_path == 1 || st.forced_path == 0) return launch_simt(p, st, s);
+    return LORDS_ERR_UNSUPPORTED;
+}
+
+}  // namespace lords
+
+using namespace lords;
+
+extern "C" {
+
+int lords_version(void) { return LORDS_VERSION; }
+
+const char *lords_strerror(int status)
+{
+    switch (status) {
+        case LORDS_OK: return "ok";
+        case LORDS_ERR_NULL: return "a required pointer is NULL";
+        case LORDS_ERR_SHAPE: return "shape out of range or n not a multiple of the pack group";
+        case LORDS_ERR_ALIGN: return "device pointer not 16-byte aligned";
+        case LORDS_ERR_BITS: return "bits must be 2, 3 or 4";
+        case LORDS_ERR_CODE_RANGE: return "code value >= 2^bits";
+        case LORDS_ERR_NOT_INIT: return "lords_init has not been called";
+        case LORDS_ERR_CUDA: return "CUDA call failed (see lords_last_cuda_error)";
+        case LORDS_ERR_TIMEOUT: return "a bounded device-side wait timed out";
+        case LORDS_ERR_WORKSPACE: return "scratch workspace too small for this problem";
+        case LORDS_ERR_OPTION: return "unknown option or bad value";
+        case LORDS_ERR_UNSUPPORTED: return "forced path does not support this shape";
+        default: return "unknown status";
+    }
+}
+
+int64_t lords_equivalent_rank(int64_t rows, int64_t cols, int64_t blk)
+{
+    if (rows < 1 || cols < 1 || blk < 1) return LORDS_ERR_SHAPE;
+    // rows*cols < 2^63 for any realistic layer; guard the product anyway
+    if (rows > (int64_t)3e9 || cols > (int64_t)3e9) return LORDS_ERR_SHAPE;
+    return (rows * cols) / (blk * (rows + cols));
+}
+
+int64_t lords_packed_bytes(int64_t m, int64_t n, int bits)
+{
+    int rc = check_pack_shape(m, n, bits);
+    if (rc != LORDS_OK) return rc;
+    return m * (n * bits / 8);  // n * bits is a multiple of 8 for every pack group
+}
+
+int lords_pack_codes(const uint8_t *codes, int64_t m, int64_t n, int bits, uint8_t *packed)
+{
+    if (!codes || !packed) return LORDS_ERR_NULL;
+    int rc = check_pack_shape(m, n, bits);
+    if (rc != LORDS_OK) return rc;
+    const int64_t row_bytes = lords_packed_bytes(1, n, bits);
+    const unsigned limit = 1u << bits;
+    for (int64_t i = 0; i < m; ++i) {
+        const uint8_t *src = codes + i * n;
+        uint8_t *dst = packed + i * row_bytes;
+        // 64-bit shift register: codes enter at the top of the valid bits, whole bytes leave at the bottom
+        uint64_t window = 0;
+        int have = 0;
+        for (int64_t j = 0; j < n; ++j) {
+            unsigned c = src[j];
+            if (c >= limit) return LORDS_ERR_CODE_RANGE;
+            window |= (uint64_t)c << have;
+            have += bits;
+            while (have >= 8) {
+                *dst++ = (uint8_t)window;
+                window >>= 8;
+                have -= 8;
+            }
+        }
+    }
+    return LORDS_OK;
+}
+
+int lords_unpack_codes(const uint8_t *packed, int64_t m, int64_t n, int bits, uint8_t *codes)
+{
+    if (!codes || !packed) return LORDS_ERR_NULL;
+    int rc = check_pack_shape(m, n, bits);
+    if (rc != LORDS_OK) return rc;
+    const int64_t row_bytes = lords_packed_bytes(1, n, bits);
+    const unsigned mask = (1u << bits) - 1u;
+    for (int64_t i = 0; i < m; ++i) {
+        const uint8_t *src = packed + i * row_bytes;
+        uint8_t *dst = codes + i * n;
+        uint64_t window = 0;
+        int have = 0;
+        for (int64_t j = 0; j < n; ++j) {
+            if (have < bits) {
+                window |= (uint64_t)(*src++) << have;
+                have += 8;
+            }
+            dst[j] = (uint8_t)(window & mask);
+            window >>= bits;
+            have -= bits;
+        }
+    }
+    return LORDS_OK;
+}
+
+int lords_init(int device, size_t workspace_bytes)
+{
+    State &st = state();
+    if (st.initialised) lords_shutdown();
+    int count = 0;
+    LORDS_CUDA_TRY(cudaGetDeviceCount(&count));
+    if (device < 0 || device >= count) return LORDS_ERR_SHAPE;
+    LORDS_CUDA_TRY(cudaSetDevice(device));
+    cudaDeviceProp prop;
+    LORDS_CUDA_TRY(cudaGetDeviceProperties(&prop, device));
+    st.device = device;
+    st.sm_count = prop.multiProcessorCount;
+    if (workspace_bytes == 0) workspace_bytes = (size_t)256 << 20;
+    LORDS_CUDA_TRY(cudaMalloc(&st.workspace, workspace_bytes));
+    st.workspace_bytes = workspace_bytes;
+    cudaError_t e = cudaMalloc(&st.status_word, 256);
+    if (e == cudaSuccess) e = cudaMemset(st.status_word, 0, 256);
+    if (e != cudaSuccess) {
+        cudaFree(st.workspace);
+        st.workspace = nullptr;
+        return cuda_fail(e);
+    }
+    st.initialised = 1;
+    return LORDS_OK;
+}
+
+int lords_shutdown(void)
+{
+    State &st = state();
+    if (st.initialised) {
+        cudaSetDevice(st.device);
+        cudaDeviceSynchronize();
+        cudaFree(st.workspace);
+        cudaFree(st.status_word);
+        if (st.stage_x) cudaFree(st.stage_x);
+        if (st.stage_y) cudaFree(st.stage_y);
+    }
+    int fp = st.forced_path, fs = st.forced_splitk;
+    st = State();
+    st.forced_path = fp;
+    st.forced_splitk = fs;
+    return LORDS_OK;
+}
+
+int lords_linear_forward(const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                         const float *codebook, int M, int m, int n, int r, void *y, void *stream)
+{
+    return forward_common(x, Qpacked, B, A, codebook, 4, M, m, n, r, y, 0, stream);
+}
+
+int lords_linear_forward_bits(const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                              const float *codebook, int bits, int M, int m, int n, int r, void *y,
+                              void *stream)
+{
+    return forward_common(x, Qpacked, B, A, codebook, bits, M, m, n, r, y, 0, stream);
+}
+
+int lords_linear_forward_f32(const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                             const float *codebook, int bits, int M, int m, int n, int r, float *y32,
+                             void *stream)
+{
+    return forward_common(x, Qpacked, B, A, codebook, bits, M, m, n, r, y32, 1, stream);
+}
+
+int lords_linear_forward_host(const void *x_host, const uint8_t *Qpacked, const void *B, const void *A,
+                              const float *codebook, int bits, int M, int m, int n, int r, void *y_host,
+                              void *stream)
+{
+    State &st = state();
+    if (!x_host || !y_host) return LORDS_ERR_NULL;
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    if (M < 1 || M > LORDS_M_MAX || m < 1 || n < 1) return LORDS_ERR_SHAPE;
+    const size_t xb = (size_t)M * n * 2, yb = (size_t)M * m * 2;
+    if (xb > st.stage_x_bytes) {
+        if (st.stage_x) cudaFree(st.stage_x);
+        st.stage_x = nullptr; st.stage_x_bytes = 0;
+        LORDS_CUDA_TRY(cudaMalloc(&st.stage_x, xb));
+        st.stage_x_bytes = xb;
+    }
+    if (yb > st.stage_y_bytes) {
+        if (st.stage_y) cudaFree(st.stage_y);
+        st.stage_y = nullptr; st.stage_y_bytes = 0;
+        LORDS_CUDA_TRY(cudaMalloc(&st.stage_y, yb));
+        st.stage_y_bytes = yb;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    LORDS_CUDA_TRY(cudaMemcpyAsync(st.stage_x, x_host, xb, cudaMemcpyHostToDevice, s));
+    int rc = forward_common(st.stage_x, Qpacked, B, A, codebook, bits, M, m, n, r, st.stage_y, 0, stream);
+    if (rc != LORDS_OK) return rc;
+    LORDS_CUDA_TRY(cudaMemcpyAsync(y_host, st.stage_y, yb, cudaMemcpyDeviceToHost, s));
+    return LORDS_OK;
+}
+
+int lords_poll_status(void *stream)
+{
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    LORDS_CUDA_TRY(cudaStreamSynchronize(s));
+    int word = 0;
+    LORDS_CUDA_TRY(cudaMemcpy(&word, st.status_word, sizeof(int), cudaMemcpyDeviceToHost));
+    if (word != 0) LORDS_CUDA_TRY(cudaMemset(st.status_word, 0, sizeof(int)));
+    return word;
+}
+
+int lords_last_cuda_error(void) { return state().last_cuda_error; }
+
+int lords_set_option(const char *key, const char *value)
+{
+    if (!key || !value) return LORDS_ERR_NULL;
+    State &st = state();
+    if (std::strcmp(key, "path") == 0) {
+        if (std::strcmp(value, "auto") == 0) st.forced_path = 0;
+        else if (std::strcmp(value, "simt") == 0) st.forced_path = 1;
+        else if (std::strcmp(value, "decode") == 0) st.forced_path = 2;
+        else if (std::strcmp(value, "prefill") == 0) st.forced_path = 3;
+        else return LORDS_ERR_OPTION;
+        return LORDS_OK;
+    }
+    if (std::strcmp(key, "splitk") == 0) {
+        char *end = nullptr;
+        long v = std::strtol(value, &end, 10);
+        if (end == value || *end != '\0' || v < 0 || v > 1024) return LORDS_ERR_OPTION;
+        st.forced_splitk = (int)v;
+        return LORDS_OK;
+    }
+    return LORDS_ERR_OPTION;
+}
+
+const char *lords_last_path(void) { return state().last_path; }
+
+int lords_last_launch_count(void) { return state().last_launches; }
+
+}  // extern "C"

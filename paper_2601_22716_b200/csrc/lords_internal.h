@@ -1,0 +1,57 @@
+// Internal declarations shared by the translation units of liblords.so (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "lords.h"
+
+namespace lords {
+
+// One forward call, validated.  Pointers are device pointers except the level table,
+// which travels by value inside the kernel parameters.
+struct Problem {
+    const uint16_t *x;   // bf16 [M][n]
+    const uint8_t *q;    // packed codes, m * n * bits / 8 bytes
+    const uint16_t *B;   // bf16 [m][r]
+    const uint16_t *A;   // bf16 [r][n]
+    float levels[16];    // L, 2^bits entries used
+    int bits, M, m, n, r;
+    void *y;             // bf16 [M][m] or float [M][m]
+    int y_f32;           // 1: store the fp32 accumulator
+};
+
+// Library-owned device memory and switches (one instance per process).
+struct State {
+    int initialised = 0;
+    int device = -1;
+    int sm_count = 0;
+    uint8_t *workspace = nullptr;   // scratch: split-K partials / converted activations
+    size_t workspace_bytes = 0;
+    int *status_word = nullptr;     // device int, 0 = OK, else a LORDS_ERR_* a kernel recorded
+    uint8_t *stage_x = nullptr;     // device staging for the host-buffer entry point
+    uint8_t *stage_y = nullptr;
+    size_t stage_x_bytes = 0, stage_y_bytes = 0;
+    int forced_path = 0;            // 0 auto, 1 simt, 2 decode, 3 prefill
+    int forced_splitk = 0;          // 0 auto
+    int last_cuda_error = 0;
+    int last_launches = 0;
+    const char *last_path = "none";
+};
+
+State &state();
+
+// Records a failed CUDA call and maps it to LORDS_ERR_CUDA.
+int cuda_fail(cudaError_t e);
+
+#define LORDS_CUDA_TRY(expr)                                   \
+    do {                                                       \
+        cudaError_t e__ = (expr);                              \
+        if (e__ != cudaSuccess) return ::lords::cuda_fail(e__);\
+    } while (0)
+
+// Generic CUDA-core path: any shape the interface accepts.
+int launch_simt(const Problem &p, State &st, cudaStream_t stream);
+
+}  // namespace lords

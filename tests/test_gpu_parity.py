@@ -1,0 +1,165 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2601_22716_b200 import inputs as gen
+from _util import DeviceLayer, check_against_oracle, error_metrics, NORMWISE_TOL, ELEMENT_TOL
+
+pytestmark = pytest.mark.gpu
+
+PATHS = ["auto", "simt"]
+
+
+@pytest.fixture(scope="module")
+def lords():
+    import torch
+    from paper_2601_22716_b200 import binding
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.lords_init(0, 0)
+    yield binding
+    binding.lords_set_option("path", "auto")
+    binding.lords_set_option("splitk", "0")
+    binding.lords_shutdown()
+
+
+def _oracle(lay, packed, rows=None):
+    return oracle.forward(lay.x, packed, lay.B, lay.A, lay.codebook, lay.bits, rows=rows)
+
+
+def _run(lords, lay, path="auto"):
+    lords.lords_set_option("path", path)
+    try:
+        dl = DeviceLayer(lay)
+        y32, ybf = dl.forward()
+    finally:
+        lords.lords_set_option("path", "auto")
+    return dl, y32, ybf
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_config0_tiny_random(lords, path):
+    lay = gen.make_layer(256, 256, 4, 4, bits=4, seed=0, scale_gain=0.1, scale_shift=0.05)
+    dl, y32, ybf = _run(lords, lay, path)
+    check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_config0_blockwise_equivalence(lords, path):
+    lay, s = gen.make_blockwise_layer(256, 256, 64, 4, bits=4, seed=0)
+    dl, y32, ybf = _run(lords, lay, path)
+    check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("bits,m,n,r,M", [(4, 160, 256, 5, 3), (3, 131, 192, 7, 2), (4, 256, 512, 32, 16),
+                                          (3, 256, 1024, 48, 1), (2, 64, 128, 3, 2)])
+def test_integer_case_is_bit_exact(lords, path, bits, m, n, r, M):
+    lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m)
+    dl, y32, ybf = _run(lords, lay, path)
+    y64 = _oracle(lay, dl.packed_host)
+    assert np.array_equal(y32.astype(np.float64), y64)
+    assert np.array_equal(ybf, oracle.round_bf16(y64))
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("bits,m,n,r,M,mixed", [
+    (4, 37, 66, 5, 3, True),        # nothing a multiple of a tile; r odd
+    (4, 300, 1000, 24, 19, False),  # several token tiles with a ragged tail
+    (3, 129, 352, 12, 9, True),     # 3-bit stream, n = 11 groups of 32
+    (3, 512, 2048, 48, 16, False),
+    (2, 96, 260, 2, 5, True),
+    (4, 64, 4096, 128, 2, False),   # largest rank
+    (4, 1, 2, 1, 1, False),         # smallest legal problem
+])
+def test_odd_shapes(lords, path, bits, m, n, r, M, mixed):
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=7 * m + n, mixed_sign=mixed)
+    dl, y32, ybf = _run(lords, lay, path)
+    check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
+
+
+@pytest.mark.parametrize("splitk", [1, 2, 5, 64])
+def test_forced_splitk_is_deterministic_and_correct(lords, splitk):
+    lay = gen.make_layer(200, 1536, 8, 3, bits=4, seed=4)
+    lords.lords_set_option("splitk", str(splitk))
+    try:
+        dl, y32, ybf = _run(lords, lay, "simt")
+        y32b, ybfb = dl.forward()
+    finally:
+        lords.lords_set_option("splitk", "0")
+    assert np.array_equal(y32, y32b) and np.array_equal(ybf, ybfb)   # bit-identical run to run
+    check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
+
+
+def test_linearity_on_gpu(lords):
+    import torch
+    m, n, r = 128, 512, 16
+    lay = gen.make_layer(m, n, r, 3, bits=4, seed=21, mixed_sign=True)
+    x = gen.bf16_to_f32(lay.x).copy()
+    x[0, n // 2:] = 0.0
+    x[1, :n // 2] = 0.0
+    x[2] = 4.0 * x[0] - 0.5 * x[1]
+    lay.x = gen.bf16_bits(torch.from_numpy(x))
+    dl, y32, ybf = _run(lords, lay)
+    want = 4.0 * y32[0].astype(np.float64) - 0.5 * y32[1].astype(np.float64)
+    nw, el = error_metrics(y32[2:3], want[None])
+    assert nw <= NORMWISE_TOL and el <= ELEMENT_TOL
+
+
+def _sampled_rows(m, count, seed):
+    rng = np.random.default_rng(seed)
+    rows = np.unique(np.concatenate([[0, m - 1], rng.integers(0, m, size=count)]))
+    return rows.astype(np.int64)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("M", [1, 8])
+def test_config1_qproj_decode_full_size(lords, path, M):
+    lay = gen.make_layer(4096, 4096, 32, M, bits=4, seed=0)
+    dl, y32, ybf = _run(lords, lay, path)
+    y64 = _oracle(lay, dl.packed_host)            # the full layer: ~0.6 GFLOP fp64 per token
+    check_against_oracle(y32, ybf, y64)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("m,n,M", [(14336, 4096, 1), (4096, 14336, 1), (4096, 14336, 16), (14336, 4096, 16)])
+def test_config2_mlp_nf3_full_size(lords, path, m, n, M):
+    lay = gen.make_layer(m, n, 48, M, bits=3, seed=0)
+    dl, y32, ybf = _run(lords, lay, path)
+    rows = _sampled_rows(m, 512, 5)
+    y64 = _oracle(lay, dl.packed_host, rows=rows)
+    check_against_oracle(y32[:, rows], ybf[:, rows], y64)
+    assert np.isfinite(y32).all()
+
+
+@pytest.mark.parametrize("path", ["auto"])
+def test_config3_prefill_full_size_sampled(lords, path):
+    lay = gen.make_layer(4096, 14336, 32, 2048, bits=4, seed=0, outlier_frac=0.01)
+    dl, y32, ybf = _run(lords, lay, path)
+    rows = _sampled_rows(4096, 96, 6)
+    y64 = _oracle(lay, dl.packed_host, rows=rows)
+    check_against_oracle(y32[:, rows], ybf[:, rows], y64)
+    assert np.isfinite(y32).all()
+
+
+def test_host_buffer_entry_point_matches_device_entry(lords):
+    import torch
+    lay = gen.make_layer(512, 1024, 16, 4, bits=4, seed=12)
+    dl, y32, ybf = _run(lords, lay)
+    xh = torch.from_numpy(lay.x.view(np.int16)).pin_memory()
+    yh = torch.zeros((lay.M, lay.m), dtype=torch.int16).pin_memory()
+    lords.lords_linear_forward_host(xh, dl.q, dl.B, dl.A, lay.codebook, lay.bits, lay.M, lay.m, lay.n, lay.r, yh)
+    torch.cuda.synchronize()
+    assert np.array_equal(yh.numpy().view(np.uint16), ybf)
+
+
+def test_four_bit_entry_point_and_launch_count(lords):
+    import torch
+    lay = gen.make_layer(256, 256, 4, 4, bits=4, seed=0)
+    dl, y32, ybf = _run(lords, lay)
+    y = torch.zeros_like(dl.y)
+    lords.lords_linear_forward(dl.x, dl.q, dl.B, dl.A, lay.codebook, lay.M, lay.m, lay.n, lay.r, y)
+    torch.cuda.synchronize()
+    assert np.array_equal(y.cpu().numpy().view(np.uint16), ybf)
+    assert lords.lords_last_launch_count() >= 1
+    assert lords.lords_last_path() in ("simt", "decode", "prefill")
