@@ -150,6 +150,27 @@ int lords_linear_forward_host(const void *x_host, const uint8_t *Qpacked, const 
                               void *stream);
 
 /*
+ * Allocation-free forward (the paper has no counterpart: this is a deployment convenience).
+ * For callers that must not allocate device memory -- for instance a plugin inside a server
+ * whose memory pool already owns all of HBM, or a latency-critical loop that cannot take the
+ * device-wide synchronisation cudaMalloc/cudaFree imply.  Same arguments and result as
+ * lords_linear_forward_bits (device pointers, host codebook, bf16 y), but it needs no
+ * lords_init and calls no allocator: it runs the split-K CUDA-core kernels with their partial
+ * sums in a fixed LORDS_NOALLOC_MAX_FLOATS-float (4 MiB) array inside the library image, which
+ * every GPU that loads the library holds until the process exits.
+ *   - limit: 2 * M * m <= LORDS_NOALLOC_MAX_FLOATS, otherwise LORDS_ERR_WORKSPACE;
+ *   - it works on the calling thread's current CUDA device; the first call on each device also
+ *     resolves the array's device address, so make that first call outside any stream capture;
+ *   - all calls share the one array: every slot a call reads it has written itself, so stale
+ *     contents are harmless, but two calls that overlap on the GPU (different streams) race --
+ *     order them on one stream.
+ */
+#define LORDS_NOALLOC_MAX_FLOATS (1u << 20)
+int lords_linear_forward_noalloc(const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                                 const float *codebook, int bits, int M, int m, int n, int r, void *y,
+                                 void *stream);
+
+/*
  * Read and clear the device status word.  Synchronises `stream` first.  Returns LORDS_OK, or
  * the error a kernel recorded (LORDS_ERR_TIMEOUT when a bounded wait ran out).
  */

@@ -47,6 +47,7 @@ def _load():
         "lords_linear_forward_bits": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_forward_f32": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_forward_host": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
+        "lords_linear_forward_noalloc": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_poll_status": (ci, [p]),
         "lords_last_cuda_error": (ci, []),
         "lords_set_option": (ci, [cs, cs]),
@@ -70,7 +71,7 @@ def exported_symbols():
     return ["lords_version", "lords_strerror", "lords_equivalent_rank", "lords_packed_bytes",
             "lords_pack_codes", "lords_unpack_codes", "lords_init", "lords_shutdown",
             "lords_linear_forward", "lords_linear_forward_bits", "lords_linear_forward_f32",
-            "lords_linear_forward_host", "lords_poll_status", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
+            "lords_linear_forward_host", "lords_linear_forward_noalloc", "lords_poll_status", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
             "lords_last_launch_count"]
 
 
@@ -172,6 +173,14 @@ def lords_linear_forward_host(x_host, Qpacked, B, A, codebook, bits, M, m, n, r,
     _check(_load().lords_linear_forward_host(x_host.data_ptr(), Qpacked.data_ptr(), B.data_ptr(), A.data_ptr(),
                                              cb.ctypes.data, bits, M, m, n, r, y_host.data_ptr(),
                                              _stream_ptr(stream)), "lords_linear_forward_host")
+
+
+def lords_linear_forward_noalloc(x, Qpacked, B, A, codebook, bits, M, m, n, r, y, stream=None) -> None:
+    """Forward that never allocates and needs no lords_init (scratch lives in the library image)."""
+    cb = _cb_ptr(codebook, bits)
+    _check(_load().lords_linear_forward_noalloc(x.data_ptr(), Qpacked.data_ptr(), B.data_ptr(), A.data_ptr(),
+                                                cb.ctypes.data, bits, M, m, n, r, y.data_ptr(),
+                                                _stream_ptr(stream)), "lords_linear_forward_noalloc")
 
 
 def lords_poll_status(stream=None) -> int:

@@ -243,3 +243,105 @@ int launch_simt(const Problem &p, State &st, cudaStream_t stream)
 }
 
 }  // namespace lords
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free entry point.
+//
+// Some hosts of this library may not allocate device memory at all: a plugin loaded into an
+// inference server that has already handed every byte of HBM to its own pool (cudaMalloc then
+// fails or steals from that pool), or a latency-critical loop that cannot afford the implicit
+// device-wide synchronisation cudaMalloc and cudaFree perform.  Such callers cannot use
+// lords_init, whose job is to allocate the scratch workspace.  For them the split-K forward
+// above is offered with its partial sums kept in a fixed array that is part of the loaded
+// module image: every GPU that loads the library holds these 4 MiB until the process exits.
+//
+// In host code the array's name is only a stand-in for the device object, so its device address
+// is looked up once per device with cudaGetSymbolAddress (that device being current) and that
+// pointer is what the kernels receive.
+// ---------------------------------------------------------------------------------------------
+namespace lords {
+namespace {
+
+constexpr size_t kNoAllocFloats = LORDS_NOALLOC_MAX_FLOATS;
+static __device__ __align__(256) float g_noalloc_partials[kNoAllocFloats];
+
+constexpr int kMaxDevices = 64;
+float *g_noalloc_ptr[kMaxDevices] = {};   // device address of g_noalloc_partials, per device
+int g_noalloc_sms[kMaxDevices] = {};
+
+}  // namespace
+}  // namespace lords
+
+extern "C" int lords_linear_forward_noalloc(const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                                            const float *codebook, int bits, int M, int m, int n, int r,
+                                            void *y, void *stream)
+{
+    using namespace lords;
+    if (!x || !Qpacked || !B || !A || !codebook || !y) return LORDS_ERR_NULL;
+    if (bits != 2 && bits != 3 && bits != 4) return LORDS_ERR_BITS;
+    const int group = bits == 4 ? 2 : (bits == 3 ? 32 : 4);
+    if (M < 1 || M > LORDS_M_MAX || m < 1 || n < 1 || r < 1 || r > LORDS_R_MAX || n % group != 0)
+        return LORDS_ERR_SHAPE;
+    const uintptr_t all = (uintptr_t)x | (uintptr_t)Qpacked | (uintptr_t)B | (uintptr_t)A | (uintptr_t)y;
+    if (all & 15u) return LORDS_ERR_ALIGN;
+    // two partial copies of the output are the least this variant needs
+    if (2 * (size_t)M * (size_t)m > kNoAllocFloats) return LORDS_ERR_WORKSPACE;
+
+    int dev = -1;
+    LORDS_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return LORDS_ERR_SHAPE;
+    if (g_noalloc_ptr[dev] == nullptr) {
+        // one-time set-up for this device (it is the current one): resolve the array's device address
+        float *ptr = nullptr;
+        LORDS_CUDA_TRY(cudaGetSymbolAddress((void **)&ptr, g_noalloc_partials));
+        int sms = 0;
+        LORDS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        g_noalloc_sms[dev] = sms;
+        g_noalloc_ptr[dev] = ptr;
+    }
+
+    SimtParams k;
+    k.x = static_cast<const uint16_t *>(x); k.q = Qpacked;
+    k.B = static_cast<const uint16_t *>(B); k.A = static_cast<const uint16_t *>(A);
+    for (int c = 0; c < 16; ++c) k.levels[c] = c < (1 << bits) ? codebook[c] : 0.0f;
+    k.bits = bits; k.M = M; k.m = m; k.n = n; k.r = r;
+    k.y = y; k.y_f32 = 0;
+
+    const int row_ctas = (m + kRowsPerCta - 1) / kRowsPerCta;
+    const int tok_tiles = (M + kTokTile - 1) / kTokTile;
+    if (tok_tiles > 65535) return LORDS_ERR_SHAPE;
+    const int nchunks = (n + kChunk - 1) / kChunk;
+    const long base = (long)row_ctas * tok_tiles;
+    int splits = (int)((4L * g_noalloc_sms[dev] + base - 1) / base);
+    if (splits > nchunks / 4) splits = nchunks / 4;
+    const size_t fit = kNoAllocFloats / ((size_t)M * m);      // >= 2, checked above
+    if ((size_t)splits > fit) splits = (int)fit;
+    if (splits < 2) splits = 2;                               // always the scratch-using variant
+    if (splits > nchunks) splits = nchunks;                   // a single chunk: one split, via scratch all the same
+    k.chunks_per_split = (nchunks + splits - 1) / splits;
+    splits = (nchunks + k.chunks_per_split - 1) / k.chunks_per_split;
+    k.splits = splits;
+    k.partial = g_noalloc_ptr[dev];
+
+    const size_t smem = ((size_t)r * kChunk + kTokTile * kChunk + (size_t)kRowsPerCta * r) * sizeof(float);
+    if (smem > 48 * 1024)
+        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (splits > 1) {
+        lords_simt_kernel<<<dim3(row_ctas, splits, tok_tiles), kWarps * 32, smem, s>>>(k);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        const size_t count = (size_t)M * m;
+        lords_splitk_reduce_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(k.partial, splits, count, y, 0);
+        LORDS_CUDA_TRY(cudaGetLastError());
+    } else {
+        // n fits one chunk: the lone split still lands in the static array, then is rounded out of it
+        k.splits = 2;  // makes the kernel take its "write partials" branch; slice 1 is never produced
+        k.chunks_per_split = nchunks;
+        lords_simt_kernel<<<dim3(row_ctas, 1, tok_tiles), kWarps * 32, smem, s>>>(k);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        const size_t count = (size_t)M * m;
+        lords_splitk_reduce_kernel<<<(unsigned)((count + 255) / 256), 256, 0, s>>>(k.partial, 1, count, y, 0);
+        LORDS_CUDA_TRY(cudaGetLastError());
+    }
+    return LORDS_OK;
+}
