@@ -73,8 +73,12 @@ static int forward_common(const void *x, const uint8_t *q, const void *B, const 
 
     // Dispatch.  The tensor-core paths decline (LORDS_ERR_UNSUPPORTED) shapes outside their
     // tiling rules; "auto" then falls back to the generic CUDA-core path.
-    if (st.forced_path == 1 || st.forced_path == 0) return launch_simt(p, st, s);
-    return LORDS_ERR_UNSUPPORTED;
+    if (st.forced_path != 1) {
+        rc = launch_umma(p, st, s);
+        if (rc != LORDS_ERR_UNSUPPORTED && rc != LORDS_ERR_WORKSPACE) return rc;
+        if (st.forced_path != 0) return rc;
+    }
+    return launch_simt(p, st, s);
 }
 
 }  // namespace lords
@@ -187,8 +191,11 @@ int lords_init(int device, size_t workspace_bytes)
     if (workspace_bytes == 0) workspace_bytes = (size_t)256 << 20;
     LORDS_CUDA_TRY(cudaMalloc(&st.workspace, workspace_bytes));
     st.workspace_bytes = workspace_bytes;
-    cudaError_t e = cudaMalloc(&st.status_word, 256);
-    if (e == cudaSuccess) e = cudaMemset(st.status_word, 0, 256);
+    st.counter_slots = 16384;
+    const size_t small_bytes = 256 + sizeof(int) * (size_t)st.counter_slots;
+    cudaError_t e = cudaMalloc(&st.status_word, small_bytes);
+    if (e == cudaSuccess) e = cudaMemset(st.status_word, 0, small_bytes);
+    st.counters = st.status_word + 64;
     if (e != cudaSuccess) {
         cudaFree(st.workspace);
         st.workspace = nullptr;

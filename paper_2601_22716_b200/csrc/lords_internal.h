@@ -30,6 +30,8 @@ struct State {
     uint8_t *workspace = nullptr;   // scratch: split-K partials / converted activations
     size_t workspace_bytes = 0;
     int *status_word = nullptr;     // device int, 0 = OK, else a LORDS_ERR_* a kernel recorded
+    int *counters = nullptr;        // split-K arrival counters, zero between calls
+    int counter_slots = 0;
     uint8_t *stage_x = nullptr;     // device staging for the host-buffer entry point
     uint8_t *stage_y = nullptr;
     size_t stage_x_bytes = 0, stage_y_bytes = 0;
@@ -53,5 +55,8 @@ int cuda_fail(cudaError_t e);
 
 // Generic CUDA-core path: any shape the interface accepts.
 int launch_simt(const Problem &p, State &st, cudaStream_t stream);
+
+// Tensor-core path (TMA + tcgen05/TMEM).  LORDS_ERR_UNSUPPORTED for shapes outside its rules.
+int launch_umma(const Problem &p, State &st, cudaStream_t stream);
 
 }  // namespace lords
