@@ -65,7 +65,19 @@ struct alignas(64) UmmaParams {
     void *y;
     int y_f32;
     int *status;
+#ifdef LORDS_TRACE
+    long long *trace;     // [3 roles][64 iterations][8 events] clock64 stamps of CTA 0 (debug builds only)
+#endif
 };
+
+#ifdef LORDS_TRACE
+#define LORDS_STAMP(role, it, ev)                                                        \
+    do {                                                                                 \
+        if (blockIdx.x == 0 && (it) < 64) p.trace[((role) * 64 + (it)) * 8 + (ev)] = clock64(); \
+    } while (0)
+#else
+#define LORDS_STAMP(role, it, ev) do { } while (0)
+#endif
 
 __device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float v)
 {
@@ -193,12 +205,14 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                     failed = true;
                     break;
                 }
+                LORDS_STAMP(2, it, 0);
                 const int j0 = (kb0 + it) * BK;
                 const uint32_t bar = bar_tma_full + 8 * st;
                 mbar_expect_tx(bar, stage_tx);
                 tma_load_2d(q_tile0 + st * kQTileBytes, &p.tm_q, j0 / 2, row0, bar);
                 tma_load_2d(a_tile0 + st * kATileBytes, &p.tm_a, j0, 0, bar);
                 tma_load_2d(x_tile0 + st * C::kXTileBytes, &p.tm_x, j0, tok0, bar);
+                LORDS_STAMP(2, it, 1);
             }
         }
     } else if (warp == kMmaWarp) {
@@ -223,8 +237,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             if (ok && nkb > 1) ok = issue_scale(1);
             for (int it = 0; ok && it < nkb; ++it) {
                 const int st = it % STAGES, buf = it & 1;
+                LORDS_STAMP(0, it, 0);
                 if (!mbar_wait(bar_w_full + 8 * buf, (uint32_t)((it >> 1) & 1))) { ok = false; break; }
                 tc_fence_after_sync();
+                LORDS_STAMP(0, it, 1);
 #pragma unroll
                 for (int k = 0; k < BK / 16; ++k) {
                     const uint64_t ad = umma_desc_sw128(w_tile0 + buf * kWTileBytes + k * 32, 1024, 16);
@@ -233,7 +249,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 }
                 umma_commit(bar_tma_empty + 8 * st);
                 umma_commit(bar_w_empty + 8 * buf);
+                LORDS_STAMP(0, it, 2);
                 if (it + 2 < nkb) ok = issue_scale(it + 2);
+                LORDS_STAMP(0, it, 3);
             }
             umma_commit(bar_acc_full);
             failed = !ok;
@@ -246,8 +264,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         const __half2 *lut = sm_lut + lane;
         for (int it = 0; it < nkb; ++it) {
             const int st = it % STAGES, buf = it & 1;
+            if (tid == 0) LORDS_STAMP(1, it, 0);
             if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * buf, (uint32_t)((it >> 1) & 1)))) { failed = true; break; }
             tc_fence_after_sync();
+            if (tid == 0) LORDS_STAMP(1, it, 1);
             uint32_t s[32];
             tmem_ld_32x32(lane_addr + kSCol + buf * 64 + half * 32, s);
             if (!__all_sync(0xffffffffu, mbar_wait(bar_tma_full + 8 * st, (uint32_t)((it / STAGES) & 1)))) {
@@ -257,6 +277,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             }
             const uint4 cw = *reinterpret_cast<const uint4 *>(sm_q + st * kQTileBytes + row * 32 + half * 16);
             tmem_wait_ld();
+            if (tid == 0) LORDS_STAMP(1, it, 2);
             const uint32_t cwv[4] = {cw.x, cw.y, cw.z, cw.w};
             uint32_t out[16];
 #pragma unroll
@@ -271,6 +292,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 failed = true;
                 break;
             }
+            if (tid == 0) LORDS_STAMP(1, it, 3);
             uint8_t *wrow = sm_w + buf * kWTileBytes + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -278,9 +300,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 *reinterpret_cast<uint4 *>(wrow + chunk * 16) =
                     make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
             }
+            if (tid == 0) LORDS_STAMP(1, it, 4);
             fence_proxy_async_smem();
             tc_fence_before_sync();
+            if (tid == 0) LORDS_STAMP(1, it, 5);
             mbar_arrive(bar_w_full + 8 * buf);
+            if (tid == 0) LORDS_STAMP(1, it, 6);
         }
 
         // ------------------------------------------------------------------ epilogue
@@ -451,6 +476,10 @@ int launch_umma(const Problem &p, State &st, cudaStream_t stream)
     k.counters = st.counters;
     k.y = p.y; k.y_f32 = p.y_f32;
     k.status = st.status_word;
+#ifdef LORDS_TRACE
+    k.trace = reinterpret_cast<long long *>(st.workspace + st.workspace_bytes - (size_t)3 * 64 * 8 * 8);
+    LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)3 * 64 * 8 * 8, stream));
+#endif
 
     if (!make_map_2d(&k.tm_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, x16, (uint64_t)p.n, (uint64_t)p.M, 64, (uint32_t)BN,
                      CU_TENSOR_MAP_SWIZZLE_128B) ||
@@ -479,5 +508,18 @@ int launch_umma(const Problem &p, State &st, cudaStream_t stream)
     st.last_path = p.M <= 16 ? "decode" : "prefill";
     return LORDS_OK;
 }
+
+#ifdef LORDS_TRACE
+// Debug builds only: copy CTA 0's clock stamps of the last tensor-core launch to the host.
+extern "C" int lords_debug_read_trace(long long *out)
+{
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    LORDS_CUDA_TRY(cudaDeviceSynchronize());
+    LORDS_CUDA_TRY(cudaMemcpy(out, st.workspace + st.workspace_bytes - (size_t)3 * 64 * 8 * 8, (size_t)3 * 64 * 8 * 8,
+                              cudaMemcpyDeviceToHost));
+    return LORDS_OK;
+}
+#endif
 
 }  // namespace lords

@@ -78,15 +78,19 @@ def test_odd_shapes(lords, path, bits, m, n, r, M, mixed):
     check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
 
 
+@pytest.mark.parametrize("path", PATHS)
 @pytest.mark.parametrize("splitk", [1, 2, 5, 64])
-def test_forced_splitk_is_deterministic_and_correct(lords, splitk):
+def test_forced_splitk_is_deterministic_and_correct(lords, splitk, path):
     lay = gen.make_layer(200, 1536, 8, 3, bits=4, seed=4)
     lords.lords_set_option("splitk", str(splitk))
+    lords.lords_set_option("path", path)
     try:
-        dl, y32, ybf = _run(lords, lay, "simt")
+        dl = DeviceLayer(lay)
+        y32, ybf = dl.forward()
         y32b, ybfb = dl.forward()
     finally:
         lords.lords_set_option("splitk", "0")
+        lords.lords_set_option("path", "auto")
     assert np.array_equal(y32, y32b) and np.array_equal(ybf, ybfb)   # bit-identical run to run
     check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
 
