@@ -180,12 +180,13 @@ int lords_poll_status(void *stream);
 int lords_last_cuda_error(void);
 
 /*
- * Measurement switches.  Keys: "path" = "auto" | "simt" | "decode" | "prefill";
+ * Measurement switches.  Keys: "path" = "auto" | "simt" | "decode" (reassociated-form kernel,
+ * M <= 2) | "umma" (scale-MMA kernel; "prefill" is an alias);
  * "splitk" = "0" (auto) or a positive integer.  Unknown keys: LORDS_ERR_OPTION.
  */
 int lords_set_option(const char *key, const char *value);
 
-/* Name of the path the most recent forward call dispatched to ("simt", "decode", "prefill"). */
+/* Name of the path the most recent forward call dispatched to ("simt", "decode", "umma"). */
 const char *lords_last_path(void);
 
 /* Number of kernels the most recent forward call launched. */

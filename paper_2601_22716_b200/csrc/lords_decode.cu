@@ -1,0 +1,665 @@
+// Decode path (M <= 2 tokens) on tcgen05/TMEM, reassociated form of W^ = L[Q] (.) (BA):
+//
+//     z[t][i][k] = sum_j L[Q_ij] * (A_kj * x_tj)          (one GEMM, N = M * r columns)
+//     y[t][i]    = sum_k B_ik * z[t][i][k]                 (a row dot product in the epilogue)
+//
+// which equals y = x (L[Q] (.) (BA))^T with S = BA of Eq. 3 never formed: the scale factors
+// ride on the small operand, so the big operand is the bare level table lookup of the codes.
+//
+// A thread-block cluster owns one tile of 128 * H rows of Q (H = 1 or 2); its CTAs split the tile's
+// k-steps (128 in-feature columns each) evenly, and the host picks H and the cluster size so that
+// all clusters are resident at once and fill the SMs.  Each CTA parks its partial y in the cluster
+// leader's shared memory (distributed shared memory) and arrives on the leader's mbarrier; the
+// leader adds the partials in rank order -- deterministic, no float atomics, no trip through
+// global memory.
+//
+// Warp roles (20 warps):
+//   0..15  worker groups of 4 * H warps take k-steps round-robin.  For its k-step a group
+//          (a) turns the factor tile A[:, k-step] (TMA, shared memory) in place into the fp16 B
+//              operand A_kj * x_tj, and
+//          (b) dequantises: warp (h, q) owns rows h*128 + q*32 .. +31; a thread reads its row's packed
+//              codes from shared memory, looks every code pair up in a lane-private fp16x2 level
+//              table and stores the row straight into TMEM as the A operand (tcgen05.st).
+//          Group 0 also runs the epilogue.
+//   16,17  MMA issuers, one per 128-row half: D_h[128 x N] += W_h[128 x 16] * AX[N x 16]^T with
+//          A from TMEM and B from shared memory, eight per k-step.
+//   18     TMA producer of the packed code tiles (HBM stream, deep ring); it also initialises the
+//          barriers and starts the stream before the rest of the CTA has finished its set-up.
+//   19     TMA producer of the factor tiles.
+//
+// Every wait is bounded; on expiry the role records LORDS_ERR_TIMEOUT and leaves its loop, so
+// the kernel always reaches its final barrier and frees its TMEM.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "lords_internal.h"
+#include "lords_ptx.cuh"
+
+namespace lords {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kWorkWarps = 16;                         // worker warps: 16 / (4 * H) groups of 4 * H
+constexpr int kIssuerWarp0 = kWorkWarps;               // 16, 17 (the second one idles when H == 1)
+constexpr int kTmaQWarp = kIssuerWarp0 + 2;            // 18
+constexpr int kTmaAWarp = kTmaQWarp + 1;               // 19
+constexpr int kWarps = kTmaAWarp + 1;                  // 20
+constexpr int kThreads = kWarps * 32;                  // 640
+constexpr int kNMax = 64;                              // accumulator columns per half (N = M * r_pad)
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kWCol = 2 * kNMax;                  // W ring starts behind the accumulators
+constexpr int kAtomBytes = kNMax * 128;                // one 64-column swizzle atom of the B operand
+constexpr int kClusterMax = 16;                        // largest cluster (split of a tile's k-range) this kernel is launched with
+constexpr int kStep = 128;                             // in-feature columns per k-step
+constexpr int kAtoms = kStep / 64;
+constexpr int kWSlotCols = kStep / 2;                  // TMEM columns of one W slot (fp16 pairs)
+
+// BITS: code width.  H: 128-row halves per CTA tile (1 or 2).
+template <int BITS, int H> struct DCfg {
+    static constexpr int TILE_ROWS = 128 * H;
+    static constexpr int GROUP_WARPS = 4 * H;                  // worker warps on one k-step
+    static constexpr int GROUPS = kWorkWarps / GROUP_WARPS;    // groups take k-steps round-robin (4 / 2)
+    static constexpr int QROW = kStep * BITS / 8;              // packed bytes per row per k-step (64 / 48)
+    static constexpr int QSTAGE = TILE_ROWS * QROW;
+    static constexpr int SQ = (BITS == 4 ? 8 : 12) / H;        // code-tile ring depth: 64 / 72 KB in flight
+    static constexpr int S_TMEM = (512 - (int)kWCol) / (H * kWSlotCols);
+    static constexpr int S = S_TMEM < 4 ? S_TMEM : 4;          // W / factor ring depth (4 / 3)
+    static constexpr int AXSTAGE = kAtoms * kAtomBytes;
+    static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;   // one entry per code pair
+    static constexpr int LUT_BYTES = LUT_ENTRIES * 128;        // 32 lane-private copies
+    static constexpr int RED_BYTES = kClusterMax * 2 * TILE_ROWS * 4;   // the cluster's partials, [rank][token][row]
+    static constexpr int BAR_BYTES = 512;
+    static constexpr int SMEM = LUT_BYTES /*alignment slack*/ + LUT_BYTES + SQ * QSTAGE + S * AXSTAGE + RED_BYTES + BAR_BYTES;
+    // the code ring's depth is a multiple of the group count, so each of its barriers is used by
+    // one group alone, which then sees every phase of it
+    static_assert(SQ % GROUPS == 0, "code ring depth must be a multiple of the group count");
+};
+
+struct alignas(64) DecodeParams {
+    CUtensorMap tm_q;     // u8 [m][n*bits/8], box {QROW, 128 * H}
+    CUtensorMap tm_a;     // bf16 [r][n], box {64, r_pad}, 128-byte swizzle
+    const uint16_t *x;    // bf16 [M][n]
+    const uint16_t *B;    // bf16 [m][r]
+    float levels[16];
+    int M, m, n, r, r_pad;
+    int ksteps;           // k-steps per tile
+    int tiles;
+    void *y;
+    int y_f32;
+    int *status;
+#ifdef LORDS_TRACE
+    long long *trace;     // [8 roles][32 iterations][8 events] clock64 stamps of one CTA (debug builds only)
+#endif
+};
+
+#ifdef LORDS_TRACE
+#ifndef LORDS_TRACE_CTA
+#define LORDS_TRACE_CTA 0
+#endif
+#define DSTAMP(role, it, ev)                                                                         \
+    do {                                                                                             \
+        if (blockIdx.x == LORDS_TRACE_CTA && (it) < 32) p.trace[((role) * 32 + (it)) * 8 + (ev)] = clock64(); \
+    } while (0)
+#else
+#define DSTAMP(role, it, ev) do { } while (0)
+#endif
+
+__device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float v)
+{
+    if (y_f32) static_cast<float *>(y)[idx] = v;
+    else static_cast<__nv_bfloat16 *>(y)[idx] = __float2bfloat16_rn(v);
+}
+
+// One row of one k-step (128 codes): packed codes (shared memory) -> fp16 level pairs -> 64 TMEM columns.
+template <int BITS>
+__device__ __forceinline__ void dequant_row_to_tmem(uint32_t qrow, uint32_t lut_lane, uint32_t taddr)
+{
+    if constexpr (BITS == 4) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const uint4 c0 = lds_v4(qrow + half * 32), c1 = lds_v4(qrow + half * 32 + 16);
+            const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+            uint32_t out[32];
+#pragma unroll
+            for (int wi = 0; wi < 8; ++wi)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    // byte b of the word holds two codes; entry offset = byte * 128
+                    const uint32_t sh = b == 0 ? (w[wi] << 7) : (w[wi] >> (8 * b - 7));
+                    out[wi * 4 + b] = lds_u32((sh & 0x7F80u) | lut_lane);
+                }
+            tmem_st_32x32(taddr + half * 32, out);
+        }
+    } else {
+        const uint4 c0 = lds_v4(qrow), c1 = lds_v4(qrow + 16), c2 = lds_v4(qrow + 32);
+        const uint32_t w[12] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w};
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint32_t out[32];
+#pragma unroll
+            for (int pp = 0; pp < 32; ++pp) {
+                // code pair P sits at bit 6P of the row's 384-bit little-endian stream
+                const int bit = 6 * (half * 32 + pp), wi = bit >> 5, off = bit & 31;
+                uint32_t sh;
+                if (off > 26) sh = __funnelshift_r(w[wi], w[wi + 1 < 12 ? wi + 1 : 11], off - 7);
+                else sh = off >= 7 ? (w[wi] >> (off - 7)) : (w[wi] << (7 - off));
+                out[pp] = lds_u32((sh & 0x1F80u) | lut_lane);
+            }
+            tmem_st_32x32(taddr + half * 32, out);
+        }
+    }
+}
+
+template <int BITS, int NTOK, int H>
+__global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_constant__ DecodeParams p)
+{
+    using C = DCfg<BITS, H>;
+    constexpr int S = C::S, SQ = C::SQ, kTileRows = C::TILE_ROWS, kGroups = C::GROUPS, kGroupWarps = C::GROUP_WARPS;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t lut = (raw + C::LUT_BYTES - 1) & ~(uint32_t)(C::LUT_BYTES - 1);   // table-size aligned: entry offsets OR in
+    const uint32_t q0 = lut + C::LUT_BYTES;
+    const uint32_t ax0 = q0 + SQ * C::QSTAGE;          // multiple of 1024
+    const uint32_t red0 = ax0 + S * C::AXSTAGE;        // [kClusterMax][NTOK][rows] floats: the cluster's partials (leader's copy is used)
+    const uint32_t bars = red0 + C::RED_BYTES;
+    // mbarriers, 8 bytes each, in one run so that a warp can initialise them lane-parallel
+    constexpr int kBarQFull = 0;                            // SQ, 1 arrival + TMA bytes
+    constexpr int kBarQEmpty = kBarQFull + SQ;              // SQ, the warps of one group
+    constexpr int kBarAFull = kBarQEmpty + SQ;              // S, 1 arrival + TMA bytes
+    constexpr int kBarReady = kBarAFull + S;                // H * S: the warps of one group (W slot and B operand written)
+    constexpr int kBarMmaDone = kBarReady + H * S;          // S, one commit per issuer
+    constexpr int kBarAccFull = kBarMmaDone + S;            // H
+    constexpr int kBarReduce = kBarAccFull + H;             // 1: every epilogue warp of every CTA of the cluster
+    constexpr int kBarCount = kBarReduce + 1;
+    static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
+    const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
+    const uint32_t bar_a_full = bars + 8 * kBarAFull, bar_ready = bars + 8 * kBarReady;
+    const uint32_t bar_mma_done = bars + 8 * kBarMmaDone, bar_acc_full = bars + 8 * kBarAccFull;
+    const uint32_t bar_reduce = bars + 8 * kBarReduce;
+    const uint32_t tmem_slot = bars + 8 * kBarCount;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // The cluster shares one tile of 128 * H rows; rank r takes the r-th slice of its k-steps.
+    const int csize = (int)cluster_nctarank(), rank = (int)cluster_ctarank();
+    const int tile = (int)blockIdx.x / csize;
+    const int ks_a = (int)((long long)rank * p.ksteps / csize);
+    const int ks_b = (int)((long long)(rank + 1) * p.ksteps / csize);
+    const int total = ks_b - ks_a;
+    const int N = NTOK * p.r_pad;
+
+    if (tid == 0) DSTAMP(7, 0, 0);
+    bool failed = false;
+
+    if (warp == kTmaQWarp) {
+        // ------------------------------------------------------------------ code tiles (HBM stream)
+        // This warp initialises every barrier, releases the rest of the CTA and starts the stream of
+        // code tiles at once: the packed codes are weights, nothing in this launch or an earlier one
+        // produces them.
+        for (int b = lane; b < kBarCount; b += 32) {
+            uint32_t count = 1;
+            if (b >= kBarQEmpty && b < kBarAFull) count = kGroupWarps;
+            else if (b >= kBarReady && b < kBarMmaDone) count = kGroupWarps;
+            else if (b >= kBarMmaDone && b < kBarAccFull) count = H;
+            else if (b == kBarReduce) count = (uint32_t)(kGroupWarps * csize);
+            mbar_init(bars + 8 * b, count);
+        }
+        fence_mbar_init();
+        __syncwarp();
+        asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");   // barriers exist; does not wait for the others
+        // split-phase cluster barrier: arrive now (this CTA's reduce barrier exists); the wait is in
+        // the epilogue, right before the first access to the leader's shared memory
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        if (lane == 0) {
+            DSTAMP(7, 0, 3);
+            tma_prefetch_desc(&p.tm_q);
+            for (int it = 0; it < total; ++it) {
+                const int sq = it % SQ;
+                if (it >= SQ && !mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1))) { failed = true; break; }
+                const uint32_t bar = bar_q_full + 8 * sq;
+                DSTAMP(3, it, 0);
+                mbar_expect_tx(bar, (uint32_t)C::QSTAGE);
+                tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (ks_a + it) * C::QROW, tile * kTileRows, bar);
+            }
+        }
+    } else {
+        if (warp == kIssuerWarp0) {
+            tmem_alloc(tmem_slot, kTmemCols);
+            tmem_relinquish();
+            if (lane == 0) DSTAMP(7, 0, 4);
+        } else if (warp == kTmaAWarp) {
+            if (lane == 0) tma_prefetch_desc(&p.tm_a);
+        } else if (warp < kWorkWarps) {
+            // level-pair table: entry e = (L[lo code], L[hi code]) as fp16x2; word e*32 + lane is lane's
+            // copy (bank = lane, so the lookups of a warp never conflict)
+            for (int e = tid; e < C::LUT_ENTRIES * 32; e += kWorkWarps * 32) {
+                const int entry = e >> 5;
+                const int lo = BITS == 4 ? (entry & 15) : (entry & 7);
+                const int hi = BITS == 4 ? (entry >> 4) : (entry >> 3);
+                const __half2 v = __floats2half2_rn(p.levels[lo], p.levels[hi]);
+                sts_u32(lut + 4u * (uint32_t)e, *reinterpret_cast<const uint32_t *>(&v));
+            }
+            if (tid == 0) DSTAMP(7, 0, 5);
+        }
+        tc_fence_before_sync();
+        asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");   // table, TMEM address and barriers are in place
+        tc_fence_after_sync();
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // see above
+    }
+    if (tid == 0) DSTAMP(7, 0, 1);
+
+    if (warp == kTmaQWarp) {
+        // all done above
+    } else if (warp == kTmaAWarp) {
+        // ------------------------------------------------------------------ factor tiles A[:, k-step]
+        if (lane == 0) {
+            const uint32_t tx = (uint32_t)(kAtoms * p.r_pad * 128);
+            for (int it = 0; it < total; ++it) {
+                const int s = it % S;
+                if (it >= S && !mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1))) { failed = true; break; }
+                const uint32_t bar = bar_a_full + 8 * s;
+                mbar_expect_tx(bar, tx);
+#pragma unroll
+                for (int at = 0; at < kAtoms; ++at)
+                    tma_load_2d(ax0 + s * C::AXSTAGE + at * kAtomBytes, &p.tm_a, (ks_a + it) * kStep + at * 64, 0, bar);
+            }
+        }
+    } else if (warp >= kIssuerWarp0 + H) {
+        // spare issuer warp of the one-half configuration: nothing to do
+    } else if (warp >= kIssuerWarp0) {
+        // ------------------------------------------------------------------ MMA issuer of half h
+        const int h = warp - kIssuerWarp0;
+        uint32_t tmem_base;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+        const uint32_t idesc = (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);  // fp16 x fp16 -> fp32, K-major
+        const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
+        const uint32_t ax_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((ax0 & 0x3FFFFu) >> 4);
+        const uint32_t acc = tmem_base + (uint32_t)(h * kNMax);
+        for (int it = 0; it < total; ++it) {
+            const int s = it % S;
+            if (h == 0 && lane == 0) DSTAMP(0, it, 0);
+            if (!mbar_wait(bar_ready + 8 * (h * S + s), (uint32_t)((it / S) & 1))) { failed = true; break; }
+            tc_fence_after_sync();
+            if (h == 0 && lane == 0) DSTAMP(0, it, 1);
+            if (lane == 0) {
+                const uint32_t wslot = tmem_base + kWCol + (uint32_t)((h * S + s) * kWSlotCols);
+                const uint32_t b_lo = ax_lo0 + (uint32_t)(s * (C::AXSTAGE >> 4));
+#pragma unroll
+                for (int k = 0; k < kStep / 16; ++k)
+                    umma_f16_ts(acc, wslot + k * 8, umma_desc_pack(b_lo + (k >> 2) * (kAtomBytes >> 4) + (k & 3) * 2, desc_hi),
+                                idesc, (it == 0 && k == 0) ? 0u : 1u);
+                umma_commit(bar_mma_done + 8 * s);
+                if (it == total - 1) umma_commit(bar_acc_full + 8 * h);
+                if (h == 0) DSTAMP(0, it, 2);
+            }
+            __syncwarp();
+        }
+    } else {
+        // ------------------------------------------------------------------ worker warps
+        const int g = warp / kGroupWarps, wg = warp % kGroupWarps, h = (warp >> 2) % H, q = warp & 3;
+        const int row_in_tile = h * 128 + q * 32 + lane;
+        uint32_t tmem_base;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t lut_lane = lut + 4u * (uint32_t)lane;
+        const bool stamper = wg == 0 && lane == 0 && g < 2;
+        // B-operand share of this lane: the 16-byte chunk c16 (8 columns) of rows rsub + kRowStep * i
+        const int c16 = lane & 7, rsub = wg * 4 + (lane >> 3);
+        constexpr int kRowStep = 4 * kGroupWarps;                        // 16 / 32
+        constexpr int kRowIters = (kNMax + kRowStep - 1) / kRowStep;     // 4 / 2
+
+        uint4 xr[NTOK][kAtoms];
+        auto load_x = [&](int ks) {
+#pragma unroll
+            for (int t = 0; t < NTOK; ++t)
+#pragma unroll
+                for (int at = 0; at < kAtoms; ++at) {
+                    const int j = ks * kStep + at * 64 + c16 * 8;
+                    xr[t][at] = j < p.n ? __ldg(reinterpret_cast<const uint4 *>(p.x + (size_t)t * p.n + j))
+                                        : make_uint4(0, 0, 0, 0);
+                }
+        };
+        // x may be the previous launch's output: everything above this line only touched weights
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (g < total) load_x(ks_a + g);
+
+        for (int it = g; it < total; it += kGroups) {
+            const int sq = it % SQ, s = it % S;
+            if (stamper) DSTAMP(1 + g, it, 0);
+            // order matters for the factor ring when its depth is odd: the MMA of step it - S being
+            // complete implies the factor tile of step it - S had landed, so the phase of a_full
+            // waited on next is the one for this step
+            bool ok = true;
+            if (it >= S) ok = mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1));
+            if (ok) ok = mbar_wait(bar_a_full + 8 * s, (uint32_t)((it / S) & 1));
+            if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+            tc_fence_after_sync();
+            if (stamper) DSTAMP(1 + g, it, 1);
+
+            // (a) B operand: A_kj * x_tj as fp16, in place (token 0) and behind it (token 1)
+#pragma unroll
+            for (int at = 0; at < kAtoms; ++at) {
+                const uint32_t atom = ax0 + s * C::AXSTAGE + at * kAtomBytes;
+                uint4 av[kRowIters];
+#pragma unroll
+                for (int i = 0; i < kRowIters; ++i) {
+                    const int k = rsub + kRowStep * i;
+                    if (k < p.r_pad) av[i] = lds_v4(atom + k * 128 + ((c16 ^ (k & 7)) << 4));
+                }
+                float xf[NTOK][8];
+#pragma unroll
+                for (int t = 0; t < NTOK; ++t) {
+                    const uint32_t xw[4] = {xr[t][at].x, xr[t][at].y, xr[t][at].z, xr[t][at].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        xf[t][2 * e] = __uint_as_float(xw[e] << 16);
+                        xf[t][2 * e + 1] = __uint_as_float(xw[e] & 0xFFFF0000u);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < kRowIters; ++i) {
+                    const int k = rsub + kRowStep * i;
+                    if (k < p.r_pad) {
+                        const uint32_t addr = atom + k * 128 + ((c16 ^ (k & 7)) << 4);
+                        const uint32_t aw4[4] = {av[i].x, av[i].y, av[i].z, av[i].w};
+#pragma unroll
+                        for (int t = 0; t < NTOK; ++t) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __half2 hv = __floats2half2_rn(__uint_as_float(aw4[e] << 16) * xf[t][2 * e],
+                                                                     __uint_as_float(aw4[e] & 0xFFFF0000u) * xf[t][2 * e + 1]);
+                                o[e] = *reinterpret_cast<const uint32_t *>(&hv);
+                            }
+                            sts_v4(addr + t * p.r_pad * 128, make_uint4(o[0], o[1], o[2], o[3]));
+                        }
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            if (it + kGroups < total) load_x(ks_a + it + kGroups);   // the group's next k-step
+            if (stamper) DSTAMP(1 + g, it, 2);
+
+            // (b) codes -> levels -> TMEM
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1)))) { failed = true; break; }
+            dequant_row_to_tmem<BITS>(q0 + sq * C::QSTAGE + row_in_tile * C::QROW, lut_lane,
+                                      lane_addr + kWCol + (uint32_t)((h * S + s) * kWSlotCols));
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+#pragma unroll
+                for (int hh = 0; hh < H; ++hh) mbar_arrive(bar_ready + 8 * (hh * S + s));
+                mbar_arrive(bar_q_empty + 8 * sq);
+            }
+            if (stamper) DSTAMP(1 + g, it, 3);
+        }
+
+        // Epilogue (group 0): z (TMEM) . B row -> this CTA's partial y, parked in the cluster
+        // leader's shared memory; the leader adds the cluster's partials in rank order.
+        if (g == 0 && !failed) {
+            const int i = tile * kTileRows + row_in_tile;
+            if (stamper) DSTAMP(5, 0, 0);
+            // B row first, so its latency hides behind the wait for the last MMAs
+            uint4 bq[kNMax / 8];
+#pragma unroll
+            for (int c = 0; c < kNMax / 8; ++c)
+                bq[c] = (i < p.m && c * 8 < p.r) ? __ldg(reinterpret_cast<const uint4 *>(p.B + (size_t)i * p.r) + c)
+                                                 : make_uint4(0, 0, 0, 0);
+            float yt[NTOK];
+#pragma unroll
+            for (int t = 0; t < NTOK; ++t) yt[t] = 0.0f;
+            bool ok = true;
+            if (total > 0) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * h, 0));
+                tc_fence_after_sync();
+                if (stamper) DSTAMP(5, 0, 1);
+                if (ok) {
+#pragma unroll
+                    for (int t = 0; t < NTOK; ++t) {
+                        float a = 0.0f;
+#pragma unroll
+                        for (int c = 0; c < kNMax / 16; ++c) {
+                            if (c * 16 < p.r_pad) {   // warp-uniform
+                                uint32_t v[16];
+                                tmem_ld_32x16(lane_addr + (uint32_t)(h * kNMax + t * p.r_pad + c * 16), v);
+                                tmem_wait_ld();
+                                const uint32_t bw[8] = {bq[2 * c].x, bq[2 * c].y, bq[2 * c].z, bq[2 * c].w,
+                                                        bq[2 * c + 1].x, bq[2 * c + 1].y, bq[2 * c + 1].z, bq[2 * c + 1].w};
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) {
+                                    a = fmaf(__uint_as_float(v[2 * e]), __uint_as_float(bw[e] << 16), a);
+                                    a = fmaf(__uint_as_float(v[2 * e + 1]), __uint_as_float(bw[e] & 0xFFFF0000u), a);
+                                }
+                            }
+                        }
+                        yt[t] = a;
+                    }
+                }
+            }
+            if (stamper) DSTAMP(5, 0, 2);
+            if (!ok) failed = true;
+            if (csize == 1) {
+                if (ok && i < p.m)
+#pragma unroll
+                    for (int t = 0; t < NTOK; ++t) store_out(p.y, p.y_f32, (size_t)t * p.m + i, yt[t]);
+            } else {
+                // a CTA that gave up still arrives (with zeros), so the leader never waits in vain
+                asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+#pragma unroll
+                for (int t = 0; t < NTOK; ++t)
+                    st_cluster_f32(map_to_rank(red0 + ((rank * NTOK + t) * kTileRows + row_in_tile) * 4, 0), yt[t]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_rank(bar_reduce, 0));
+                if (stamper) DSTAMP(5, 0, 3);
+                if (rank == 0) {
+                    if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0))) failed = true;
+                    else if (i < p.m) {
+#pragma unroll
+                        for (int t = 0; t < NTOK; ++t) {
+                            float a = 0.0f;
+                            for (int rr = 0; rr < csize; ++rr)
+                                a += __uint_as_float(lds_u32(red0 + ((rr * NTOK + t) * kTileRows + row_in_tile) * 4));
+                            store_out(p.y, p.y_f32, (size_t)t * p.m + i, a);
+                        }
+                    }
+                    if (stamper) DSTAMP(5, 0, 4);
+                }
+            }
+        }
+    }
+
+    if (failed) atomicExch(p.status, LORDS_ERR_TIMEOUT);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) DSTAMP(7, 0, 2);
+    if (warp == kIssuerWarp0) {
+        tc_fence_after_sync();
+        uint32_t tmem_base;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *ptr, uint64_t inner,
+                 uint64_t outer, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swz)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {inner * (uint64_t)elem_bytes};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// One (code width, tokens, halves) instantiation: its launch attributes, how many clusters of each
+// size the device can hold at once, and the launch itself.
+template <int BITS, int NTOK, int H> struct DecodeVariant {
+    static int prepare()
+    {
+        static bool done = false;
+        if (!done) {
+            auto kernel = lords_decode_kernel<BITS, NTOK, H>;
+            LORDS_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DCfg<BITS, H>::SMEM));
+            // cluster sizes above 8 are outside the portable range; they are used only where the
+            // occupancy query below says such a cluster fits
+            LORDS_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+            done = true;
+        }
+        return LORDS_OK;
+    }
+    static void fill(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int cs, int clusters, cudaStream_t stream)
+    {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg = cudaLaunchConfig_t{};
+        cfg.gridDim = dim3((unsigned)(clusters * cs));
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = DCfg<BITS, H>::SMEM;
+        cfg.stream = stream;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+    // Clusters of `cs` CTAs that can be resident at the same time (0 if such a cluster cannot run).
+    static int max_clusters(int cs)
+    {
+        static int cache[kClusterMax + 1];   // 0 = not asked yet, -1 = cannot run
+        if (cache[cs] == 0) {
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attr[1];
+            fill(cfg, attr, cs, 1, nullptr);
+            int n = 0;
+            const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_decode_kernel<BITS, NTOK, H>, &cfg);
+            if (e != cudaSuccess) (void)cudaGetLastError();
+            cache[cs] = (e == cudaSuccess && n >= 1) ? n : -1;
+        }
+        return cache[cs] > 0 ? cache[cs] : 0;
+    }
+    static int launch(const DecodeParams &k, int tiles, int cs, cudaStream_t stream)
+    {
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attr[1];
+        fill(cfg, attr, cs, tiles, stream);
+        LORDS_CUDA_TRY(cudaLaunchKernelEx(&cfg, lords_decode_kernel<BITS, NTOK, H>, k));
+        return LORDS_OK;
+    }
+};
+
+// Cluster size for `tiles` tiles of `ksteps` k-steps: the largest split that still lets every cluster
+// be resident at once (one wave); 1 when there are more tiles than that.  `cost` receives a relative
+// time estimate, k-steps per CTA x waves x the per-step weight of the tile height.
+template <int BITS, int NTOK, int H> int choose_cluster(int tiles, int ksteps, int forced, double &cost)
+{
+    using V = DecodeVariant<BITS, NTOK, H>;
+    int cs = 1;
+    if (forced > 0) {
+        cs = forced < kClusterMax ? forced : kClusterMax;
+        if (cs > ksteps) cs = ksteps;
+        while (cs > 1 && V::max_clusters(cs) == 0) --cs;
+    } else {
+        for (int c = kClusterMax < ksteps ? kClusterMax : ksteps; c > 1; --c)
+            if (V::max_clusters(c) >= tiles) { cs = c; break; }
+    }
+    const int resident = V::max_clusters(cs) > 0 ? V::max_clusters(cs) : 1;
+    const int waves = (tiles + resident - 1) / resident;
+    const int steps = (ksteps + cs - 1) / cs;
+    // a two-half step covers twice the rows in about 1.7 times the time of a one-half step, and every
+    // launch pays a fixed prologue + reduction worth a few steps
+    cost = (double)waves * ((double)steps * (H == 2 ? 1.7 : 1.0) + 2.0);
+    return cs;
+}
+
+template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem &p, int forced_cs, cudaStream_t stream)
+{
+    const int qrow = DCfg<BITS, 1>::QROW;
+    k.ksteps = (p.n + kStep - 1) / kStep;
+    int rc = DecodeVariant<BITS, NTOK, 1>::prepare();
+    if (rc == LORDS_OK) rc = DecodeVariant<BITS, NTOK, 2>::prepare();
+    if (rc != LORDS_OK) return rc;
+    const int tiles1 = (p.m + 127) / 128, tiles2 = (p.m + 255) / 256;
+    if (tiles1 > 65535) return LORDS_ERR_UNSUPPORTED;
+    double cost1 = 0, cost2 = 0;
+    const int cs1 = choose_cluster<BITS, NTOK, 1>(tiles1, k.ksteps, forced_cs, cost1);
+    const int cs2 = choose_cluster<BITS, NTOK, 2>(tiles2, k.ksteps, forced_cs, cost2);
+    const bool two = cost2 < cost1;
+    const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
+    if (!make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)qrow,
+                     two ? 256u : 128u, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.A, (uint64_t)p.n, (uint64_t)p.r, 64, (uint32_t)k.r_pad,
+                     CU_TENSOR_MAP_SWIZZLE_128B))
+        return LORDS_ERR_CUDA;
+    k.tiles = two ? tiles2 : tiles1;
+    return two ? DecodeVariant<BITS, NTOK, 2>::launch(k, tiles2, cs2, stream)
+               : DecodeVariant<BITS, NTOK, 1>::launch(k, tiles1, cs1, stream);
+}
+
+}  // namespace
+
+// Rules of this path: 3- or 4-bit codes; M <= 2 with M * ceil16(r) <= 64; r a multiple of 8 (16-byte
+// rows of B); n a multiple of 32 (4-bit) or 128 (3-bit), which makes every TMA row pitch a multiple
+// of 16 bytes.  Anything else: LORDS_ERR_UNSUPPORTED.
+int launch_decode(const Problem &p, State &st, cudaStream_t stream)
+{
+    if (p.bits != 3 && p.bits != 4) return LORDS_ERR_UNSUPPORTED;
+    if (p.M > 2 || p.r % 8 != 0) return LORDS_ERR_UNSUPPORTED;
+    const int r_pad = (p.r + 15) / 16 * 16;
+    if (p.M * r_pad > kNMax) return LORDS_ERR_UNSUPPORTED;
+    if (p.n % (p.bits == 4 ? 32 : 128) != 0) return LORDS_ERR_UNSUPPORTED;
+
+    DecodeParams k;
+    k.x = p.x; k.B = p.B;
+    for (int c = 0; c < 16; ++c) k.levels[c] = p.levels[c];
+    k.M = p.M; k.m = p.m; k.n = p.n; k.r = p.r; k.r_pad = r_pad;
+    k.y = p.y; k.y_f32 = p.y_f32;
+    k.status = st.status_word;
+#ifdef LORDS_TRACE
+    k.trace = reinterpret_cast<long long *>(st.workspace + st.workspace_bytes - (size_t)8 * 32 * 8 * 8);
+    LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)8 * 32 * 8 * 8, stream));
+#endif
+    int rc;
+    if (p.bits == 4) rc = p.M == 1 ? launch_bits_tok<4, 1>(k, p, st.forced_splitk, stream) : launch_bits_tok<4, 2>(k, p, st.forced_splitk, stream);
+    else rc = p.M == 1 ? launch_bits_tok<3, 1>(k, p, st.forced_splitk, stream) : launch_bits_tok<3, 2>(k, p, st.forced_splitk, stream);
+    if (rc != LORDS_OK) return rc;
+    st.last_launches = 1;
+    st.last_path = "decode";
+    return LORDS_OK;
+}
+
+#ifdef LORDS_TRACE
+// Debug builds only: copy the traced CTA's clock stamps of the last decode launch to the host.
+extern "C" int lords_debug_read_decode_trace(long long *out)
+{
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    LORDS_CUDA_TRY(cudaDeviceSynchronize());
+    LORDS_CUDA_TRY(cudaMemcpy(out, st.workspace + st.workspace_bytes - (size_t)8 * 32 * 8 * 8, (size_t)8 * 32 * 8 * 8,
+                              cudaMemcpyDeviceToHost));
+    return LORDS_OK;
+}
+#endif
+
+}  // namespace lords

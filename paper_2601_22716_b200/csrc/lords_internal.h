@@ -35,7 +35,7 @@ struct State {
     uint8_t *stage_x = nullptr;     // device staging for the host-buffer entry point
     uint8_t *stage_y = nullptr;
     size_t stage_x_bytes = 0, stage_y_bytes = 0;
-    int forced_path = 0;            // 0 auto, 1 simt, 2 decode, 3 prefill
+    int forced_path = 0;            // 0 auto, 1 simt, 2 decode (reassociated form), 3 umma (scale-MMA form)
     int forced_splitk = 0;          // 0 auto
     int last_cuda_error = 0;
     int last_launches = 0;
@@ -56,7 +56,12 @@ int cuda_fail(cudaError_t e);
 // Generic CUDA-core path: any shape the interface accepts.
 int launch_simt(const Problem &p, State &st, cudaStream_t stream);
 
-// Tensor-core path (TMA + tcgen05/TMEM).  LORDS_ERR_UNSUPPORTED for shapes outside its rules.
+// Tensor-core path (TMA + tcgen05/TMEM), scale matrix rebuilt per tile by a small MMA.
+// LORDS_ERR_UNSUPPORTED for shapes outside its rules.
 int launch_umma(const Problem &p, State &st, cudaStream_t stream);
+
+// Tensor-core decode path (M <= 2), reassociated form with the scale factors folded into the
+// activation operand.  LORDS_ERR_UNSUPPORTED for shapes outside its rules.
+int launch_decode(const Problem &p, State &st, cudaStream_t stream);
 
 }  // namespace lords

@@ -505,7 +505,7 @@ int launch_umma(const Problem &p, State &st, cudaStream_t stream)
     }
     if (rc != LORDS_OK) return rc;
     st.last_launches = 2;
-    st.last_path = p.M <= 16 ? "decode" : "prefill";
+    st.last_path = "umma";
     return LORDS_OK;
 }
 

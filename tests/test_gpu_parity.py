@@ -95,6 +95,69 @@ def test_forced_splitk_is_deterministic_and_correct(lords, splitk, path):
     check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
 
 
+# ---- the decode kernel (reassociated form, M <= 2), forced so that a decline is an error -----------
+
+DECODE_SHAPES = [
+    # bits, m, n, r, M, mixed
+    (4, 512, 4096, 32, 2, False),
+    (4, 300, 1056, 8, 1, True),      # ragged rows; n = 8.25 k-steps; r padded to 16
+    (4, 1000, 2048, 24, 2, True),    # r padded to 32, two tokens
+    (4, 64, 8192, 64, 1, False),     # one tile, the largest cluster
+    (4, 40000, 64, 16, 1, False),    # more tiles than resident clusters, half a k-step each
+    (4, 256, 32, 8, 1, True),        # a quarter-filled k-step
+    (3, 520, 1152, 48, 1, True),
+    (3, 256, 128, 16, 2, False),
+    (3, 2048, 4096, 32, 2, False),
+]
+
+
+@pytest.mark.parametrize("bits,m,n,r,M,mixed", DECODE_SHAPES)
+def test_decode_kernel_shapes(lords, bits, m, n, r, M, mixed):
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=3 * m + n + r, mixed_sign=mixed)
+    dl, y32, ybf = _run(lords, lay, "decode")
+    assert lords.lords_last_path() == "decode" and lords.lords_last_launch_count() == 1
+    y64 = _oracle(lay, dl.packed_host)
+    check_against_oracle(y32, ybf, y64)
+
+
+@pytest.mark.parametrize("bits,m,n,r,M", [(4, 700, 2048, 32, 1), (4, 256, 1024, 16, 2), (3, 384, 1024, 48, 1),
+                                          (3, 131, 256, 8, 2)])
+def test_decode_kernel_integer_case_is_bit_exact(lords, bits, m, n, r, M):
+    lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m)
+    dl, y32, ybf = _run(lords, lay, "decode")
+    assert lords.lords_last_path() == "decode"
+    y64 = _oracle(lay, dl.packed_host)
+    assert np.array_equal(y32.astype(np.float64), y64)
+    assert np.array_equal(ybf, oracle.round_bf16(y64))
+
+
+@pytest.mark.parametrize("cluster", [1, 3, 7, 100])
+def test_decode_kernel_cluster_split_is_deterministic(lords, cluster):
+    lay = gen.make_layer(600, 3072, 32, 2, bits=4, seed=17)
+    lords.lords_set_option("splitk", str(cluster))
+    lords.lords_set_option("path", "decode")
+    try:
+        dl = DeviceLayer(lay)
+        y32, ybf = dl.forward()
+        y32b, ybfb = dl.forward()
+    finally:
+        lords.lords_set_option("splitk", "0")
+        lords.lords_set_option("path", "auto")
+    assert np.array_equal(y32, y32b) and np.array_equal(ybf, ybfb)
+    check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
+
+
+def test_decode_kernel_declines_what_it_cannot_run(lords):
+    lay = gen.make_layer(256, 256, 4, 4, bits=4, seed=0)      # M = 4, r = 4
+    lords.lords_set_option("path", "decode")
+    try:
+        with pytest.raises(lords.LordsError) as ei:
+            DeviceLayer(lay).forward()
+        assert ei.value.status == -11
+    finally:
+        lords.lords_set_option("path", "auto")
+
+
 def test_linearity_on_gpu(lords):
     import torch
     m, n, r = 128, 512, 16
@@ -166,4 +229,4 @@ def test_four_bit_entry_point_and_launch_count(lords):
     torch.cuda.synchronize()
     assert np.array_equal(y.cpu().numpy().view(np.uint16), ybf)
     assert lords.lords_last_launch_count() >= 1
-    assert lords.lords_last_path() in ("simt", "decode", "prefill")
+    assert lords.lords_last_path() in ("simt", "decode", "umma")
