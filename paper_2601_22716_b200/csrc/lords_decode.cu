@@ -14,15 +14,16 @@
 // global memory.
 //
 // Warp roles (20 warps):
-//   0..15  worker groups of 4 * H warps take k-steps round-robin.  For its k-step a group
+//   0..15  two worker groups of eight warps take k-steps alternately.  For its k-step a group
 //          (a) turns the factor tile A[:, k-step] (TMA, shared memory) in place into the fp16 B
 //              operand A_kj * x_tj, and
-//          (b) dequantises: warp (h, q) owns rows h*128 + q*32 .. +31; a thread reads its row's packed
-//              codes from shared memory, looks every code pair up in a lane-private fp16x2 level
-//              table and stores the row straight into TMEM as the A operand (tcgen05.st).
+//          (b) dequantises: a warp owns 32 rows (H = 2: all 128 columns of the k-step; H = 1: one
+//              64-column half); a thread reads its row's packed codes from shared memory, looks every
+//              code pair up in a lane-private fp16x2 level table and stores the levels straight into
+//              TMEM as the A operand (tcgen05.st).
 //          Group 0 also runs the epilogue.
-//   16,17  MMA issuers, one per 128-row half: D_h[128 x N] += W_h[128 x 16] * AX[N x 16]^T with
-//          A from TMEM and B from shared memory, eight per k-step.
+//   16,17  MMA issuers: D[128 x N] += W[128 x 16] * AX[N x 16]^T with A from TMEM and B from shared
+//          memory, eight per k-step; one issuer per 128-row half (H = 2) or per k-step parity (H = 1).
 //   18     TMA producer of the packed code tiles (HBM stream, deep ring); it also initialises the
 //          barriers and starts the stream before the rest of the CTA has finished its set-up.
 //   19     TMA producer of the factor tiles.
@@ -33,6 +34,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "lords_internal.h"
 #include "lords_ptx.cuh"
 
@@ -42,8 +45,8 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kWorkWarps = 16;                         // worker warps: 16 / (4 * H) groups of 4 * H
-constexpr int kIssuerWarp0 = kWorkWarps;               // 16, 17 (the second one idles when H == 1)
+constexpr int kWorkWarps = 16;                         // worker warps: two groups of eight
+constexpr int kIssuerWarp0 = kWorkWarps;               // 16, 17: one per half (H == 2) or per k-step parity (H == 1)
 constexpr int kTmaQWarp = kIssuerWarp0 + 2;            // 18
 constexpr int kTmaAWarp = kTmaQWarp + 1;               // 19
 constexpr int kWarps = kTmaAWarp + 1;                  // 20
@@ -60,8 +63,9 @@ constexpr int kWSlotCols = kStep / 2;                  // TMEM columns of one W 
 // BITS: code width.  H: 128-row halves per CTA tile (1 or 2).
 template <int BITS, int H> struct DCfg {
     static constexpr int TILE_ROWS = 128 * H;
-    static constexpr int GROUP_WARPS = 4 * H;                  // worker warps on one k-step
-    static constexpr int GROUPS = kWorkWarps / GROUP_WARPS;    // groups take k-steps round-robin (4 / 2)
+    static constexpr int GROUP_WARPS = 8;                      // worker warps on one k-step
+    static constexpr int GROUPS = kWorkWarps / GROUP_WARPS;    // two groups take k-steps alternately
+    static constexpr int COLS = kStep * H / 2;                 // columns of the k-step one thread dequantises (64 / 128)
     static constexpr int QROW = kStep * BITS / 8;              // packed bytes per row per k-step (64 / 48)
     static constexpr int QSTAGE = TILE_ROWS * QROW;
     static constexpr int SQ = (BITS == 4 ? 8 : 12) / H;        // code-tile ring depth: 64 / 72 KB in flight
@@ -114,13 +118,20 @@ __device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float 
 }
 
 // One row of one k-step (128 codes): packed codes (shared memory) -> fp16 level pairs -> 64 TMEM columns.
-template <int BITS>
-__device__ __forceinline__ void dequant_row_to_tmem(uint32_t qrow, uint32_t lut_lane, uint32_t taddr)
+// 4-bit rows are 64 bytes and arrive 64-byte-swizzled (16-byte chunk c of row i sits at chunk
+// c ^ ((i >> 1) & 3)), which spreads the 16-byte reads of eight consecutive rows over all banks;
+// 3-bit rows are 48 bytes, a stride that is conflict-free as it is.
+template <int BITS, int COLS>
+__device__ __forceinline__ void dequant_row_to_tmem(uint32_t qrow, int row, int ch, uint32_t lut_lane, uint32_t taddr)
 {
+    // COLS == 128: the thread does the whole row (two 64-column halves); COLS == 64: only half `ch`.
+    constexpr int kHalves = COLS / 64;
     if constexpr (BITS == 4) {
+        const uint32_t sw = (uint32_t)((row >> 1) & 3);
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const uint4 c0 = lds_v4(qrow + half * 32), c1 = lds_v4(qrow + half * 32 + 16);
+        for (int hh = 0; hh < kHalves; ++hh) {
+            const int half = kHalves == 2 ? hh : ch;
+            const uint4 c0 = lds_v4(qrow + (((2 * half) ^ sw) << 4)), c1 = lds_v4(qrow + (((2 * half + 1) ^ sw) << 4));
             const uint32_t w[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
             uint32_t out[32];
 #pragma unroll
@@ -136,8 +147,8 @@ __device__ __forceinline__ void dequant_row_to_tmem(uint32_t qrow, uint32_t lut_
     } else {
         const uint4 c0 = lds_v4(qrow), c1 = lds_v4(qrow + 16), c2 = lds_v4(qrow + 32);
         const uint32_t w[12] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w};
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        auto half_row = [&](auto half_c) {
+            constexpr int half = decltype(half_c)::value;
             uint32_t out[32];
 #pragma unroll
             for (int pp = 0; pp < 32; ++pp) {
@@ -149,7 +160,9 @@ __device__ __forceinline__ void dequant_row_to_tmem(uint32_t qrow, uint32_t lut_
                 out[pp] = lds_u32((sh & 0x1F80u) | lut_lane);
             }
             tmem_st_32x32(taddr + half * 32, out);
-        }
+        };
+        if (kHalves == 2 || ch == 0) half_row(std::integral_constant<int, 0>{});
+        if (kHalves == 2 || ch == 1) half_row(std::integral_constant<int, 1>{});
     }
 }
 
@@ -170,9 +183,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     constexpr int kBarQEmpty = kBarQFull + SQ;              // SQ, the warps of one group
     constexpr int kBarAFull = kBarQEmpty + SQ;              // S, 1 arrival + TMA bytes
     constexpr int kBarReady = kBarAFull + S;                // H * S: the warps of one group (W slot and B operand written)
-    constexpr int kBarMmaDone = kBarReady + H * S;          // S, one commit per issuer
-    constexpr int kBarAccFull = kBarMmaDone + S;            // H
-    constexpr int kBarReduce = kBarAccFull + H;             // 1: every epilogue warp of every CTA of the cluster
+    constexpr int kBarMmaDone = kBarReady + H * S;          // S, one commit per half
+    constexpr int kBarAccFull = kBarMmaDone + S;            // 2: one per issuer
+    constexpr int kBarReduce = kBarAccFull + 2;             // 1: every epilogue warp of every CTA of the cluster
     constexpr int kBarCount = kBarReduce + 1;
     static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
     const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
@@ -194,6 +207,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     if (tid == 0) DSTAMP(7, 0, 0);
     bool failed = false;
 
+    if (warp == kTmaQWarp && lane == 0) DSTAMP(6, 0, 0);
     if (warp == kTmaQWarp) {
         // ------------------------------------------------------------------ code tiles (HBM stream)
         // This warp initialises every barrier, releases the rest of the CTA and starts the stream of
@@ -203,16 +217,17 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             uint32_t count = 1;
             if (b >= kBarQEmpty && b < kBarAFull) count = kGroupWarps;
             else if (b >= kBarReady && b < kBarMmaDone) count = kGroupWarps;
-            else if (b >= kBarMmaDone && b < kBarAccFull) count = H;
-            else if (b == kBarReduce) count = (uint32_t)(kGroupWarps * csize);
+            else if (b >= kBarMmaDone && b < kBarAccFull) count = H;   // H == 1: the step's one issuer
+            else if (b == kBarReduce) count = (uint32_t)(4 * H * csize);
             mbar_init(bars + 8 * b, count);
         }
         fence_mbar_init();
         __syncwarp();
         asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");   // barriers exist; does not wait for the others
-        // split-phase cluster barrier: arrive now (this CTA's reduce barrier exists); the wait is in
-        // the epilogue, right before the first access to the leader's shared memory
-        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        // split-phase cluster barrier: arrive now (this CTA's reduce barrier exists and the fence above
+        // has published it cluster-wide, so a relaxed arrival is enough); the wait is in the epilogue,
+        // right before the first access to the leader's shared memory
+        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
         if (lane == 0) {
             DSTAMP(7, 0, 3);
             tma_prefetch_desc(&p.tm_q);
@@ -235,20 +250,26 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         } else if (warp < kWorkWarps) {
             // level-pair table: entry e = (L[lo code], L[hi code]) as fp16x2; word e*32 + lane is lane's
             // copy (bank = lane, so the lookups of a warp never conflict)
-            for (int e = tid; e < C::LUT_ENTRIES * 32; e += kWorkWarps * 32) {
-                const int entry = e >> 5;
+            // warp w writes entries w, w + 16, ...; the loads of the levels are independent
+#pragma unroll
+            for (int i = 0; i < C::LUT_ENTRIES / kWorkWarps; ++i) {
+                const int entry = warp + kWorkWarps * i;
                 const int lo = BITS == 4 ? (entry & 15) : (entry & 7);
                 const int hi = BITS == 4 ? (entry >> 4) : (entry >> 3);
                 const __half2 v = __floats2half2_rn(p.levels[lo], p.levels[hi]);
-                sts_u32(lut + 4u * (uint32_t)e, *reinterpret_cast<const uint32_t *>(&v));
+                sts_u32(lut + 4u * (uint32_t)(entry * 32 + lane), *reinterpret_cast<const uint32_t *>(&v));
             }
             if (tid == 0) DSTAMP(7, 0, 5);
         }
         tc_fence_before_sync();
+        if (tid == 0) DSTAMP(6, 0, 1);
         asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");   // table, TMEM address and barriers are in place
         tc_fence_after_sync();
-        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");   // see above
+        if (tid == 0) DSTAMP(6, 0, 2);
+        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");   // see above
     }
+    // let a dependent launch (the next layer) begin its own weight prefetch as SMs become free
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) DSTAMP(7, 0, 1);
 
     if (warp == kTmaQWarp) {
@@ -267,39 +288,47 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                     tma_load_2d(ax0 + s * C::AXSTAGE + at * kAtomBytes, &p.tm_a, (ks_a + it) * kStep + at * 64, 0, bar);
             }
         }
-    } else if (warp >= kIssuerWarp0 + H) {
-        // spare issuer warp of the one-half configuration: nothing to do
     } else if (warp >= kIssuerWarp0) {
-        // ------------------------------------------------------------------ MMA issuer of half h
-        const int h = warp - kIssuerWarp0;
+        // ------------------------------------------------------------------ MMA issuers
+        // H == 2: issuer j owns half j and takes every k-step.  H == 1: the two issuers take the
+        // k-steps alternately, each into its own accumulator (the epilogue adds the two), which
+        // doubles the rate at which MMAs leave the CTA.
+        const int j = warp - kIssuerWarp0;
+        const int h = H == 2 ? j : 0;
+        constexpr int kStride = H == 2 ? 1 : 2;
+        static_assert(H == 2 || S % 2 == 0, "with alternating issuers every ring barrier belongs to one of them");
         uint32_t tmem_base;
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         const uint32_t idesc = (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);  // fp16 x fp16 -> fp32, K-major
         const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
         const uint32_t ax_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((ax0 & 0x3FFFFu) >> 4);
-        const uint32_t acc = tmem_base + (uint32_t)(h * kNMax);
-        for (int it = 0; it < total; ++it) {
+        const uint32_t acc = tmem_base + (uint32_t)(j * kNMax);
+        const int first = H == 2 ? 0 : j;
+        for (int it = first; it < total; it += kStride) {
             const int s = it % S;
-            if (h == 0 && lane == 0) DSTAMP(0, it, 0);
+            if (j == 0 && lane == 0) DSTAMP(0, it, 0);
             if (!mbar_wait(bar_ready + 8 * (h * S + s), (uint32_t)((it / S) & 1))) { failed = true; break; }
             tc_fence_after_sync();
-            if (h == 0 && lane == 0) DSTAMP(0, it, 1);
+            if (j == 0 && lane == 0) DSTAMP(0, it, 1);
             if (lane == 0) {
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)((h * S + s) * kWSlotCols);
                 const uint32_t b_lo = ax_lo0 + (uint32_t)(s * (C::AXSTAGE >> 4));
 #pragma unroll
                 for (int k = 0; k < kStep / 16; ++k)
                     umma_f16_ts(acc, wslot + k * 8, umma_desc_pack(b_lo + (k >> 2) * (kAtomBytes >> 4) + (k & 3) * 2, desc_hi),
-                                idesc, (it == 0 && k == 0) ? 0u : 1u);
+                                idesc, (it == first && k == 0) ? 0u : 1u);
                 umma_commit(bar_mma_done + 8 * s);
-                if (it == total - 1) umma_commit(bar_acc_full + 8 * h);
-                if (h == 0) DSTAMP(0, it, 2);
+                if (it + kStride >= total) umma_commit(bar_acc_full + 8 * j);
+                if (j == 0) DSTAMP(0, it, 2);
             }
             __syncwarp();
         }
     } else {
         // ------------------------------------------------------------------ worker warps
-        const int g = warp / kGroupWarps, wg = warp % kGroupWarps, h = (warp >> 2) % H, q = warp & 3;
+        // warp wg of a group: lane quadrant q; H == 2: row half h, all 128 columns of the k-step;
+        // H == 1: the one row half, column half ch
+        const int g = warp / kGroupWarps, wg = warp % kGroupWarps, q = warp & 3;
+        const int h = H == 2 ? (wg >> 2) : 0, ch = H == 2 ? 0 : (wg >> 2);
         const int row_in_tile = h * 128 + q * 32 + lane;
         uint32_t tmem_base;
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
@@ -308,8 +337,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         const bool stamper = wg == 0 && lane == 0 && g < 2;
         // B-operand share of this lane: the 16-byte chunk c16 (8 columns) of rows rsub + kRowStep * i
         const int c16 = lane & 7, rsub = wg * 4 + (lane >> 3);
-        constexpr int kRowStep = 4 * kGroupWarps;                        // 16 / 32
-        constexpr int kRowIters = (kNMax + kRowStep - 1) / kRowStep;     // 4 / 2
+        constexpr int kRowStep = 4 * kGroupWarps;                        // 32
+        constexpr int kRowIters = (kNMax + kRowStep - 1) / kRowStep;     // 2
 
         uint4 xr[NTOK][kAtoms];
         auto load_x = [&](int ks) {
@@ -323,7 +352,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 }
         };
         // x may be the previous launch's output: everything above this line only touched weights
+        if (tid == 0) DSTAMP(6, 0, 3);
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (tid == 0) DSTAMP(6, 0, 4);
         if (g < total) load_x(ks_a + g);
 
         for (int it = g; it < total; it += kGroups) {
@@ -379,14 +410,17 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                     }
                 }
             }
-            fence_proxy_async_smem();
             if (it + kGroups < total) load_x(ks_a + it + kGroups);   // the group's next k-step
             if (stamper) DSTAMP(1 + g, it, 2);
 
             // (b) codes -> levels -> TMEM
             if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1)))) { failed = true; break; }
-            dequant_row_to_tmem<BITS>(q0 + sq * C::QSTAGE + row_in_tile * C::QROW, lut_lane,
+            if (stamper) DSTAMP(1 + g, it, 4);
+            dequant_row_to_tmem<BITS, C::COLS>(q0 + sq * C::QSTAGE + row_in_tile * C::QROW, row_in_tile, ch, lut_lane,
                                       lane_addr + kWCol + (uint32_t)((h * S + s) * kWSlotCols));
+            // one settling point for both products of the step: the B-operand stores become visible
+            // to the tensor core's (async-proxy) reads, the TMEM stores complete
+            fence_proxy_async_smem();
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
@@ -400,7 +434,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
 
         // Epilogue (group 0): z (TMEM) . B row -> this CTA's partial y, parked in the cluster
         // leader's shared memory; the leader adds the cluster's partials in rank order.
-        if (g == 0 && !failed) {
+        if (g == 0 && ch == 0 && !failed) {
             const int i = tile * kTileRows + row_in_tile;
             if (stamper) DSTAMP(5, 0, 0);
             // B row first, so its latency hides behind the wait for the last MMAs
@@ -413,30 +447,37 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
 #pragma unroll
             for (int t = 0; t < NTOK; ++t) yt[t] = 0.0f;
             bool ok = true;
-            if (total > 0) {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * h, 0));
-                tc_fence_after_sync();
-                if (stamper) DSTAMP(5, 0, 1);
-                if (ok) {
+            // H == 2: this half's accumulator.  H == 1: the accumulators of both issuers (the second
+            // one only if it had a k-step at all).
+            constexpr int kAccs = H == 2 ? 1 : 2;
 #pragma unroll
-                    for (int t = 0; t < NTOK; ++t) {
-                        float a = 0.0f;
+            for (int a = 0; a < kAccs; ++a) {
+                const int j = H == 2 ? h : a;
+                if (ok && j < total + (H == 2 ? 2 : 0)) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * j, 0));
+                    tc_fence_after_sync();
+                    if (stamper) DSTAMP(5, 0, 1);
+                    if (ok) {
 #pragma unroll
-                        for (int c = 0; c < kNMax / 16; ++c) {
-                            if (c * 16 < p.r_pad) {   // warp-uniform
-                                uint32_t v[16];
-                                tmem_ld_32x16(lane_addr + (uint32_t)(h * kNMax + t * p.r_pad + c * 16), v);
-                                tmem_wait_ld();
-                                const uint32_t bw[8] = {bq[2 * c].x, bq[2 * c].y, bq[2 * c].z, bq[2 * c].w,
-                                                        bq[2 * c + 1].x, bq[2 * c + 1].y, bq[2 * c + 1].z, bq[2 * c + 1].w};
+                        for (int t = 0; t < NTOK; ++t) {
+                            float acc = yt[t];
 #pragma unroll
-                                for (int e = 0; e < 8; ++e) {
-                                    a = fmaf(__uint_as_float(v[2 * e]), __uint_as_float(bw[e] << 16), a);
-                                    a = fmaf(__uint_as_float(v[2 * e + 1]), __uint_as_float(bw[e] & 0xFFFF0000u), a);
+                            for (int c = 0; c < kNMax / 16; ++c) {
+                                if (c * 16 < p.r_pad) {   // warp-uniform
+                                    uint32_t v[16];
+                                    tmem_ld_32x16(lane_addr + (uint32_t)(j * kNMax + t * p.r_pad + c * 16), v);
+                                    tmem_wait_ld();
+                                    const uint32_t bw[8] = {bq[2 * c].x, bq[2 * c].y, bq[2 * c].z, bq[2 * c].w,
+                                                            bq[2 * c + 1].x, bq[2 * c + 1].y, bq[2 * c + 1].z, bq[2 * c + 1].w};
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) {
+                                        acc = fmaf(__uint_as_float(v[2 * e]), __uint_as_float(bw[e] << 16), acc);
+                                        acc = fmaf(__uint_as_float(v[2 * e + 1]), __uint_as_float(bw[e] & 0xFFFF0000u), acc);
+                                    }
                                 }
                             }
+                            yt[t] = acc;
                         }
-                        yt[t] = a;
                     }
                 }
             }
@@ -536,13 +577,17 @@ template <int BITS, int NTOK, int H> struct DecodeVariant {
         attr[0].val.clusterDim.x = (unsigned)cs;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        // programmatic dependent launch: this kernel may start while the previous kernel in the stream
+        // drains; it touches only weights until its griddepcontrol.wait
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg = cudaLaunchConfig_t{};
         cfg.gridDim = dim3((unsigned)(clusters * cs));
         cfg.blockDim = dim3(kThreads);
         cfg.dynamicSmemBytes = DCfg<BITS, H>::SMEM;
         cfg.stream = stream;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = 2;
     }
     // Clusters of `cs` CTAs that can be resident at the same time (0 if such a cluster cannot run).
     static int max_clusters(int cs)
@@ -550,7 +595,7 @@ template <int BITS, int NTOK, int H> struct DecodeVariant {
         static int cache[kClusterMax + 1];   // 0 = not asked yet, -1 = cannot run
         if (cache[cs] == 0) {
             cudaLaunchConfig_t cfg;
-            cudaLaunchAttribute attr[1];
+            cudaLaunchAttribute attr[2];
             fill(cfg, attr, cs, 1, nullptr);
             int n = 0;
             const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_decode_kernel<BITS, NTOK, H>, &cfg);
@@ -562,7 +607,7 @@ template <int BITS, int NTOK, int H> struct DecodeVariant {
     static int launch(const DecodeParams &k, int tiles, int cs, cudaStream_t stream)
     {
         cudaLaunchConfig_t cfg;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         fill(cfg, attr, cs, tiles, stream);
         LORDS_CUDA_TRY(cudaLaunchKernelEx(&cfg, lords_decode_kernel<BITS, NTOK, H>, k));
         return LORDS_OK;
@@ -608,7 +653,7 @@ template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem
     const bool two = cost2 < cost1;
     const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
     if (!make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)qrow,
-                     two ? 256u : 128u, CU_TENSOR_MAP_SWIZZLE_NONE) ||
+                     two ? 256u : 128u, BITS == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE) ||
         !make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.A, (uint64_t)p.n, (uint64_t)p.r, 64, (uint32_t)k.r_pad,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return LORDS_ERR_CUDA;
