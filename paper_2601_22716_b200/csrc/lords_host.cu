@@ -221,10 +221,11 @@ int lords_shutdown(void)
         if (st.stage_x) cudaFree(st.stage_x);
         if (st.stage_y) cudaFree(st.stage_y);
     }
-    int fp = st.forced_path, fs = st.forced_splitk;
+    int fp = st.forced_path, fs = st.forced_splitk, fb = st.forced_bn;
     st = State();
     st.forced_path = fp;
     st.forced_splitk = fs;
+    st.forced_bn = fb;
     return LORDS_OK;
 }
 
@@ -308,6 +309,13 @@ int lords_set_option(const char *key, const char *value)
         long v = std::strtol(value, &end, 10);
         if (end == value || *end != '\0' || v < 0 || v > 1024) return LORDS_ERR_OPTION;
         st.forced_splitk = (int)v;
+        return LORDS_OK;
+    }
+    if (std::strcmp(key, "bn") == 0) {
+        char *end = nullptr;
+        long v = std::strtol(value, &end, 10);
+        if (end == value || *end != '\0' || (v != 0 && v != 32 && v != 64 && v != 128 && v != 256)) return LORDS_ERR_OPTION;
+        st.forced_bn = (int)v;
         return LORDS_OK;
     }
     return LORDS_ERR_OPTION;

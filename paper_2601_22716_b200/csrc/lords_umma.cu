@@ -1,19 +1,23 @@
-// Tensor-core path (sm_100a): TMA-staged operands, tcgen05.mma with accumulators in TMEM.
+// Scale-MMA path on tcgen05/TMEM for any token count: W^ = L[Q] (.) (BA) is rebuilt tile by tile.
 //
-// One CTA owns a 128-row tile of W^ (out-features), a tile of BN tokens and a range of
-// 64-column k-blocks (split-K over the in-feature axis).  Per k-block:
-//   1. the TMA warp loads the packed code tile Q[128 x 64] (4-bit: 32 B per row), the factor
-//      tile A[r x 64] (bf16) and the activation tile x16[BN x 64] (fp16) into a shared-memory ring;
-//   2. the MMA thread issues the scale MMA  S = B_tile (128 x r) * A_tile (r x 64)  (Eq. 3,
-//      bf16 operands, fp32 accumulator in TMEM);
-//   3. eight dequant warps read S from TMEM, look up the levels of their codes, form
-//      W^ = L[Q] (.) S as fp16 and store it as the 128-byte-swizzled K-major A operand;
-//   4. the MMA thread issues  D[128 x BN] += W^_tile * x_tile^T  (fp16 operands, fp32 in TMEM).
-// Epilogue: D -> registers -> y (bf16 RNE or fp32), or -> split-K scratch, where the last CTA
-// of a tile to arrive adds the partials in split order (deterministic) and stores y.
+// One CTA owns a 128-row tile of W^ (out-features), a tile of BN tokens and a range of 64-column
+// k-steps.  Per k-step:
+//   1. TMA brings the factor tile A[r x 64] (bf16) and the activation tile x[BN x 64] into a
+//      shared-memory ring; the packed code tile Q[128 x 128 columns] comes once per two k-steps;
+//   2. the issuer thread runs the scale MMA  S = B_tile (128 x r) * A_tile (r x 64)  (Eq. 3; bf16
+//      operands from shared memory, fp32 result in TMEM), a few k-steps ahead of the main MMA;
+//   3. two worker groups of eight warps take the k-steps alternately: a thread reads its 32 columns
+//      of S from TMEM, looks its code pairs up in a lane-private fp16x2 level table, forms
+//      W^ = L[Q] (.) S in fp16 and stores it straight back into TMEM as the A operand;
+//   4. the issuer runs  D[128 x BN] += W^ (TMEM) * x_tile^T (shared memory), fp32 in TMEM.
+// The activations enter the MMA as fp16: for BN = 16 the workers convert the bf16 tile in place,
+// for larger token tiles a pre-pass converts x once into scratch.
+// Epilogue: D -> registers -> y (bf16 round-to-nearest-even, or fp32).  For BN = 16 the k-range of
+// a tile is split over a thread-block cluster whose partial sums meet in the leader's shared
+// memory (distributed shared memory) and are added in rank order: deterministic, no atomics.
 //
-// Every mbarrier wait is bounded; on expiry the kernel records LORDS_ERR_TIMEOUT, all roles
-// drain, TMEM is released and the kernel returns.
+// Every wait is bounded; on expiry the role records LORDS_ERR_TIMEOUT and leaves its loop, so the
+// kernel always reaches its final barrier and frees its TMEM.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -27,57 +31,52 @@ namespace {
 
 using namespace ptx;
 
-constexpr int BM = 128;            // W^ rows per CTA = UMMA M
-constexpr int BK = 64;             // in-feature columns per k-block (one swizzle row of fp16)
-constexpr int kRMaxUmma = 64;      // largest rank this path takes (one swizzle atom of K)
-constexpr int kDequantWarps = 8;
-constexpr int kDequantThreads = kDequantWarps * 32;
-constexpr int kTmaWarp = kDequantWarps;
-constexpr int kMmaWarp = kDequantWarps + 1;
-constexpr int kThreads = (kDequantWarps + 2) * 32;
+constexpr int BM = 128;                        // W^ rows per CTA = UMMA M
+constexpr int BK = 64;                         // in-feature columns per k-step
+constexpr int kRMaxUmma = 64;                  // largest rank this path takes (one swizzle atom of K)
+constexpr int kWorkWarps = 16;                 // two groups of eight
+constexpr int kGroupWarps = 8;
+constexpr int kIssuerWarp = kWorkWarps;        // 16
+constexpr int kTmaWarp = kWorkWarps + 1;       // 17
+constexpr int kThreads = (kWorkWarps + 2) * 32;   // 576
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kSCol = 256;    // S buffers live at TMEM columns 256 and 320
+constexpr uint32_t kWCol = 384;                // W ring: 4 slots of 32 columns
+constexpr int WD = 4;                          // W ring depth
+constexpr int SQ = 4;                          // code-tile ring depth (128 columns per stage)
 constexpr int kATileBytes = kRMaxUmma * 128;
-constexpr int kQTileBytes = BM * 32;
-constexpr int kWTileBytes = BM * 128;
-constexpr int kLutBytes = 256 * 32 * 4;
+constexpr int kBTileBytes = BM * 128;
+constexpr int kClusterMax = 8;                 // largest k-split (cluster size) of the BN = 16 kernel
 
-template <int BN> struct Cfg {
-    static constexpr int kStages = BN >= 256 ? 3 : 4;
-    static constexpr int kXTileBytes = BN * 128;
-    static constexpr int kStageBytes = kXTileBytes + kATileBytes + kQTileBytes;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 2 * kWTileBytes + kWTileBytes /*B tile*/ +
-                                      kLutBytes + 256 /*barriers*/ + 1024 /*alignment slack*/;
+template <int BITS, int BN> struct UCfg {
+    static constexpr int QROW = 128 * BITS / 8;                  // packed bytes per row per code stage (64 / 48)
+    static constexpr int QSTAGE = BM * QROW;
+    static constexpr int SX = BN >= 256 ? 3 : 4;                 // factor / activation ring depth
+    static constexpr int XTILE = BN * 128;
+    static constexpr int AXSTAGE = kATileBytes + XTILE;
+    static constexpr uint32_t SCOL = BN > 128 ? 256 : 128;       // S ring starts behind the accumulator
+    static constexpr int SD = (int)(kWCol - SCOL) / 64;          // S ring depth (2 / 4)
+    static constexpr int LEAD = SD < SX - 1 ? SD : SX - 1;       // k-steps the scale MMA runs ahead of the main MMA
+    static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;
+    static constexpr int LUT_BYTES = LUT_ENTRIES * 128;
+    static constexpr int RED_BYTES = BN == 16 ? kClusterMax * 16 * BM * 4 : 0;
+    static constexpr int BAR_BYTES = 512;
+    static constexpr int SMEM = 1024 + SX * AXSTAGE + SQ * QSTAGE + kBTileBytes + LUT_BYTES + RED_BYTES + BAR_BYTES;
+    static constexpr bool kConvertInKernel = BN == 16;           // x tile arrives as bf16 and is converted in place
 };
 
 struct alignas(64) UmmaParams {
-    CUtensorMap tm_x;     // fp16 [M][n], box {64, BN}
-    CUtensorMap tm_a;     // bf16 [r][n], box {64, r_pad}
-    CUtensorMap tm_q;     // u8 [m][n/2], box {32, 128}
+    CUtensorMap tm_x;     // BN == 16: bf16 [M][n]; else fp16 [M][n]; box {64, BN}, 128-byte swizzle
+    CUtensorMap tm_a;     // bf16 [r][n], box {64, r_pad}, 128-byte swizzle
+    CUtensorMap tm_q;     // u8 [m][n*bits/8], box {QROW, 128}
     const uint16_t *B;    // bf16 [m][r]
     float levels[16];
     int M, m, n, r, r_pad;
-    int kblocks;          // ceil(n / 64)
-    int splits, kb_per_split;
+    int npairs;           // 128-column pairs of k-steps per tile
     int tok_tiles;
-    float *partial;       // [splits][M][m]
-    int *counters;        // one per (row tile, token tile), zero between calls
     void *y;
     int y_f32;
     int *status;
-#ifdef LORDS_TRACE
-    long long *trace;     // [3 roles][64 iterations][8 events] clock64 stamps of CTA 0 (debug builds only)
-#endif
 };
-
-#ifdef LORDS_TRACE
-#define LORDS_STAMP(role, it, ev)                                                        \
-    do {                                                                                 \
-        if (blockIdx.x == 0 && (it) < 64) p.trace[((role) * 64 + (it)) * 8 + (ev)] = clock64(); \
-    } while (0)
-#else
-#define LORDS_STAMP(role, it, ev) do { } while (0)
-#endif
 
 __device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float v)
 {
@@ -85,280 +84,352 @@ __device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float 
     else static_cast<__nv_bfloat16 *>(y)[idx] = __float2bfloat16_rn(v);
 }
 
-__device__ __forceinline__ void named_bar_sync(int id, int count)
+// The 32 columns (chunk c of the 128-column code stage) of one row: codes -> level pairs, times the
+// matching pairs of S, as 16 fp16x2 words.
+template <int BITS>
+__device__ __forceinline__ void dequant_chunk(uint32_t qrow, int row, int c, uint32_t lut_lane, const uint32_t (&s)[32],
+                                              uint32_t (&out)[16])
 {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+    uint32_t lv[16];
+    if constexpr (BITS == 4) {
+        // 64-byte rows, 64-byte swizzle: 16-byte chunk c of row i sits at chunk c ^ ((i >> 1) & 3)
+        const uint4 cw = lds_v4(qrow + (((uint32_t)c ^ (uint32_t)((row >> 1) & 3)) << 4));
+        const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
+#pragma unroll
+        for (int wi = 0; wi < 4; ++wi)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const uint32_t sh = b == 0 ? (w[wi] << 7) : (w[wi] >> (8 * b - 7));
+                lv[wi * 4 + b] = lds_u32(lut_lane + (sh & 0x7F80u));
+            }
+    } else {
+        // 48-byte rows: chunk c is the 96-bit group at byte 12c; pair p sits at bit 6p of it
+        const uint32_t w[3] = {lds_u32(qrow + 12 * c), lds_u32(qrow + 12 * c + 4), lds_u32(qrow + 12 * c + 8)};
+#pragma unroll
+        for (int pp = 0; pp < 16; ++pp) {
+            const int bit = 6 * pp, wi = bit >> 5, off = bit & 31;
+            uint32_t sh;
+            if (off > 26) sh = __funnelshift_r(w[wi], w[wi + 1 < 3 ? wi + 1 : 2], off - 7);
+            else sh = off >= 7 ? (w[wi] >> (off - 7)) : (w[wi] << (7 - off));
+            lv[pp] = lds_u32(lut_lane + (sh & 0x1F80u));
+        }
+    }
+#pragma unroll
+    for (int pp = 0; pp < 16; ++pp) {
+        const __half2 sv = __floats2half2_rn(__uint_as_float(s[2 * pp]), __uint_as_float(s[2 * pp + 1]));
+        const __half2 wv = __hmul2(*reinterpret_cast<const __half2 *>(&lv[pp]), sv);
+        out[pp] = *reinterpret_cast<const uint32_t *>(&wv);
+    }
 }
 
-template <int BN>
+template <int BITS, int BN>
 __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_constant__ UmmaParams p)
 {
-    using C = Cfg<BN>;
-    constexpr int STAGES = C::kStages;
+    using C = UCfg<BITS, BN>;
+    constexpr int SX = C::SX, SD = C::SD, LEAD = C::LEAD;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t *sm = smem_raw + (base - raw);
-
-    // carve-up (all tile bases are multiples of 1024 bytes)
-    const uint32_t x_tile0 = base;
-    const uint32_t a_tile0 = x_tile0 + STAGES * C::kXTileBytes;
-    const uint32_t q_tile0 = a_tile0 + STAGES * kATileBytes;
-    const uint32_t w_tile0 = q_tile0 + STAGES * kQTileBytes;
-    const uint32_t b_tile = w_tile0 + 2 * kWTileBytes;
-    const uint32_t lut_addr = b_tile + kWTileBytes;
-    const uint32_t bars = lut_addr + kLutBytes;
-    const uint32_t bar_tma_full = bars;                 // STAGES
-    const uint32_t bar_tma_empty = bars + 8 * 4;        // STAGES
-    const uint32_t bar_s_full = bars + 8 * 8;           // 2
-    const uint32_t bar_w_full = bars + 8 * 10;          // 2
-    const uint32_t bar_w_empty = bars + 8 * 12;         // 2
-    const uint32_t bar_acc_full = bars + 8 * 14;        // 1
-    const uint32_t tmem_slot = bars + 8 * 16;           // u32
-    uint8_t *sm_q = sm + (q_tile0 - base);
-    uint8_t *sm_w = sm + (w_tile0 - base);
-    uint8_t *sm_b = sm + (b_tile - base);
-    __half2 *sm_lut = reinterpret_cast<__half2 *>(sm + (lut_addr - base));
-    volatile uint32_t *sm_tmem = reinterpret_cast<volatile uint32_t *>(sm + (tmem_slot - base));
-    __shared__ float s_levels[16];
-    __shared__ int s_last;
+    // carve-up (tile bases are multiples of 1024 bytes)
+    const uint32_t ax0 = base;                                  // SX x { A tile 8 KB | x tile }
+    const uint32_t q0 = ax0 + SX * C::AXSTAGE;                  // SQ code stages
+    const uint32_t b_tile = q0 + SQ * C::QSTAGE;                // B[128 x 64 ranks] bf16, K-major, swizzled
+    const uint32_t lut = b_tile + kBTileBytes;
+    const uint32_t red0 = lut + C::LUT_BYTES;
+    const uint32_t bars = red0 + C::RED_BYTES;
+    constexpr int kBarAxFull = 0;                       // SX: TMA bytes of the factor and activation tiles
+    constexpr int kBarAxEmpty = kBarAxFull + SX;        // SX: main MMA of the step done (commit)
+    constexpr int kBarQFull = kBarAxEmpty + SX;         // SQ
+    constexpr int kBarQEmpty = kBarQFull + SQ;          // SQ: all 16 worker warps (two steps)
+    constexpr int kBarSFull = kBarQEmpty + SQ;          // SD: scale MMA done (commit)
+    constexpr int kBarSEmpty = kBarSFull + SD;          // SD: one group has read S
+    constexpr int kBarWFull = kBarSEmpty + SD;          // WD: one group has written W^ (and converted x)
+    constexpr int kBarWEmpty = kBarWFull + WD;          // WD: main MMA of the step done (commit)
+    constexpr int kBarAccFull = kBarWEmpty + WD;        // 1
+    constexpr int kBarReduce = kBarAccFull + 1;         // 1: the epilogue warps of every CTA of the cluster
+    constexpr int kBarCount = kBarReduce + 1;
+    static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
+    const uint32_t bar_ax_full = bars + 8 * kBarAxFull, bar_ax_empty = bars + 8 * kBarAxEmpty;
+    const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
+    const uint32_t bar_s_full = bars + 8 * kBarSFull, bar_s_empty = bars + 8 * kBarSEmpty;
+    const uint32_t bar_w_full = bars + 8 * kBarWFull, bar_w_empty = bars + 8 * kBarWEmpty;
+    const uint32_t bar_acc_full = bars + 8 * kBarAccFull, bar_reduce = bars + 8 * kBarReduce;
+    const uint32_t tmem_slot = bars + 8 * kBarCount;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    // work assignment
-    const int tiles_per_split = (int)gridDim.x / p.splits;
-    const int split = (int)blockIdx.x / tiles_per_split;
-    const int tile = (int)blockIdx.x - split * tiles_per_split;
-    const int row_tile = tile / p.tok_tiles;
-    const int tok_tile = tile - row_tile * p.tok_tiles;
-    const int row0 = row_tile * BM;
-    const int tok0 = tok_tile * BN;
-    const int kb0 = split * p.kb_per_split;
-    const int nkb = min(p.kb_per_split, p.kblocks - kb0);
-
-    if (tid < 16) s_levels[tid] = p.levels[tid];
-    if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(bar_tma_full + 8 * s, 1);
-            mbar_init(bar_tma_empty + 8 * s, 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar_s_full + 8 * b, 1);
-            mbar_init(bar_w_full + 8 * b, kDequantThreads);
-            mbar_init(bar_w_empty + 8 * b, 1);
-        }
-        mbar_init(bar_acc_full, 1);
-        fence_mbar_init();
-    }
-    if (warp == kMmaWarp) {
-        tmem_alloc(tmem_slot, kTmemCols);
-        tmem_relinquish();
-    }
-    if (warp == kTmaWarp && lane == 0) {
-        tma_prefetch_desc(&p.tm_x);
-        tma_prefetch_desc(&p.tm_a);
-        tma_prefetch_desc(&p.tm_q);
-    }
-    __syncthreads();   // s_levels visible
-
-    if (warp < kDequantWarps) {
-        // level-pair table: entry e = (L[e & 15], L[e >> 4]) as fp16x2, one private copy per lane
-        // (word e*32 + lane sits in bank `lane`: lookups never conflict)
-        for (int e0 = 0; e0 < 256; e0 += kDequantWarps) {
-            const int e = e0 + warp;
-            sm_lut[e * 32 + lane] = __floats2half2_rn(s_levels[e & 15], s_levels[e >> 4]);
-        }
-        // B tile: 128 rows x 64 ranks (zero padded) bf16, K-major, 128-byte swizzle
-        {
-            const int rr = tid >> 1, half = tid & 1;
-            const int i = row0 + rr;
-            for (int c = 0; c < 4; ++c) {
-                const int chunk = half * 4 + c;
-                uint32_t w4[4];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int k = chunk * 8 + e * 2;
-                    uint32_t lo = (i < p.m && k < p.r) ? p.B[(size_t)i * p.r + k] : 0u;
-                    uint32_t hi = (i < p.m && k + 1 < p.r) ? p.B[(size_t)i * p.r + k + 1] : 0u;
-                    w4[e] = lo | (hi << 16);
-                }
-                uint8_t *dst = sm_b + (rr >> 3) * 1024 + (rr & 7) * 128 + ((chunk ^ (rr & 7)) * 16);
-                *reinterpret_cast<uint4 *>(dst) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-            }
-        }
-        fence_proxy_async_smem();
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem_base = *sm_tmem;
+    // work assignment: cluster = one (row tile, token tile); rank = slice of its k-range
+    const int csize = (int)cluster_nctarank(), rank = (int)cluster_ctarank();
+    const int tile = (int)blockIdx.x / csize;
+    const int row_tile = tile / p.tok_tiles, tok_tile = tile - row_tile * p.tok_tiles;
+    const int row0 = row_tile * BM, tok0 = tok_tile * BN;
+    const int pa = (int)((long long)rank * p.npairs / csize), pb = (int)((long long)(rank + 1) * p.npairs / csize);
+    const int pairs = pb - pa;
+    const int total = 2 * pairs;          // k-steps of this CTA; global k-step = 2 * pa + it
 
     bool failed = false;
 
     if (warp == kTmaWarp) {
         // ------------------------------------------------------------------ TMA producer
+        // It also initialises the barriers and starts the weight stream before the rest of the CTA
+        // has finished its set-up.
+        for (int b = lane; b < kBarCount; b += 32) {
+            uint32_t count = 1;
+            if (b >= kBarQEmpty && b < kBarSFull) count = kWorkWarps;
+            else if (b >= kBarSEmpty && b < kBarWEmpty) count = kGroupWarps;   // s_empty and w_full
+            else if (b == kBarReduce) count = (uint32_t)(4 * csize);
+            mbar_init(bars + 8 * b, count);
+        }
+        fence_mbar_init();
+        __syncwarp();
+        asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");   // barriers exist; does not wait for the others
+        // split-phase cluster barrier: the fence above has published this CTA's barriers cluster-wide,
+        // a relaxed arrival is enough; the wait is in the epilogue before the first remote access
+        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
         if (lane == 0) {
-            const uint32_t stage_tx = (uint32_t)(C::kXTileBytes + p.r_pad * 128 + kQTileBytes);
-            for (int it = 0; it < nkb; ++it) {
-                const int st = it % STAGES;
-                if (it >= STAGES && !mbar_wait(bar_tma_empty + 8 * st, (uint32_t)((it / STAGES - 1) & 1))) {
-                    failed = true;
-                    break;
-                }
-                LORDS_STAMP(2, it, 0);
-                const int j0 = (kb0 + it) * BK;
-                const uint32_t bar = bar_tma_full + 8 * st;
-                mbar_expect_tx(bar, stage_tx);
-                tma_load_2d(q_tile0 + st * kQTileBytes, &p.tm_q, j0 / 2, row0, bar);
-                tma_load_2d(a_tile0 + st * kATileBytes, &p.tm_a, j0, 0, bar);
-                tma_load_2d(x_tile0 + st * C::kXTileBytes, &p.tm_x, j0, tok0, bar);
-                LORDS_STAMP(2, it, 1);
+            tma_prefetch_desc(&p.tm_q);
+            tma_prefetch_desc(&p.tm_a);
+            tma_prefetch_desc(&p.tm_x);
+            // the first code stages are weights: start them before anything else
+            const int pre = pairs < SQ ? pairs : SQ;
+            for (int pr = 0; pr < pre; ++pr) {
+                const uint32_t bar = bar_q_full + 8 * pr;
+                mbar_expect_tx(bar, (uint32_t)C::QSTAGE);
+                tma_load_2d(q0 + pr * C::QSTAGE, &p.tm_q, (pa + pr) * C::QROW, row0, bar);
             }
-        }
-    } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = umma_idesc_f16(1, 0, 1, BM, 64);     // bf16, B operand MN-major
-            constexpr uint32_t idesc_m = umma_idesc_f16(0, 0, 0, BM, BN);     // fp16, both K-major
-            const int ksteps = p.r_pad / 16;
-            auto issue_scale = [&](int it) -> bool {
-                const int st = it % STAGES, buf = it & 1;
-                if (!mbar_wait(bar_tma_full + 8 * st, (uint32_t)((it / STAGES) & 1))) return false;
-                tc_fence_after_sync();
-                for (int k = 0; k < ksteps; ++k) {
-                    const uint64_t ad = umma_desc_sw128(b_tile + k * 32, 1024, 16);
-                    const uint64_t bd = umma_desc_sw128(a_tile0 + st * kATileBytes + k * 2048, 1024, 16);
-                    umma_f16_ss(tmem_base + kSCol + buf * 64, ad, bd, idesc_s, k > 0);
-                }
-                umma_commit(bar_s_full + 8 * buf);
-                return true;
-            };
-            bool ok = nkb > 0 ? issue_scale(0) : true;
-            if (ok && nkb > 1) ok = issue_scale(1);
-            for (int it = 0; ok && it < nkb; ++it) {
-                const int st = it % STAGES, buf = it & 1;
-                LORDS_STAMP(0, it, 0);
-                if (!mbar_wait(bar_w_full + 8 * buf, (uint32_t)((it >> 1) & 1))) { ok = false; break; }
-                tc_fence_after_sync();
-                LORDS_STAMP(0, it, 1);
-#pragma unroll
-                for (int k = 0; k < BK / 16; ++k) {
-                    const uint64_t ad = umma_desc_sw128(w_tile0 + buf * kWTileBytes + k * 32, 1024, 16);
-                    const uint64_t bd = umma_desc_sw128(x_tile0 + st * C::kXTileBytes + k * 32, 1024, 16);
-                    umma_f16_ss(tmem_base, ad, bd, idesc_m, (it > 0 || k > 0) ? 1u : 0u);
-                }
-                umma_commit(bar_tma_empty + 8 * st);
-                umma_commit(bar_w_empty + 8 * buf);
-                LORDS_STAMP(0, it, 2);
-                if (it + 2 < nkb) ok = issue_scale(it + 2);
-                LORDS_STAMP(0, it, 3);
-            }
-            umma_commit(bar_acc_full);
-            failed = !ok;
-        }
-    } else {
-        // ------------------------------------------------------------------ dequant warps
-        const int quad = warp & 3, half = warp >> 2;
-        const int row = quad * 32 + lane;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-        const __half2 *lut = sm_lut + lane;
-        for (int it = 0; it < nkb; ++it) {
-            const int st = it % STAGES, buf = it & 1;
-            if (tid == 0) LORDS_STAMP(1, it, 0);
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * buf, (uint32_t)((it >> 1) & 1)))) { failed = true; break; }
-            tc_fence_after_sync();
-            if (tid == 0) LORDS_STAMP(1, it, 1);
-            uint32_t s[32];
-            tmem_ld_32x32(lane_addr + kSCol + buf * 64 + half * 32, s);
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_tma_full + 8 * st, (uint32_t)((it / STAGES) & 1)))) {
-                tmem_wait_ld();
-                failed = true;
-                break;
-            }
-            const uint4 cw = *reinterpret_cast<const uint4 *>(sm_q + st * kQTileBytes + row * 32 + half * 16);
-            tmem_wait_ld();
-            if (tid == 0) LORDS_STAMP(1, it, 2);
-            const uint32_t cwv[4] = {cw.x, cw.y, cw.z, cw.w};
-            uint32_t out[16];
-#pragma unroll
-            for (int b = 0; b < 16; ++b) {
-                const uint32_t byte = (cwv[b >> 2] >> (8 * (b & 3))) & 0xFFu;
-                const __half2 lv = lut[byte * 32];
-                const __half2 sv = __floats2half2_rn(__uint_as_float(s[2 * b]), __uint_as_float(s[2 * b + 1]));
-                const __half2 wv = __hmul2(lv, sv);
-                out[b] = *reinterpret_cast<const uint32_t *>(&wv);
-            }
-            if (it >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar_w_empty + 8 * buf, (uint32_t)(((it >> 1) - 1) & 1)))) {
-                failed = true;
-                break;
-            }
-            if (tid == 0) LORDS_STAMP(1, it, 3);
-            uint8_t *wrow = sm_w + buf * kWTileBytes + (row >> 3) * 1024 + (row & 7) * 128;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const int chunk = (half * 4 + c) ^ (row & 7);
-                *reinterpret_cast<uint4 *>(wrow + chunk * 16) =
-                    make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
-            }
-            if (tid == 0) LORDS_STAMP(1, it, 4);
-            fence_proxy_async_smem();
-            tc_fence_before_sync();
-            if (tid == 0) LORDS_STAMP(1, it, 5);
-            mbar_arrive(bar_w_full + 8 * buf);
-            if (tid == 0) LORDS_STAMP(1, it, 6);
-        }
-
-        // ------------------------------------------------------------------ epilogue
-        if (!failed && !__all_sync(0xffffffffu, mbar_wait(bar_acc_full, 0))) failed = true;
-        failed = __any_sync(0xffffffffu, failed);
-        tc_fence_after_sync();
-        if (!failed && nkb > 0) {
-            const int i = row0 + row;
-            constexpr int kColsPerHalf = BN >= 32 ? BN / 2 : BN;
-            const bool active = BN >= 32 || half == 0;
-            if (active) {
-                for (int c0 = half * kColsPerHalf; c0 < (half + 1) * kColsPerHalf; c0 += 16) {
-                    uint32_t v[16];
-                    tmem_ld_32x16(lane_addr + c0, v);
-                    tmem_wait_ld();
-                    if (i < p.m) {
-#pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const int t = tok0 + c0 + c;
-                            if (t < p.M) {
-                                const float f = __uint_as_float(v[c]);
-                                if (p.splits > 1) p.partial[((size_t)split * p.M + t) * p.m + i] = f;
-                                else store_out(p.y, p.y_f32, (size_t)t * p.m + i, f);
-                            }
-                        }
+            // x may be the previous launch's output
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            const uint32_t ax_tx = (uint32_t)(p.r_pad * 128 + C::XTILE);
+            for (int it = 0; it < total; ++it) {
+                const int sx = it % SX;
+                if (it >= SX && !mbar_wait(bar_ax_empty + 8 * sx, (uint32_t)((it / SX - 1) & 1))) { failed = true; break; }
+                const int j0 = (2 * pa + it) * BK;
+                const uint32_t bar = bar_ax_full + 8 * sx;
+                mbar_expect_tx(bar, ax_tx);
+                tma_load_2d(ax0 + sx * C::AXSTAGE, &p.tm_a, j0, 0, bar);
+                tma_load_2d(ax0 + sx * C::AXSTAGE + kATileBytes, &p.tm_x, j0, tok0, bar);
+                if ((it & 1) == 0 && it >= 2) {
+                    // refill the code stage of the pair whose two k-steps both have their tiles by now
+                    const int pr = it / 2 - 1 + SQ;
+                    if (pr < pairs) {
+                        const int sq = pr % SQ;
+                        if (!mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((pr / SQ - 1) & 1))) { failed = true; break; }
+                        const uint32_t qbar = bar_q_full + 8 * sq;
+                        mbar_expect_tx(qbar, (uint32_t)C::QSTAGE);
+                        tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (pa + pr) * C::QROW, row0, qbar);
                     }
                 }
             }
         }
-        tc_fence_before_sync();
-
-        if (p.splits > 1) {
-            // last CTA of this (row tile, token tile) to arrive adds the partials in split order
-            __threadfence();
-            named_bar_sync(1, kDequantThreads);
-            if (tid == 0) {
-                const int prev = atomicAdd(p.counters + tile, 1);
-                const int last = (prev == p.splits - 1);
-                if (last) p.counters[tile] = 0;
-                s_last = last;
+    } else {
+        if (warp == kIssuerWarp) {
+            tmem_alloc(tmem_slot, kTmemCols);
+            tmem_relinquish();
+        } else {
+            // level-pair table: entry e = (L[lo code], L[hi code]) as fp16x2; word e*32 + lane is lane's
+            // copy (bank = lane, so the lookups of a warp never conflict)
+#pragma unroll
+            for (int i = 0; i < C::LUT_ENTRIES / kWorkWarps; ++i) {
+                const int entry = warp + kWorkWarps * i;
+                const int lo = BITS == 4 ? (entry & 15) : (entry & 7);
+                const int hi = BITS == 4 ? (entry >> 4) : (entry >> 3);
+                const __half2 v = __floats2half2_rn(p.levels[lo], p.levels[hi]);
+                sts_u32(lut + 4u * (uint32_t)(entry * 32 + lane), *reinterpret_cast<const uint32_t *>(&v));
             }
-            named_bar_sync(1, kDequantThreads);
-            if (s_last) {
-                __threadfence();
-                const int ntok = min(BN, p.M - tok0);
-                const int rr = tid & (BM - 1);
+            // B tile: 128 rows x 64 ranks (zero padded) bf16, K-major, 128-byte swizzle
+            if (tid < 256) {
+                const int rr = tid >> 1, half = tid & 1;
                 const int i = row0 + rr;
-                if (i < p.m) {
-                    for (int tt = tid >> 7; tt < ntok; tt += kDequantThreads / BM) {
-                        const int t = tok0 + tt;
-                        float acc = 0.0f;
-                        for (int s = 0; s < p.splits; ++s) acc += __ldcg(p.partial + ((size_t)s * p.M + t) * p.m + i);
-                        store_out(p.y, p.y_f32, (size_t)t * p.m + i, acc);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const int chunk = half * 4 + c;
+                    uint32_t w4[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int k = chunk * 8 + e * 2;
+                        const uint32_t lo = (i < p.m && k < p.r) ? p.B[(size_t)i * p.r + k] : 0u;
+                        const uint32_t hi = (i < p.m && k + 1 < p.r) ? p.B[(size_t)i * p.r + k + 1] : 0u;
+                        w4[e] = lo | (hi << 16);
+                    }
+                    sts_v4(b_tile + (rr >> 3) * 1024 + (rr & 7) * 128 + ((chunk ^ (rr & 7)) * 16),
+                           make_uint4(w4[0], w4[1], w4[2], w4[3]));
+                }
+            }
+            fence_proxy_async_smem();
+        }
+        tc_fence_before_sync();
+        asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");   // tables, TMEM address and barriers are in place
+        tc_fence_after_sync();
+        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+    }
+    // let a dependent launch begin its own weight prefetch as SMs become free
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    if (warp == kTmaWarp) {
+        // all done above
+    } else if (warp == kIssuerWarp) {
+        // ------------------------------------------------------------------ MMA issuer
+        uint32_t tmem_base;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+        constexpr uint32_t idesc_s = umma_idesc_f16(1, 0, 1, BM, 64);     // bf16, B operand MN-major, N = 64
+        constexpr uint32_t idesc_m = umma_idesc_f16(0, 0, 0, BM, BN);     // fp16, K-major
+        const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
+        const uint32_t lbo_lo = (uint32_t)umma_desc_sw128(0, 1024, 16);
+        const uint32_t b_lo = lbo_lo | ((b_tile & 0x3FFFFu) >> 4);
+        const uint32_t ax_lo0 = lbo_lo | ((ax0 & 0x3FFFFu) >> 4);
+        const int ksteps = p.r_pad / 16;
+        // scale MMA of step j into S buffer j % SD
+        auto issue_scale = [&](int j) -> bool {
+            const int sx = j % SX, sd = j % SD;
+            if (!mbar_wait(bar_ax_full + 8 * sx, (uint32_t)((j / SX) & 1))) return false;
+            if (j >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((j / SD - 1) & 1))) return false;
+            tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t a_lo = ax_lo0 + (uint32_t)(sx * (C::AXSTAGE >> 4));
+                for (int k = 0; k < ksteps; ++k)
+                    umma_f16_ss(tmem_base + C::SCOL + sd * 64, umma_desc_pack(b_lo + k * 2, desc_hi),
+                                umma_desc_pack(a_lo + k * 128, desc_hi), idesc_s, k > 0);
+                umma_commit(bar_s_full + 8 * sd);
+            }
+            __syncwarp();
+            return true;
+        };
+        // The scale MMA of step it + LEAD is queued ahead of the main MMA of step it.  LEAD <= SD
+        // (its S buffer is free once the workers have read step it + LEAD - SD) and LEAD < SX (its
+        // factor tile needs the ring stage of step it + LEAD - SX, whose main MMA is already queued).
+        bool ok = true;
+        for (int j = 0; ok && j < LEAD && j < total; ++j) ok = issue_scale(j);
+        for (int it = 0; ok && it < total; ++it) {
+            const int sx = it % SX, ws = it % WD;
+            if (it + LEAD < total) ok = issue_scale(it + LEAD);
+            if (!ok) break;
+            if (!mbar_wait(bar_w_full + 8 * ws, (uint32_t)((it / WD) & 1))) { ok = false; break; }
+            tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t wslot = tmem_base + kWCol + (uint32_t)(ws * 32);
+                const uint32_t x_lo = ax_lo0 + (uint32_t)((sx * C::AXSTAGE + kATileBytes) >> 4);
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    umma_f16_ts(tmem_base, wslot + k * 8, umma_desc_pack(x_lo + k * 2, desc_hi), idesc_m,
+                                (it > 0 || k > 0) ? 1u : 0u);
+                umma_commit(bar_ax_empty + 8 * sx);
+                umma_commit(bar_w_empty + 8 * ws);
+                if (it == total - 1) umma_commit(bar_acc_full);
+            }
+            __syncwarp();
+        }
+        failed = !ok;
+    } else {
+        // ------------------------------------------------------------------ worker warps
+        const int g = warp / kGroupWarps, wg = warp % kGroupWarps, q = warp & 3, ch = wg >> 2;
+        const int row = q * 32 + lane;
+        uint32_t tmem_base;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t lut_lane = lut + 4u * (uint32_t)lane;
+
+        for (int it = g; it < total; it += 2) {
+            const int sx = it % SX, sd = it % SD, ws = it % WD, pr = it >> 1, sq = pr % SQ;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * sd, (uint32_t)((it / SD) & 1)))) { failed = true; break; }
+            tc_fence_after_sync();
+            uint32_t s[32];
+            tmem_ld_32x32(lane_addr + C::SCOL + (uint32_t)(sd * 64 + ch * 32), s);
+            bool ok = mbar_wait(bar_q_full + 8 * sq, (uint32_t)((pr / SQ) & 1));
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_s_empty + 8 * sd);      // S is in registers: the buffer may be refilled
+            if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+            uint32_t out[16];
+            dequant_chunk<BITS>(q0 + sq * C::QSTAGE + row * C::QROW, row, (it & 1) * 2 + ch, lut_lane, s, out);
+            if constexpr (C::kConvertInKernel) {
+                // The activation tile arrived as bf16 (16 tokens x 64 columns, together with the factor
+                // tile the scale MMA has already consumed): convert it in place, one 16-byte chunk per
+                // thread of the first four warps of the group (element-wise, so the swizzled position
+                // of the chunk does not matter).
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_ax_full + 8 * sx, (uint32_t)((it / SX) & 1)))) { failed = true; break; }
+                if (wg < 4) {
+                    const uint32_t addr = ax0 + sx * C::AXSTAGE + kATileBytes + (uint32_t)((wg * 32 + lane) * 16);
+                    const uint4 v = lds_v4(addr);
+                    const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+                    uint32_t o[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const __half2 hv = __floats2half2_rn(__uint_as_float(in[e] << 16), __uint_as_float(in[e] & 0xFFFF0000u));
+                        o[e] = *reinterpret_cast<const uint32_t *>(&hv);
+                    }
+                    sts_v4(addr, make_uint4(o[0], o[1], o[2], o[3]));
+                }
+                fence_proxy_async_smem();
+            }
+            if (it >= WD && !__all_sync(0xffffffffu, mbar_wait(bar_w_empty + 8 * ws, (uint32_t)((it / WD - 1) & 1)))) {
+                failed = true;
+                break;
+            }
+            tc_fence_after_sync();
+            tmem_st_32x16(lane_addr + kWCol + (uint32_t)(ws * 32 + ch * 16), out);
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(bar_w_full + 8 * ws);
+                mbar_arrive(bar_q_empty + 8 * sq);
+            }
+        }
+
+        // ------------------------------------------------------------------ epilogue
+        constexpr int CPG = BN >= 64 ? BN / 4 : 16;      // accumulator columns per warp column group
+        const int cg = warp >> 2;
+        if (cg * CPG < BN && !failed) {
+            bool ok = true;
+            if (total > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, 0));
+            tc_fence_after_sync();
+            const int i = row0 + row;
+            if (!ok) failed = true;
+            if (BN > 16 || csize == 1) {
+                if (ok && total > 0) {
+#pragma unroll 1
+                    for (int c0 = cg * CPG; c0 < (cg + 1) * CPG; c0 += 16) {
+                        uint32_t v[16];
+                        tmem_ld_32x16(lane_addr + (uint32_t)c0, v);
+                        tmem_wait_ld();
+                        if (i < p.m) {
+#pragma unroll
+                            for (int c = 0; c < 16; ++c) {
+                                const int t = tok0 + c0 + c;
+                                if (t < p.M) store_out(p.y, p.y_f32, (size_t)t * p.m + i, __uint_as_float(v[c]));
+                            }
+                        }
+                    }
+                }
+            } else {
+                // BN == 16 with the k-range split over the cluster: park the partials in the leader's
+                // shared memory; a CTA that gave up still arrives (with zeros)
+                uint32_t v[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) v[c] = 0u;
+                if (ok && total > 0) {
+                    tmem_ld_32x16(lane_addr, v);
+                    tmem_wait_ld();
+                }
+                asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+#pragma unroll
+                for (int c = 0; c < 16; ++c)
+                    st_cluster_f32(map_to_rank(red0 + (uint32_t)(((rank * 16 + c) * BM + row) * 4), 0), __uint_as_float(v[c]));
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_rank(bar_reduce, 0));
+                if (rank == 0) {
+                    if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0))) failed = true;
+                    else if (i < p.m) {
+#pragma unroll 1
+                        for (int c = 0; c < 16; ++c) {
+                            const int t = tok0 + c;
+                            if (t >= p.M) break;
+                            float a = 0.0f;
+                            for (int rr = 0; rr < csize; ++rr)
+                                a += __uint_as_float(lds_u32(red0 + (uint32_t)(((rr * 16 + c) * BM + row) * 4)));
+                            store_out(p.y, p.y_f32, (size_t)t * p.m + i, a);
+                        }
                     }
                 }
             }
@@ -366,10 +437,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
     }
 
     if (failed) atomicExch(p.status, LORDS_ERR_TIMEOUT);
+    tc_fence_before_sync();
     __syncthreads();
-    if (warp == kMmaWarp) {
-        __syncwarp();
+    if (warp == kIssuerWarp) {
         tc_fence_after_sync();
+        uint32_t tmem_base;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         tmem_dealloc(tmem_base, kTmemCols);
     }
 }
@@ -418,108 +491,145 @@ bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const
     cuuint64_t strides[1] = {inner * (uint64_t)elem_bytes};
     cuuint32_t box[2] = {box_inner, box_outer};
     cuuint32_t estr[2] = {1, 1};
-    CUresult rc = fn(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return rc == CUDA_SUCCESS;
+    return fn(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN> int launch_bn(const UmmaParams &k, int grid, cudaStream_t stream)
-{
-    static bool attr_set = false;
-    if (!attr_set) {
-        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_umma_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            Cfg<BN>::kSmemBytes));
-        attr_set = true;
+template <int BITS, int BN> struct UmmaVariant {
+    static int prepare()
+    {
+        static bool done = false;
+        if (!done) {
+            LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_umma_kernel<BITS, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                UCfg<BITS, BN>::SMEM));
+            done = true;
+        }
+        return LORDS_OK;
     }
-    lords_umma_kernel<BN><<<grid, kThreads, Cfg<BN>::kSmemBytes, stream>>>(k);
-    LORDS_CUDA_TRY(cudaGetLastError());
+    static void fill(cudaLaunchConfig_t &cfg, cudaLaunchAttribute *attr, int cs, int clusters, cudaStream_t stream)
+    {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        // programmatic dependent launch: the kernel touches only weights until its griddepcontrol.wait
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg = cudaLaunchConfig_t{};
+        cfg.gridDim = dim3((unsigned)(clusters * cs));
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = UCfg<BITS, BN>::SMEM;
+        cfg.stream = stream;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+    }
+    // Clusters of `cs` CTAs that can be resident at the same time (0 if such a cluster cannot run).
+    static int max_clusters(int cs)
+    {
+        static int cache[kClusterMax + 1];   // 0 = not asked yet, -1 = cannot run
+        if (cache[cs] == 0) {
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attr[2];
+            fill(cfg, attr, cs, 1, nullptr);
+            int n = 0;
+            const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_umma_kernel<BITS, BN>, &cfg);
+            if (e != cudaSuccess) (void)cudaGetLastError();
+            cache[cs] = (e == cudaSuccess && n >= 1) ? n : -1;
+        }
+        return cache[cs] > 0 ? cache[cs] : 0;
+    }
+    static int launch(const UmmaParams &k, int tiles, int cs, cudaStream_t stream)
+    {
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attr[2];
+        fill(cfg, attr, cs, tiles, stream);
+        LORDS_CUDA_TRY(cudaLaunchKernelEx(&cfg, lords_umma_kernel<BITS, BN>, k));
+        return LORDS_OK;
+    }
+};
+
+template <int BITS, int BN> int launch_variant(UmmaParams &k, const Problem &p, State &st, cudaStream_t stream)
+{
+    using V = UmmaVariant<BITS, BN>;
+    int rc = V::prepare();
+    if (rc != LORDS_OK) return rc;
+    k.tok_tiles = (p.M + BN - 1) / BN;
+    const int row_tiles = (p.m + BM - 1) / BM;
+    const long long tiles = (long long)row_tiles * k.tok_tiles;
+    if (tiles > 0x3fffffffLL) return LORDS_ERR_UNSUPPORTED;
+
+    // k-split over a cluster: only the BN = 16 kernel has the shared-memory reduction
+    int cs = 1;
+    if (BN == 16) {
+        const bool forced = st.forced_splitk > 0;
+        const long long want = forced ? st.forced_splitk : st.sm_count / tiles;
+        int lim = want < kClusterMax ? (int)want : kClusterMax;
+        if (lim > k.npairs) lim = k.npairs;
+        for (int c = lim; c > 1; --c)
+            if (V::max_clusters(c) >= (forced ? 1 : tiles)) { cs = c; break; }
+    }
+
+    const void *xsrc = p.x;
+    if (!UCfg<BITS, BN>::kConvertInKernel) {
+        const size_t x16_bytes = (size_t)p.M * p.n * 2;
+        if (x16_bytes > st.workspace_bytes) return LORDS_ERR_WORKSPACE;
+        const size_t n_vec = (size_t)p.M * p.n / 8;
+        lords_x_to_f16_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, stream>>>(
+            reinterpret_cast<const uint4 *>(p.x), reinterpret_cast<uint4 *>(st.workspace), n_vec);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        xsrc = st.workspace;
+    }
+    const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
+    if (!make_map_2d(&k.tm_x, UCfg<BITS, BN>::kConvertInKernel ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16,
+                     2, xsrc, (uint64_t)p.n, (uint64_t)p.M, 64, (uint32_t)BN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.A, (uint64_t)p.n, (uint64_t)p.r, 64, (uint32_t)k.r_pad,
+                     CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)UCfg<BITS, BN>::QROW, BM,
+                     BITS == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE))
+        return LORDS_ERR_CUDA;
+    rc = V::launch(k, (int)tiles, cs, stream);
+    if (rc != LORDS_OK) return rc;
+    st.last_launches = UCfg<BITS, BN>::kConvertInKernel ? 1 : 2;
     return LORDS_OK;
+}
+
+template <int BITS> int launch_bits(UmmaParams &k, const Problem &p, State &st, cudaStream_t stream)
+{
+    if (p.M <= 16) return launch_variant<BITS, 16>(k, p, st, stream);
+    // token tile: the largest that still gives CTAs for most of the SMs
+    const long long row_tiles = (p.m + BM - 1) / BM;
+    int bn = 256;
+    while (bn > 32 && (p.M <= bn / 2 || 5 * row_tiles * ((p.M + bn - 1) / bn) < 3 * (long long)st.sm_count)) bn /= 2;
+    if (st.forced_bn > 0) bn = st.forced_bn;   // measurement switch
+    switch (bn) {
+        case 32: return launch_variant<BITS, 32>(k, p, st, stream);
+        case 64: return launch_variant<BITS, 64>(k, p, st, stream);
+        case 128: return launch_variant<BITS, 128>(k, p, st, stream);
+        default: return launch_variant<BITS, 256>(k, p, st, stream);
+    }
 }
 
 }  // namespace
 
-// Returns LORDS_ERR_UNSUPPORTED when the shape is outside this path's rules:
-// 4-bit codes, n a multiple of 64, r <= 64, scratch large enough.
+// Rules of this path: 3- or 4-bit codes; r <= 64; n a multiple of 64 (4-bit) or 128 (3-bit), which
+// makes every TMA row pitch a multiple of 16 bytes.  Anything else: LORDS_ERR_UNSUPPORTED.
 int launch_umma(const Problem &p, State &st, cudaStream_t stream)
 {
-    if (p.bits != 4 || p.n % 64 != 0 || p.r > kRMaxUmma) return LORDS_ERR_UNSUPPORTED;
+    if (p.bits != 3 && p.bits != 4) return LORDS_ERR_UNSUPPORTED;
+    if (p.r > kRMaxUmma || p.n % (p.bits == 4 ? 64 : 128) != 0) return LORDS_ERR_UNSUPPORTED;
 
-    const int BN = p.M <= 16 ? 16 : p.M <= 32 ? 32 : p.M <= 64 ? 64 : p.M <= 128 ? 128 : 256;
     UmmaParams k;
     k.B = p.B;
     for (int c = 0; c < 16; ++c) k.levels[c] = p.levels[c];
     k.M = p.M; k.m = p.m; k.n = p.n; k.r = p.r;
     k.r_pad = (p.r + 15) / 16 * 16;
-    k.kblocks = p.n / BK;
-    k.tok_tiles = (p.M + BN - 1) / BN;
-    const int row_tiles = (p.m + BM - 1) / BM;
-    const long tiles = (long)row_tiles * k.tok_tiles;
-    if (tiles > st.counter_slots) return LORDS_ERR_UNSUPPORTED;
-
-    int splits = st.forced_splitk;
-    if (splits <= 0) {
-        splits = (int)(st.sm_count / tiles);                 // one wave: never more CTAs than SMs
-        if (splits > k.kblocks / 4) splits = k.kblocks / 4;  // at least 4 k-blocks per CTA
-        if (splits < 1) splits = 1;
-    }
-    if (splits > k.kblocks) splits = k.kblocks;
-    k.kb_per_split = (k.kblocks + splits - 1) / splits;
-    splits = (k.kblocks + k.kb_per_split - 1) / k.kb_per_split;
-    k.splits = splits;
-
-    // scratch: [ x as fp16 | split-K partials ]
-    const size_t x16_bytes = ((size_t)p.M * p.n * 2 + 1023) & ~(size_t)1023;
-    const size_t part_bytes = splits > 1 ? (size_t)splits * p.M * p.m * sizeof(float) : 0;
-    if (x16_bytes + part_bytes > st.workspace_bytes) return LORDS_ERR_WORKSPACE;
-    uint8_t *x16 = st.workspace;
-    k.partial = reinterpret_cast<float *>(st.workspace + x16_bytes);
-    k.counters = st.counters;
+    k.npairs = (p.n + 127) / 128;
     k.y = p.y; k.y_f32 = p.y_f32;
     k.status = st.status_word;
-#ifdef LORDS_TRACE
-    k.trace = reinterpret_cast<long long *>(st.workspace + st.workspace_bytes - (size_t)3 * 64 * 8 * 8);
-    LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)3 * 64 * 8 * 8, stream));
-#endif
-
-    if (!make_map_2d(&k.tm_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, x16, (uint64_t)p.n, (uint64_t)p.M, 64, (uint32_t)BN,
-                     CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.A, (uint64_t)p.n, (uint64_t)p.r, 64,
-                     (uint32_t)k.r_pad, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, (uint64_t)p.n / 2, (uint64_t)p.m, 32, BM,
-                     CU_TENSOR_MAP_SWIZZLE_NONE))
-        return LORDS_ERR_CUDA;
-
-    const size_t n_vec = (size_t)p.M * p.n / 8;
-    lords_x_to_f16_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, stream>>>(
-        reinterpret_cast<const uint4 *>(p.x), reinterpret_cast<uint4 *>(x16), n_vec);
-    LORDS_CUDA_TRY(cudaGetLastError());
-
-    const int grid = (int)(tiles * splits);
-    int rc;
-    switch (BN) {
-        case 16: rc = launch_bn<16>(k, grid, stream); break;
-        case 32: rc = launch_bn<32>(k, grid, stream); break;
-        case 64: rc = launch_bn<64>(k, grid, stream); break;
-        case 128: rc = launch_bn<128>(k, grid, stream); break;
-        default: rc = launch_bn<256>(k, grid, stream); break;
-    }
+    const int rc = p.bits == 4 ? launch_bits<4>(k, p, st, stream) : launch_bits<3>(k, p, st, stream);
     if (rc != LORDS_OK) return rc;
-    st.last_launches = 2;
     st.last_path = "umma";
     return LORDS_OK;
 }
-
-#ifdef LORDS_TRACE
-// Debug builds only: copy CTA 0's clock stamps of the last tensor-core launch to the host.
-extern "C" int lords_debug_read_trace(long long *out)
-{
-    State &st = state();
-    if (!st.initialised) return LORDS_ERR_NOT_INIT;
-    LORDS_CUDA_TRY(cudaDeviceSynchronize());
-    LORDS_CUDA_TRY(cudaMemcpy(out, st.workspace + st.workspace_bytes - (size_t)3 * 64 * 8 * 8, (size_t)3 * 64 * 8 * 8,
-                              cudaMemcpyDeviceToHost));
-    return LORDS_OK;
-}
-#endif
 
 }  // namespace lords

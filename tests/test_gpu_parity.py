@@ -20,6 +20,7 @@ def lords():
     yield binding
     binding.lords_set_option("path", "auto")
     binding.lords_set_option("splitk", "0")
+    binding.lords_set_option("bn", "0")
     binding.lords_shutdown()
 
 
@@ -156,6 +157,49 @@ def test_decode_kernel_declines_what_it_cannot_run(lords):
         assert ei.value.status == -11
     finally:
         lords.lords_set_option("path", "auto")
+
+
+# ---- the scale-MMA kernel, forced; token tiles forced too so that every instantiation runs ----------
+
+UMMA_SHAPES = [
+    # bits, m, n, r, M, bn, mixed
+    (4, 384, 1024, 32, 5, 0, True),
+    (3, 260, 1152, 48, 16, 0, True),
+    (3, 128, 256, 16, 2, 0, False),
+    (4, 130, 128, 64, 1, 0, False),      # one pair of k-steps, largest rank
+    (4, 256, 2048, 24, 40, 32, True),
+    (3, 200, 1024, 32, 70, 64, False),
+    (4, 300, 1536, 16, 100, 128, True),
+    (3, 384, 1280, 48, 300, 256, False),
+    (4, 256, 1024, 8, 257, 256, True),   # a second token tile with one token in it
+]
+
+
+@pytest.mark.parametrize("bits,m,n,r,M,bn,mixed", UMMA_SHAPES)
+def test_umma_kernel_shapes(lords, bits, m, n, r, M, bn, mixed):
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=5 * m + n + r + M, mixed_sign=mixed)
+    lords.lords_set_option("bn", str(bn))
+    try:
+        dl, y32, ybf = _run(lords, lay, "umma")
+    finally:
+        lords.lords_set_option("bn", "0")
+    assert lords.lords_last_path() == "umma"
+    check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
+
+
+@pytest.mark.parametrize("bits,m,n,r,M,bn", [(4, 256, 512, 32, 16, 0), (3, 131, 384, 7, 9, 0), (4, 140, 256, 16, 33, 32),
+                                             (3, 256, 512, 48, 200, 256)])
+def test_umma_kernel_integer_case_is_bit_exact(lords, bits, m, n, r, M, bn):
+    lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m + M)
+    lords.lords_set_option("bn", str(bn))
+    try:
+        dl, y32, ybf = _run(lords, lay, "umma")
+    finally:
+        lords.lords_set_option("bn", "0")
+    assert lords.lords_last_path() == "umma"
+    y64 = _oracle(lay, dl.packed_host)
+    assert np.array_equal(y32.astype(np.float64), y64)
+    assert np.array_equal(ybf, oracle.round_bf16(y64))
 
 
 def test_linearity_on_gpu(lords):
