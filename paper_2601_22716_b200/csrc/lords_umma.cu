@@ -50,7 +50,9 @@ constexpr int kClusterMax = 8;                 // largest k-split (cluster size)
 template <int BITS, int BN> struct UCfg {
     static constexpr int QROW = 128 * BITS / 8;                  // packed bytes per row per code stage (64 / 48)
     static constexpr int QSTAGE = BM * QROW;
-    static constexpr int SX = BN >= 256 ? 3 : 4;                 // factor / activation ring depth
+    // factor / activation ring depth: as deep as shared memory allows, the tiles come from L2 with a
+    // latency of several k-steps
+    static constexpr int SX = BN >= 256 ? 3 : BN >= 128 ? 5 : 8;
     static constexpr int XTILE = BN * 128;
     static constexpr int AXSTAGE = kATileBytes + XTILE;
     static constexpr uint32_t SCOL = BN > 128 ? 256 : 128;       // S ring starts behind the accumulator
@@ -76,7 +78,22 @@ struct alignas(64) UmmaParams {
     void *y;
     int y_f32;
     int *status;
+#ifdef LORDS_TRACE
+    long long *trace;     // [8 roles][32 iterations][8 events] clock64 stamps of one CTA (debug builds only)
+#endif
 };
+
+#ifdef LORDS_TRACE
+#ifndef LORDS_TRACE_CTA
+#define LORDS_TRACE_CTA 0
+#endif
+#define USTAMP(role, it, ev)                                                                         \
+    do {                                                                                             \
+        if (blockIdx.x == LORDS_TRACE_CTA && (it) < 32) p.trace[((role) * 32 + (it)) * 8 + (ev)] = clock64(); \
+    } while (0)
+#else
+#define USTAMP(role, it, ev) do { } while (0)
+#endif
 
 __device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float v)
 {
@@ -190,35 +207,44 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             tma_prefetch_desc(&p.tm_q);
             tma_prefetch_desc(&p.tm_a);
             tma_prefetch_desc(&p.tm_x);
-            // the first code stages are weights: start them before anything else
-            const int pre = pairs < SQ ? pairs : SQ;
-            for (int pr = 0; pr < pre; ++pr) {
-                const uint32_t bar = bar_q_full + 8 * pr;
-                mbar_expect_tx(bar, (uint32_t)C::QSTAGE);
-                tma_load_2d(q0 + pr * C::QSTAGE, &p.tm_q, (pa + pr) * C::QROW, row0, bar);
-            }
+            // Code stages (weights) are issued as early as their ring slot allows: the first SQ at
+            // once, later ones whenever a slot is seen free (a non-blocking look), and at the latest --
+            // then waiting for the slot -- right before the tiles of the k-steps that need them.
+            int next_q = 0;
+            auto issue_q = [&](bool blocking) -> bool {
+                while (next_q < pairs) {
+                    const int sq = next_q % SQ;
+                    if (next_q >= SQ) {
+                        const uint32_t par = (uint32_t)((next_q / SQ - 1) & 1);
+                        if (blocking) {
+                            if (!mbar_wait(bar_q_empty + 8 * sq, par)) return false;
+                        } else if (!mbar_try_wait(bar_q_empty + 8 * sq, par)) {
+                            return true;
+                        }
+                    }
+                    const uint32_t qbar = bar_q_full + 8 * sq;
+                    mbar_expect_tx(qbar, (uint32_t)C::QSTAGE);
+                    tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (pa + next_q) * C::QROW, row0, qbar);
+                    ++next_q;
+                    if (blocking) return true;     // one stage was due, no more
+                }
+                return true;
+            };
+            issue_q(false);
             // x may be the previous launch's output
             asm volatile("griddepcontrol.wait;" ::: "memory");
             const uint32_t ax_tx = (uint32_t)(p.r_pad * 128 + C::XTILE);
             for (int it = 0; it < total; ++it) {
                 const int sx = it % SX;
+                if (next_q <= (it >> 1) && !issue_q(true)) { failed = true; break; }   // the pair this k-step reads
                 if (it >= SX && !mbar_wait(bar_ax_empty + 8 * sx, (uint32_t)((it / SX - 1) & 1))) { failed = true; break; }
                 const int j0 = (2 * pa + it) * BK;
                 const uint32_t bar = bar_ax_full + 8 * sx;
+                USTAMP(3, it, 0);
                 mbar_expect_tx(bar, ax_tx);
                 tma_load_2d(ax0 + sx * C::AXSTAGE, &p.tm_a, j0, 0, bar);
                 tma_load_2d(ax0 + sx * C::AXSTAGE + kATileBytes, &p.tm_x, j0, tok0, bar);
-                if ((it & 1) == 0 && it >= 2) {
-                    // refill the code stage of the pair whose two k-steps both have their tiles by now
-                    const int pr = it / 2 - 1 + SQ;
-                    if (pr < pairs) {
-                        const int sq = pr % SQ;
-                        if (!mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((pr / SQ - 1) & 1))) { failed = true; break; }
-                        const uint32_t qbar = bar_q_full + 8 * sq;
-                        mbar_expect_tx(qbar, (uint32_t)C::QSTAGE);
-                        tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (pa + pr) * C::QROW, row0, qbar);
-                    }
-                }
+                issue_q(false);
             }
         }
     } else {
@@ -301,10 +327,13 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         for (int j = 0; ok && j < LEAD && j < total; ++j) ok = issue_scale(j);
         for (int it = 0; ok && it < total; ++it) {
             const int sx = it % SX, ws = it % WD;
+            if (lane == 0) USTAMP(0, it, 0);
             if (it + LEAD < total) ok = issue_scale(it + LEAD);
             if (!ok) break;
+            if (lane == 0) USTAMP(0, it, 1);
             if (!mbar_wait(bar_w_full + 8 * ws, (uint32_t)((it / WD) & 1))) { ok = false; break; }
             tc_fence_after_sync();
+            if (lane == 0) USTAMP(0, it, 2);
             if (lane == 0) {
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)(ws * 32);
                 const uint32_t x_lo = ax_lo0 + (uint32_t)((sx * C::AXSTAGE + kATileBytes) >> 4);
@@ -315,6 +344,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 umma_commit(bar_ax_empty + 8 * sx);
                 umma_commit(bar_w_empty + 8 * ws);
                 if (it == total - 1) umma_commit(bar_acc_full);
+                USTAMP(0, it, 3);
             }
             __syncwarp();
         }
@@ -330,8 +360,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 
         for (int it = g; it < total; it += 2) {
             const int sx = it % SX, sd = it % SD, ws = it % WD, pr = it >> 1, sq = pr % SQ;
+            const bool stamper = wg == 0 && lane == 0;
+            if (stamper) USTAMP(1 + g, it, 0);
             if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * sd, (uint32_t)((it / SD) & 1)))) { failed = true; break; }
             tc_fence_after_sync();
+            if (stamper) USTAMP(1 + g, it, 1);
             uint32_t s[32];
             tmem_ld_32x32(lane_addr + C::SCOL + (uint32_t)(sd * 64 + ch * 32), s);
             bool ok = mbar_wait(bar_q_full + 8 * sq, (uint32_t)((pr / SQ) & 1));
@@ -340,6 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s_empty + 8 * sd);      // S is in registers: the buffer may be refilled
             if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+            if (stamper) USTAMP(1 + g, it, 2);
             uint32_t out[16];
             dequant_chunk<BITS>(q0 + sq * C::QSTAGE + row * C::QROW, row, (it & 1) * 2 + ch, lut_lane, s, out);
             if constexpr (C::kConvertInKernel) {
@@ -367,6 +401,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 break;
             }
             tc_fence_after_sync();
+            if (stamper) USTAMP(1 + g, it, 3);
             tmem_st_32x16(lane_addr + kWCol + (uint32_t)(ws * 32 + ch * 16), out);
             tmem_wait_st();
             tc_fence_before_sync();
@@ -375,6 +410,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 mbar_arrive(bar_w_full + 8 * ws);
                 mbar_arrive(bar_q_empty + 8 * sq);
             }
+            if (stamper) USTAMP(1 + g, it, 4);
         }
 
         // ------------------------------------------------------------------ epilogue
@@ -626,6 +662,10 @@ int launch_umma(const Problem &p, State &st, cudaStream_t stream)
     k.npairs = (p.n + 127) / 128;
     k.y = p.y; k.y_f32 = p.y_f32;
     k.status = st.status_word;
+#ifdef LORDS_TRACE
+    k.trace = reinterpret_cast<long long *>(st.workspace + st.workspace_bytes - (size_t)8 * 32 * 8 * 8);
+    LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)8 * 32 * 8 * 8, stream));
+#endif
     const int rc = p.bits == 4 ? launch_bits<4>(k, p, st, stream) : launch_bits<3>(k, p, st, stream);
     if (rc != LORDS_OK) return rc;
     st.last_path = "umma";
