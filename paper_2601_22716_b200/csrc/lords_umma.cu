@@ -4,12 +4,12 @@
 // k-steps.  Per k-step:
 //   1. TMA brings the factor tile A[r x 64] (bf16) and the activation tile x[BN x 64] into a
 //      shared-memory ring; the packed code tile Q[128 x 128 columns] comes once per two k-steps;
-//   2. the issuer thread runs the scale MMA  S = B_tile (128 x r) * A_tile (r x 64)  (Eq. 3; bf16
-//      operands from shared memory, fp32 result in TMEM), a few k-steps ahead of the main MMA;
+//   2. the scale issuer runs  S = B_tile (128 x r) * A_tile (r x 64)  (Eq. 3; bf16 operands from
+//      shared memory, fp32 result in TMEM) as far ahead of the main MMA as the S ring allows;
 //   3. two worker groups of eight warps take the k-steps alternately: a thread reads its 32 columns
 //      of S from TMEM, looks its code pairs up in a lane-private fp16x2 level table, forms
 //      W^ = L[Q] (.) S in fp16 and stores it straight back into TMEM as the A operand;
-//   4. the issuer runs  D[128 x BN] += W^ (TMEM) * x_tile^T (shared memory), fp32 in TMEM.
+//   4. the main issuer runs  D[128 x BN] += W^ (TMEM) * x_tile^T (shared memory), fp32 in TMEM.
 // The activations enter the MMA as fp16: for BN = 16 the workers convert the bf16 tile in place,
 // for larger token tiles a pre-pass converts x once into scratch.
 // Epilogue: D -> registers -> y (bf16 round-to-nearest-even, or fp32).  For BN = 16 the k-range of
@@ -36,9 +36,11 @@ constexpr int BK = 64;                         // in-feature columns per k-step
 constexpr int kRMaxUmma = 64;                  // largest rank this path takes (one swizzle atom of K)
 constexpr int kWorkWarps = 16;                 // two groups of eight
 constexpr int kGroupWarps = 8;
-constexpr int kIssuerWarp = kWorkWarps;        // 16
-constexpr int kTmaWarp = kWorkWarps + 1;       // 17
-constexpr int kThreads = (kWorkWarps + 2) * 32;   // 576
+constexpr int kIssuerWarp = kWorkWarps;        // 16: main MMAs
+constexpr int kScaleWarp = kWorkWarps + 1;     // 17: scale MMAs, as far ahead as the S ring and the tiles allow
+constexpr int kTmaWarp = kWorkWarps + 2;       // 18
+constexpr int kThreads = (kWorkWarps + 3) * 32;   // 608
+constexpr int DR = 8;                          // "main MMA of k-step done" barriers, indexed by k-step mod DR
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kWCol = 384;                // W ring: 4 slots of 32 columns
 constexpr int WD = 4;                          // W ring depth
@@ -57,7 +59,6 @@ template <int BITS, int BN> struct UCfg {
     static constexpr int AXSTAGE = kATileBytes + XTILE;
     static constexpr uint32_t SCOL = BN > 128 ? 256 : 128;       // S ring starts behind the accumulator
     static constexpr int SD = (int)(kWCol - SCOL) / 64;          // S ring depth (2 / 4)
-    static constexpr int LEAD = SD < SX - 1 ? SD : SX - 1;       // k-steps the scale MMA runs ahead of the main MMA
     static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;
     static constexpr int LUT_BYTES = LUT_ENTRIES * 128;
     static constexpr int RED_BYTES = BN == 16 ? kClusterMax * 16 * BM * 4 : 0;
@@ -143,7 +144,8 @@ template <int BITS, int BN>
 __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_constant__ UmmaParams p)
 {
     using C = UCfg<BITS, BN>;
-    constexpr int SX = C::SX, SD = C::SD, LEAD = C::LEAD;
+    constexpr int SX = C::SX, SD = C::SD;
+    static_assert(DR >= SX && DR >= WD && DR % WD == 0 && DR % 2 == 0, "done-barrier ring");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -155,21 +157,20 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
     const uint32_t red0 = lut + C::LUT_BYTES;
     const uint32_t bars = red0 + C::RED_BYTES;
     constexpr int kBarAxFull = 0;                       // SX: TMA bytes of the factor and activation tiles
-    constexpr int kBarAxEmpty = kBarAxFull + SX;        // SX: main MMA of the step done (commit)
-    constexpr int kBarQFull = kBarAxEmpty + SX;         // SQ
+    constexpr int kBarDone = kBarAxFull + SX;           // DR: main MMA of the k-step done (commit): frees its tiles and its W slot
+    constexpr int kBarQFull = kBarDone + DR;            // SQ
     constexpr int kBarQEmpty = kBarQFull + SQ;          // SQ: all 16 worker warps (two steps)
     constexpr int kBarSFull = kBarQEmpty + SQ;          // SD: scale MMA done (commit)
     constexpr int kBarSEmpty = kBarSFull + SD;          // SD: one group has read S
     constexpr int kBarWFull = kBarSEmpty + SD;          // WD: one group has written W^ (and converted x)
-    constexpr int kBarWEmpty = kBarWFull + WD;          // WD: main MMA of the step done (commit)
-    constexpr int kBarAccFull = kBarWEmpty + WD;        // 1
+    constexpr int kBarAccFull = kBarWFull + WD;         // 1
     constexpr int kBarReduce = kBarAccFull + 1;         // 1: the epilogue warps of every CTA of the cluster
     constexpr int kBarCount = kBarReduce + 1;
     static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
-    const uint32_t bar_ax_full = bars + 8 * kBarAxFull, bar_ax_empty = bars + 8 * kBarAxEmpty;
+    const uint32_t bar_ax_full = bars + 8 * kBarAxFull, bar_done = bars + 8 * kBarDone;
     const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
     const uint32_t bar_s_full = bars + 8 * kBarSFull, bar_s_empty = bars + 8 * kBarSEmpty;
-    const uint32_t bar_w_full = bars + 8 * kBarWFull, bar_w_empty = bars + 8 * kBarWEmpty;
+    const uint32_t bar_w_full = bars + 8 * kBarWFull;
     const uint32_t bar_acc_full = bars + 8 * kBarAccFull, bar_reduce = bars + 8 * kBarReduce;
     const uint32_t tmem_slot = bars + 8 * kBarCount;
 
@@ -193,7 +194,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         for (int b = lane; b < kBarCount; b += 32) {
             uint32_t count = 1;
             if (b >= kBarQEmpty && b < kBarSFull) count = kWorkWarps;
-            else if (b >= kBarSEmpty && b < kBarWEmpty) count = kGroupWarps;   // s_empty and w_full
+            else if (b >= kBarSEmpty && b < kBarAccFull) count = kGroupWarps;   // s_empty and w_full
             else if (b == kBarReduce) count = (uint32_t)(4 * csize);
             mbar_init(bars + 8 * b, count);
         }
@@ -237,7 +238,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             for (int it = 0; it < total; ++it) {
                 const int sx = it % SX;
                 if (next_q <= (it >> 1) && !issue_q(true)) { failed = true; break; }   // the pair this k-step reads
-                if (it >= SX && !mbar_wait(bar_ax_empty + 8 * sx, (uint32_t)((it / SX - 1) & 1))) { failed = true; break; }
+                if (it >= SX && !mbar_wait(bar_done + 8 * ((it - SX) % DR), (uint32_t)(((it - SX) / DR) & 1))) { failed = true; break; }
                 const int j0 = (2 * pa + it) * BK;
                 const uint32_t bar = bar_ax_full + 8 * sx;
                 USTAMP(3, it, 0);
@@ -251,7 +252,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         if (warp == kIssuerWarp) {
             tmem_alloc(tmem_slot, kTmemCols);
             tmem_relinquish();
-        } else {
+        } else if (warp < kWorkWarps) {
             // level-pair table: entry e = (L[lo code], L[hi code]) as fp16x2; word e*32 + lane is lane's
             // copy (bank = lane, so the lookups of a warp never conflict)
 #pragma unroll
@@ -293,62 +294,62 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 
     if (warp == kTmaWarp) {
         // all done above
-    } else if (warp == kIssuerWarp) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == kScaleWarp) {
+        // ------------------------------------------------------------------ scale-MMA issuer
+        // S of k-step j goes into S buffer j % SD as soon as the factor tile has landed and the workers
+        // have read the buffer's previous content: it runs ahead of the main MMAs by itself.
         uint32_t tmem_base;
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         constexpr uint32_t idesc_s = umma_idesc_f16(1, 0, 1, BM, 64);     // bf16, B operand MN-major, N = 64
-        constexpr uint32_t idesc_m = umma_idesc_f16(0, 0, 0, BM, BN);     // fp16, K-major
         const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
         const uint32_t lbo_lo = (uint32_t)umma_desc_sw128(0, 1024, 16);
         const uint32_t b_lo = lbo_lo | ((b_tile & 0x3FFFFu) >> 4);
         const uint32_t ax_lo0 = lbo_lo | ((ax0 & 0x3FFFFu) >> 4);
         const int ksteps = p.r_pad / 16;
-        // scale MMA of step j into S buffer j % SD
-        auto issue_scale = [&](int j) -> bool {
+        for (int j = 0; j < total; ++j) {
             const int sx = j % SX, sd = j % SD;
-            if (!mbar_wait(bar_ax_full + 8 * sx, (uint32_t)((j / SX) & 1))) return false;
-            if (j >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((j / SD - 1) & 1))) return false;
+            if (lane == 0) USTAMP(4, j, 0);
+            if (!mbar_wait(bar_ax_full + 8 * sx, (uint32_t)((j / SX) & 1))) { failed = true; break; }
+            if (j >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((j / SD - 1) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
+                USTAMP(4, j, 1);
                 const uint32_t a_lo = ax_lo0 + (uint32_t)(sx * (C::AXSTAGE >> 4));
                 for (int k = 0; k < ksteps; ++k)
                     umma_f16_ss(tmem_base + C::SCOL + sd * 64, umma_desc_pack(b_lo + k * 2, desc_hi),
                                 umma_desc_pack(a_lo + k * 128, desc_hi), idesc_s, k > 0);
                 umma_commit(bar_s_full + 8 * sd);
+                USTAMP(4, j, 2);
             }
             __syncwarp();
-            return true;
-        };
-        // The scale MMA of step it + LEAD is queued ahead of the main MMA of step it.  LEAD <= SD
-        // (its S buffer is free once the workers have read step it + LEAD - SD) and LEAD < SX (its
-        // factor tile needs the ring stage of step it + LEAD - SX, whose main MMA is already queued).
-        bool ok = true;
-        for (int j = 0; ok && j < LEAD && j < total; ++j) ok = issue_scale(j);
-        for (int it = 0; ok && it < total; ++it) {
+        }
+    } else if (warp == kIssuerWarp) {
+        // ------------------------------------------------------------------ main-MMA issuer
+        uint32_t tmem_base;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+        constexpr uint32_t idesc_m = umma_idesc_f16(0, 0, 0, BM, BN);     // fp16, K-major
+        const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
+        const uint32_t ax_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((ax0 & 0x3FFFFu) >> 4);
+        for (int it = 0; it < total; ++it) {
             const int sx = it % SX, ws = it % WD;
             if (lane == 0) USTAMP(0, it, 0);
-            if (it + LEAD < total) ok = issue_scale(it + LEAD);
-            if (!ok) break;
-            if (lane == 0) USTAMP(0, it, 1);
-            if (!mbar_wait(bar_w_full + 8 * ws, (uint32_t)((it / WD) & 1))) { ok = false; break; }
+            // W^ of the k-step is in TMEM; that implies its scale MMA ran, hence its tiles had landed
+            if (!mbar_wait(bar_w_full + 8 * ws, (uint32_t)((it / WD) & 1))) { failed = true; break; }
             tc_fence_after_sync();
-            if (lane == 0) USTAMP(0, it, 2);
             if (lane == 0) {
+                USTAMP(0, it, 2);
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)(ws * 32);
                 const uint32_t x_lo = ax_lo0 + (uint32_t)((sx * C::AXSTAGE + kATileBytes) >> 4);
 #pragma unroll
                 for (int k = 0; k < BK / 16; ++k)
                     umma_f16_ts(tmem_base, wslot + k * 8, umma_desc_pack(x_lo + k * 2, desc_hi), idesc_m,
                                 (it > 0 || k > 0) ? 1u : 0u);
-                umma_commit(bar_ax_empty + 8 * sx);
-                umma_commit(bar_w_empty + 8 * ws);
+                umma_commit(bar_done + 8 * (it % DR));
                 if (it == total - 1) umma_commit(bar_acc_full);
                 USTAMP(0, it, 3);
             }
             __syncwarp();
         }
-        failed = !ok;
     } else {
         // ------------------------------------------------------------------ worker warps
         const int g = warp / kGroupWarps, wg = warp % kGroupWarps, q = warp & 3, ch = wg >> 2;
@@ -396,7 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 }
                 fence_proxy_async_smem();
             }
-            if (it >= WD && !__all_sync(0xffffffffu, mbar_wait(bar_w_empty + 8 * ws, (uint32_t)((it / WD - 1) & 1)))) {
+            if (it >= WD && !__all_sync(0xffffffffu, mbar_wait(bar_done + 8 * ((it - WD) % DR), (uint32_t)(((it - WD) / DR) & 1)))) {
                 failed = true;
                 break;
             }
