@@ -2,8 +2,9 @@
 //
 // One CTA owns a 128-row tile of W^ (out-features), a tile of BN tokens and a range of 64-column
 // k-steps.  Per k-step:
-//   1. TMA brings the factor tile A[r x 64] (bf16) and the activation tile x[BN x 64] into a
-//      shared-memory ring; the packed code tile Q[128 x 128 columns] comes once per two k-steps;
+//   1. TMA brings the factor tile A[r x 64] (bf16) and the activation tile x[BN x 64] into two
+//      shared-memory rings of their own (the small factor tiles run ahead of the large activation
+//      tiles); the packed code tile Q[128 x 128 columns] comes once per two k-steps;
 //   2. the scale issuer runs  S = B_tile (128 x r) * A_tile (r x 64)  (Eq. 3; bf16 operands from
 //      shared memory, fp32 result in TMEM) as far ahead of the main MMA as the S ring allows;
 //   3. two worker groups of eight warps take the k-steps alternately: a thread reads its 32 columns
@@ -38,8 +39,10 @@ constexpr int kWorkWarps = 16;                 // two groups of eight
 constexpr int kGroupWarps = 8;
 constexpr int kIssuerWarp = kWorkWarps;        // 16: main MMAs
 constexpr int kScaleWarp = kWorkWarps + 1;     // 17: scale MMAs, as far ahead as the S ring and the tiles allow
-constexpr int kTmaWarp = kWorkWarps + 2;       // 18
-constexpr int kThreads = (kWorkWarps + 3) * 32;   // 608
+constexpr int kTmaWarp = kWorkWarps + 2;       // 18: activation tiles and code stages
+constexpr int kTmaAWarp = kWorkWarps + 3;      // 19: factor tiles
+constexpr int kThreads = (kWorkWarps + 4) * 32;   // 640
+constexpr int SA = 4;                          // factor-tile ring depth
 constexpr int DR = 8;                          // "main MMA of k-step done" barriers, indexed by k-step mod DR
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kWCol = 384;                // W ring: 4 slots of 32 columns
@@ -52,18 +55,18 @@ constexpr int kClusterMax = 8;                 // largest k-split (cluster size)
 template <int BITS, int BN> struct UCfg {
     static constexpr int QROW = 128 * BITS / 8;                  // packed bytes per row per code stage (64 / 48)
     static constexpr int QSTAGE = BM * QROW;
-    // factor / activation ring depth: as deep as shared memory allows, the tiles come from L2 with a
-    // latency of several k-steps
-    static constexpr int SX = BN >= 256 ? 3 : BN >= 128 ? 5 : 8;
+    // activation ring depth: as deep as shared memory allows, the tiles come from L2 with a latency of
+    // several k-steps.  The factor tiles have a ring of their own, so that the scale MMA and the
+    // workers run ahead of the (much larger) activation tiles.
+    static constexpr int SX = BN >= 256 ? 3 : BN >= 128 ? 6 : 8;
     static constexpr int XTILE = BN * 128;
-    static constexpr int AXSTAGE = kATileBytes + XTILE;
     static constexpr uint32_t SCOL = BN > 128 ? 256 : 128;       // S ring starts behind the accumulator
     static constexpr int SD = (int)(kWCol - SCOL) / 64;          // S ring depth (2 / 4)
     static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;
     static constexpr int LUT_BYTES = LUT_ENTRIES * 128;
     static constexpr int RED_BYTES = BN == 16 ? kClusterMax * 16 * BM * 4 : 0;
     static constexpr int BAR_BYTES = 512;
-    static constexpr int SMEM = 1024 + SX * AXSTAGE + SQ * QSTAGE + kBTileBytes + LUT_BYTES + RED_BYTES + BAR_BYTES;
+    static constexpr int SMEM = 1024 + SX * XTILE + SA * kATileBytes + SQ * QSTAGE + kBTileBytes + LUT_BYTES + RED_BYTES + BAR_BYTES;
     static constexpr bool kConvertInKernel = BN == 16;           // x tile arrives as bf16 and is converted in place
 };
 
@@ -150,14 +153,17 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     // carve-up (tile bases are multiples of 1024 bytes)
-    const uint32_t ax0 = base;                                  // SX x { A tile 8 KB | x tile }
-    const uint32_t q0 = ax0 + SX * C::AXSTAGE;                  // SQ code stages
+    const uint32_t x0 = base;                                   // SX activation tiles
+    const uint32_t a0 = x0 + SX * C::XTILE;                     // SA factor tiles
+    const uint32_t q0 = a0 + SA * kATileBytes;                  // SQ code stages
     const uint32_t b_tile = q0 + SQ * C::QSTAGE;                // B[128 x 64 ranks] bf16, K-major, swizzled
     const uint32_t lut = b_tile + kBTileBytes;
     const uint32_t red0 = lut + C::LUT_BYTES;
     const uint32_t bars = red0 + C::RED_BYTES;
-    constexpr int kBarAxFull = 0;                       // SX: TMA bytes of the factor and activation tiles
-    constexpr int kBarDone = kBarAxFull + SX;           // DR: main MMA of the k-step done (commit): frees its tiles and its W slot
+    constexpr int kBarXFull = 0;                        // SX: TMA bytes of the activation tile
+    constexpr int kBarAFull = kBarXFull + SX;           // SA: TMA bytes of the factor tile
+    constexpr int kBarADone = kBarAFull + SA;           // SA: scale MMA of the k-step done (commit): frees the factor tile
+    constexpr int kBarDone = kBarADone + SA;            // DR: main MMA of the k-step done (commit): frees its x tile and its W slot
     constexpr int kBarQFull = kBarDone + DR;            // SQ
     constexpr int kBarQEmpty = kBarQFull + SQ;          // SQ: all 16 worker warps (two steps)
     constexpr int kBarSFull = kBarQEmpty + SQ;          // SD: scale MMA done (commit)
@@ -167,7 +173,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
     constexpr int kBarReduce = kBarAccFull + 1;         // 1: the epilogue warps of every CTA of the cluster
     constexpr int kBarCount = kBarReduce + 1;
     static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
-    const uint32_t bar_ax_full = bars + 8 * kBarAxFull, bar_done = bars + 8 * kBarDone;
+    const uint32_t bar_x_full = bars + 8 * kBarXFull, bar_done = bars + 8 * kBarDone;
+    const uint32_t bar_a_full = bars + 8 * kBarAFull, bar_a_done = bars + 8 * kBarADone;
     const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
     const uint32_t bar_s_full = bars + 8 * kBarSFull, bar_s_empty = bars + 8 * kBarSEmpty;
     const uint32_t bar_w_full = bars + 8 * kBarWFull;
@@ -206,7 +213,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
         if (lane == 0) {
             tma_prefetch_desc(&p.tm_q);
-            tma_prefetch_desc(&p.tm_a);
             tma_prefetch_desc(&p.tm_x);
             // Code stages (weights) are issued as early as their ring slot allows: the first SQ at
             // once, later ones whenever a slot is seen free (a non-blocking look), and at the latest --
@@ -234,17 +240,14 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             issue_q(false);
             // x may be the previous launch's output
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            const uint32_t ax_tx = (uint32_t)(p.r_pad * 128 + C::XTILE);
             for (int it = 0; it < total; ++it) {
                 const int sx = it % SX;
                 if (next_q <= (it >> 1) && !issue_q(true)) { failed = true; break; }   // the pair this k-step reads
                 if (it >= SX && !mbar_wait(bar_done + 8 * ((it - SX) % DR), (uint32_t)(((it - SX) / DR) & 1))) { failed = true; break; }
-                const int j0 = (2 * pa + it) * BK;
-                const uint32_t bar = bar_ax_full + 8 * sx;
+                const uint32_t bar = bar_x_full + 8 * sx;
                 USTAMP(3, it, 0);
-                mbar_expect_tx(bar, ax_tx);
-                tma_load_2d(ax0 + sx * C::AXSTAGE, &p.tm_a, j0, 0, bar);
-                tma_load_2d(ax0 + sx * C::AXSTAGE + kATileBytes, &p.tm_x, j0, tok0, bar);
+                mbar_expect_tx(bar, (uint32_t)C::XTILE);
+                tma_load_2d(x0 + sx * C::XTILE, &p.tm_x, (2 * pa + it) * BK, tok0, bar);
                 issue_q(false);
             }
         }
@@ -294,6 +297,19 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 
     if (warp == kTmaWarp) {
         // all done above
+    } else if (warp == kTmaAWarp) {
+        // ------------------------------------------------------------------ factor tiles (weights)
+        if (lane == 0) {
+            tma_prefetch_desc(&p.tm_a);
+            const uint32_t tx = (uint32_t)(p.r_pad * 128);
+            for (int j = 0; j < total; ++j) {
+                const int sa = j % SA;
+                if (j >= SA && !mbar_wait(bar_a_done + 8 * sa, (uint32_t)((j / SA - 1) & 1))) { failed = true; break; }
+                const uint32_t bar = bar_a_full + 8 * sa;
+                mbar_expect_tx(bar, tx);
+                tma_load_2d(a0 + sa * kATileBytes, &p.tm_a, (2 * pa + j) * BK, 0, bar);
+            }
+        }
     } else if (warp == kScaleWarp) {
         // ------------------------------------------------------------------ scale-MMA issuer
         // S of k-step j goes into S buffer j % SD as soon as the factor tile has landed and the workers
@@ -304,21 +320,22 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
         const uint32_t lbo_lo = (uint32_t)umma_desc_sw128(0, 1024, 16);
         const uint32_t b_lo = lbo_lo | ((b_tile & 0x3FFFFu) >> 4);
-        const uint32_t ax_lo0 = lbo_lo | ((ax0 & 0x3FFFFu) >> 4);
+        const uint32_t a_lo0 = lbo_lo | ((a0 & 0x3FFFFu) >> 4);
         const int ksteps = p.r_pad / 16;
         for (int j = 0; j < total; ++j) {
-            const int sx = j % SX, sd = j % SD;
+            const int sa = j % SA, sd = j % SD;
             if (lane == 0) USTAMP(4, j, 0);
-            if (!mbar_wait(bar_ax_full + 8 * sx, (uint32_t)((j / SX) & 1))) { failed = true; break; }
+            if (!mbar_wait(bar_a_full + 8 * sa, (uint32_t)((j / SA) & 1))) { failed = true; break; }
             if (j >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((j / SD - 1) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
                 USTAMP(4, j, 1);
-                const uint32_t a_lo = ax_lo0 + (uint32_t)(sx * (C::AXSTAGE >> 4));
+                const uint32_t a_lo = a_lo0 + (uint32_t)(sa * (kATileBytes >> 4));
                 for (int k = 0; k < ksteps; ++k)
                     umma_f16_ss(tmem_base + C::SCOL + sd * 64, umma_desc_pack(b_lo + k * 2, desc_hi),
                                 umma_desc_pack(a_lo + k * 128, desc_hi), idesc_s, k > 0);
                 umma_commit(bar_s_full + 8 * sd);
+                umma_commit(bar_a_done + 8 * sa);
                 USTAMP(4, j, 2);
             }
             __syncwarp();
@@ -329,17 +346,18 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         constexpr uint32_t idesc_m = umma_idesc_f16(0, 0, 0, BM, BN);     // fp16, K-major
         const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
-        const uint32_t ax_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((ax0 & 0x3FFFFu) >> 4);
+        const uint32_t x_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((x0 & 0x3FFFFu) >> 4);
         for (int it = 0; it < total; ++it) {
             const int sx = it % SX, ws = it % WD;
             if (lane == 0) USTAMP(0, it, 0);
-            // W^ of the k-step is in TMEM; that implies its scale MMA ran, hence its tiles had landed
+            // W^ of the k-step is in TMEM and its activation tile has landed
             if (!mbar_wait(bar_w_full + 8 * ws, (uint32_t)((it / WD) & 1))) { failed = true; break; }
+            if (!mbar_wait(bar_x_full + 8 * sx, (uint32_t)((it / SX) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
                 USTAMP(0, it, 2);
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)(ws * 32);
-                const uint32_t x_lo = ax_lo0 + (uint32_t)((sx * C::AXSTAGE + kATileBytes) >> 4);
+                const uint32_t x_lo = x_lo0 + (uint32_t)((sx * C::XTILE) >> 4);
 #pragma unroll
                 for (int k = 0; k < BK / 16; ++k)
                     umma_f16_ts(tmem_base, wslot + k * 8, umma_desc_pack(x_lo + k * 2, desc_hi), idesc_m,
@@ -378,13 +396,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             uint32_t out[16];
             dequant_chunk<BITS>(q0 + sq * C::QSTAGE + row * C::QROW, row, (it & 1) * 2 + ch, lut_lane, s, out);
             if constexpr (C::kConvertInKernel) {
-                // The activation tile arrived as bf16 (16 tokens x 64 columns, together with the factor
-                // tile the scale MMA has already consumed): convert it in place, one 16-byte chunk per
+                // The activation tile arrived as bf16 (16 tokens x 64 columns): convert it in place, one 16-byte chunk per
                 // thread of the first four warps of the group (element-wise, so the swizzled position
                 // of the chunk does not matter).
-                if (!__all_sync(0xffffffffu, mbar_wait(bar_ax_full + 8 * sx, (uint32_t)((it / SX) & 1)))) { failed = true; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_x_full + 8 * sx, (uint32_t)((it / SX) & 1)))) { failed = true; break; }
                 if (wg < 4) {
-                    const uint32_t addr = ax0 + sx * C::AXSTAGE + kATileBytes + (uint32_t)((wg * 32 + lane) * 16);
+                    const uint32_t addr = x0 + sx * C::XTILE + (uint32_t)((wg * 32 + lane) * 16);
                     const uint4 v = lds_v4(addr);
                     const uint32_t in[4] = {v.x, v.y, v.z, v.w};
                     uint32_t o[4];
