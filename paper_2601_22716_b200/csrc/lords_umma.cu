@@ -48,17 +48,18 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kWCol = 384;                // W ring: 4 slots of 32 columns
 constexpr int WD = 4;                          // W ring depth
 constexpr int SQ = 4;                          // code-tile ring depth (128 columns per stage)
-constexpr int kATileBytes = kRMaxUmma * 128;
 constexpr int kBTileBytes = BM * 128;
 constexpr int kClusterMax = 8;                 // largest k-split (cluster size) of the BN = 16 kernel
 
-template <int BITS, int BN> struct UCfg {
+// BITS: code width.  BN: token tile.  RP: padded rank the factor-tile slots are sized for (32 or 64).
+template <int BITS, int BN, int RP> struct UCfg {
     static constexpr int QROW = 128 * BITS / 8;                  // packed bytes per row per code stage (64 / 48)
     static constexpr int QSTAGE = BM * QROW;
     // activation ring depth: as deep as shared memory allows, the tiles come from L2 with a latency of
     // several k-steps.  The factor tiles have a ring of their own, so that the scale MMA and the
     // workers run ahead of the (much larger) activation tiles.
-    static constexpr int SX = BN >= 256 ? 3 : BN >= 128 ? 6 : 8;
+    static constexpr int ATILE = RP * 128;
+    static constexpr int SX = BN >= 256 ? (RP <= 32 ? 4 : 3) : BN >= 128 ? 6 : 8;
     static constexpr int XTILE = BN * 128;
     static constexpr uint32_t SCOL = BN > 128 ? 256 : 128;       // S ring starts behind the accumulator
     static constexpr int SD = (int)(kWCol - SCOL) / 64;          // S ring depth (2 / 4)
@@ -66,7 +67,7 @@ template <int BITS, int BN> struct UCfg {
     static constexpr int LUT_BYTES = LUT_ENTRIES * 128;
     static constexpr int RED_BYTES = BN == 16 ? kClusterMax * 16 * BM * 4 : 0;
     static constexpr int BAR_BYTES = 512;
-    static constexpr int SMEM = 1024 + SX * XTILE + SA * kATileBytes + SQ * QSTAGE + kBTileBytes + LUT_BYTES + RED_BYTES + BAR_BYTES;
+    static constexpr int SMEM = 1024 + SX * XTILE + SA * ATILE + SQ * QSTAGE + kBTileBytes + LUT_BYTES + RED_BYTES + BAR_BYTES;
     static constexpr bool kConvertInKernel = BN == 16;           // x tile arrives as bf16 and is converted in place
 };
 
@@ -143,11 +144,11 @@ __device__ __forceinline__ void dequant_chunk(uint32_t qrow, int row, int c, uin
     }
 }
 
-template <int BITS, int BN>
+template <int BITS, int BN, int RP>
 __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_constant__ UmmaParams p)
 {
-    using C = UCfg<BITS, BN>;
-    constexpr int SX = C::SX, SD = C::SD;
+    using C = UCfg<BITS, BN, RP>;
+    constexpr int SX = C::SX, SD = C::SD, kATileBytes = C::ATILE;
     static_assert(DR >= SX && DR >= WD && DR % WD == 0 && DR % 2 == 0, "done-barrier ring");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -549,13 +550,13 @@ bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BITS, int BN> struct UmmaVariant {
+template <int BITS, int BN, int RP> struct UmmaVariant {
     static int prepare()
     {
         static bool done = false;
         if (!done) {
-            LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_umma_kernel<BITS, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                UCfg<BITS, BN>::SMEM));
+            LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_umma_kernel<BITS, BN, RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                UCfg<BITS, BN, RP>::SMEM));
             done = true;
         }
         return LORDS_OK;
@@ -572,7 +573,7 @@ template <int BITS, int BN> struct UmmaVariant {
         cfg = cudaLaunchConfig_t{};
         cfg.gridDim = dim3((unsigned)(clusters * cs));
         cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = UCfg<BITS, BN>::SMEM;
+        cfg.dynamicSmemBytes = UCfg<BITS, BN, RP>::SMEM;
         cfg.stream = stream;
         cfg.attrs = attr;
         cfg.numAttrs = 2;
@@ -586,7 +587,7 @@ template <int BITS, int BN> struct UmmaVariant {
             cudaLaunchAttribute attr[2];
             fill(cfg, attr, cs, 1, nullptr);
             int n = 0;
-            const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_umma_kernel<BITS, BN>, &cfg);
+            const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_umma_kernel<BITS, BN, RP>, &cfg);
             if (e != cudaSuccess) (void)cudaGetLastError();
             cache[cs] = (e == cudaSuccess && n >= 1) ? n : -1;
         }
@@ -597,14 +598,14 @@ template <int BITS, int BN> struct UmmaVariant {
         cudaLaunchConfig_t cfg;
         cudaLaunchAttribute attr[2];
         fill(cfg, attr, cs, tiles, stream);
-        LORDS_CUDA_TRY(cudaLaunchKernelEx(&cfg, lords_umma_kernel<BITS, BN>, k));
+        LORDS_CUDA_TRY(cudaLaunchKernelEx(&cfg, lords_umma_kernel<BITS, BN, RP>, k));
         return LORDS_OK;
     }
 };
 
-template <int BITS, int BN> int launch_variant(UmmaParams &k, const Problem &p, State &st, cudaStream_t stream)
+template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Problem &p, State &st, cudaStream_t stream)
 {
-    using V = UmmaVariant<BITS, BN>;
+    using V = UmmaVariant<BITS, BN, RP>;
     int rc = V::prepare();
     if (rc != LORDS_OK) return rc;
     k.tok_tiles = (p.M + BN - 1) / BN;
@@ -624,7 +625,7 @@ template <int BITS, int BN> int launch_variant(UmmaParams &k, const Problem &p, 
     }
 
     const void *xsrc = p.x;
-    if (!UCfg<BITS, BN>::kConvertInKernel) {
+    if (!UCfg<BITS, BN, RP>::kConvertInKernel) {
         const size_t x16_bytes = (size_t)p.M * p.n * 2;
         if (x16_bytes > st.workspace_bytes) return LORDS_ERR_WORKSPACE;
         const size_t n_vec = (size_t)p.M * p.n / 8;
@@ -634,33 +635,38 @@ template <int BITS, int BN> int launch_variant(UmmaParams &k, const Problem &p, 
         xsrc = st.workspace;
     }
     const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
-    if (!make_map_2d(&k.tm_x, UCfg<BITS, BN>::kConvertInKernel ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16,
+    if (!make_map_2d(&k.tm_x, UCfg<BITS, BN, RP>::kConvertInKernel ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16,
                      2, xsrc, (uint64_t)p.n, (uint64_t)p.M, 64, (uint32_t)BN, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.A, (uint64_t)p.n, (uint64_t)p.r, 64, (uint32_t)k.r_pad,
                      CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)UCfg<BITS, BN>::QROW, BM,
+        !make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)UCfg<BITS, BN, RP>::QROW, BM,
                      BITS == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE))
         return LORDS_ERR_CUDA;
     rc = V::launch(k, (int)tiles, cs, stream);
     if (rc != LORDS_OK) return rc;
-    st.last_launches = UCfg<BITS, BN>::kConvertInKernel ? 1 : 2;
+    st.last_launches = UCfg<BITS, BN, RP>::kConvertInKernel ? 1 : 2;
     return LORDS_OK;
 }
 
-template <int BITS> int launch_bits(UmmaParams &k, const Problem &p, State &st, cudaStream_t stream)
+template <int BITS, int RP> int launch_bits_rank(UmmaParams &k, const Problem &p, State &st, cudaStream_t stream)
 {
-    if (p.M <= 16) return launch_variant<BITS, 16>(k, p, st, stream);
+    if (p.M <= 16) return launch_variant<BITS, 16, RP>(k, p, st, stream);
     // token tile: the largest that still gives CTAs for most of the SMs
     const long long row_tiles = (p.m + BM - 1) / BM;
     int bn = 256;
     while (bn > 32 && (p.M <= bn / 2 || 5 * row_tiles * ((p.M + bn - 1) / bn) < 3 * (long long)st.sm_count)) bn /= 2;
     if (st.forced_bn > 0) bn = st.forced_bn;   // measurement switch
     switch (bn) {
-        case 32: return launch_variant<BITS, 32>(k, p, st, stream);
-        case 64: return launch_variant<BITS, 64>(k, p, st, stream);
-        case 128: return launch_variant<BITS, 128>(k, p, st, stream);
-        default: return launch_variant<BITS, 256>(k, p, st, stream);
+        case 32: return launch_variant<BITS, 32, RP>(k, p, st, stream);
+        case 64: return launch_variant<BITS, 64, RP>(k, p, st, stream);
+        case 128: return launch_variant<BITS, 128, RP>(k, p, st, stream);
+        default: return launch_variant<BITS, 256, RP>(k, p, st, stream);
     }
+}
+
+template <int BITS> int launch_bits(UmmaParams &k, const Problem &p, State &st, cudaStream_t stream)
+{
+    return k.r_pad <= 32 ? launch_bits_rank<BITS, 32>(k, p, st, stream) : launch_bits_rank<BITS, 64>(k, p, st, stream);
 }
 
 }  // namespace
