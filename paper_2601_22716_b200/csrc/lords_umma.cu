@@ -80,6 +80,9 @@ struct alignas(64) UmmaParams {
     int M, m, n, r, r_pad;
     int npairs;           // 128-column pairs of k-steps per tile
     int tok_tiles;
+    int whole_pairs;      // pair mode (BN > 16, clusters of 2): clusters below this index run two whole tiles,
+                          // the others share one tile, half of its k-range each; -1 = no pair mode
+    float *pair_scratch;  // pair mode: [shared tile][BN][128] partial sums of the second half
     void *y;
     int y_f32;
     int *status;
@@ -186,10 +189,23 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 
     // work assignment: cluster = one (row tile, token tile); rank = slice of its k-range
     const int csize = (int)cluster_nctarank(), rank = (int)cluster_ctarank();
-    const int tile = (int)blockIdx.x / csize;
+    int tile = (int)blockIdx.x / csize, ksplit = csize, kslice = rank;
+    bool pair_split = false;       // this CTA shares its tile with its cluster partner (pair mode)
+    int pair_index = 0;
+    if (BN > 16 && p.whole_pairs >= 0) {
+        // Pair mode fills the idle slots of the last wave: clusters of two CTAs; the first `whole_pairs`
+        // clusters run two whole tiles (one per CTA), the remaining clusters split one tile's k-range.
+        const int c = (int)blockIdx.x >> 1;
+        if (c < p.whole_pairs) {
+            tile = 2 * c + rank; ksplit = 1; kslice = 0;
+        } else {
+            pair_index = c - p.whole_pairs;
+            tile = 2 * p.whole_pairs + pair_index; ksplit = 2; kslice = rank; pair_split = true;
+        }
+    }
     const int row_tile = tile / p.tok_tiles, tok_tile = tile - row_tile * p.tok_tiles;
     const int row0 = row_tile * BM, tok0 = tok_tile * BN;
-    const int pa = (int)((long long)rank * p.npairs / csize), pb = (int)((long long)(rank + 1) * p.npairs / csize);
+    const int pa = (int)((long long)kslice * p.npairs / ksplit), pb = (int)((long long)(kslice + 1) * p.npairs / ksplit);
     const int pairs = pb - pa;
     const int total = 2 * pairs;          // k-steps of this CTA; global k-step = 2 * pa + it
 
@@ -203,7 +219,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             uint32_t count = 1;
             if (b >= kBarQEmpty && b < kBarSFull) count = kWorkWarps;
             else if (b >= kBarSEmpty && b < kBarAccFull) count = kGroupWarps;   // s_empty and w_full
-            else if (b == kBarReduce) count = (uint32_t)(4 * csize);
+            else if (b == kBarReduce) count = BN == 16 ? (uint32_t)(4 * csize) : (uint32_t)(4 * (BN / (BN >= 64 ? BN / 4 : 16)));
             mbar_init(bars + 8 * b, count);
         }
         fence_mbar_init();
@@ -442,20 +458,38 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             const int i = row0 + row;
             if (!ok) failed = true;
             if (BN > 16 || csize == 1) {
+                float *const part = p.pair_scratch + (size_t)pair_index * BN * BM;
+                if (pair_split && rank == 0) {
+                    // the partner's half of the k-range comes through global scratch; its arrival on
+                    // this CTA's barrier (release / acquire at cluster scope) orders the data
+                    if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0))) { ok = false; failed = true; }
+                }
                 if (ok && total > 0) {
 #pragma unroll 1
                     for (int c0 = cg * CPG; c0 < (cg + 1) * CPG; c0 += 16) {
                         uint32_t v[16];
                         tmem_ld_32x16(lane_addr + (uint32_t)c0, v);
                         tmem_wait_ld();
-                        if (i < p.m) {
+                        if (pair_split && rank == 1) {
+#pragma unroll
+                            for (int c = 0; c < 16; ++c) part[(size_t)(c0 + c) * BM + row] = __uint_as_float(v[c]);
+                        } else if (i < p.m) {
 #pragma unroll
                             for (int c = 0; c < 16; ++c) {
                                 const int t = tok0 + c0 + c;
-                                if (t < p.M) store_out(p.y, p.y_f32, (size_t)t * p.m + i, __uint_as_float(v[c]));
+                                if (t < p.M) {
+                                    float a = __uint_as_float(v[c]);
+                                    if (pair_split) a += __ldcg(part + (size_t)(c0 + c) * BM + row);   // fixed order: first half + second half
+                                    store_out(p.y, p.y_f32, (size_t)t * p.m + i, a);
+                                }
                             }
                         }
                     }
+                }
+                if (pair_split && rank == 1) {
+                    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // the partner's barrier exists
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_rank(bar_reduce, 0));
                 }
             } else {
                 // BN == 16 with the k-range split over the cluster: park the partials in the leader's
@@ -624,10 +658,33 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
             if (V::max_clusters(c) >= (forced ? 1 : tiles)) { cs = c; break; }
     }
 
+    // Pair mode (BN > 16): when the tiles need more than one wave of CTAs, idle slots of the last wave
+    // are filled by splitting that many tiles' k-range over the two CTAs of a cluster.
+    k.whole_pairs = -1;
+    k.pair_scratch = nullptr;
+    int clusters = (int)tiles;
+    size_t pair_bytes = 0;
+    if (BN > 16 && k.npairs >= 2) {
+        const long long resident = 2LL * V::max_clusters(2);
+        if (resident > 0 && tiles > resident) {
+            const long long waves = (tiles + resident - 1) / resident;
+            long long split = waves * resident - tiles;
+            if (split > tiles) split = tiles;
+            if ((tiles - split) & 1) --split;
+            if (split > 0) {
+                k.whole_pairs = (int)((tiles - split) / 2);
+                clusters = k.whole_pairs + (int)split;
+                cs = 2;
+                pair_bytes = (size_t)split * BN * BM * sizeof(float);
+            }
+        }
+    }
+
     const void *xsrc = p.x;
     if (!UCfg<BITS, BN, RP>::kConvertInKernel) {
-        const size_t x16_bytes = (size_t)p.M * p.n * 2;
-        if (x16_bytes > st.workspace_bytes) return LORDS_ERR_WORKSPACE;
+        const size_t x16_bytes = ((size_t)p.M * p.n * 2 + 255) & ~(size_t)255;
+        if (x16_bytes + pair_bytes > st.workspace_bytes) return LORDS_ERR_WORKSPACE;
+        k.pair_scratch = reinterpret_cast<float *>(st.workspace + x16_bytes);
         const size_t n_vec = (size_t)p.M * p.n / 8;
         lords_x_to_f16_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, stream>>>(
             reinterpret_cast<const uint4 *>(p.x), reinterpret_cast<uint4 *>(st.workspace), n_vec);
@@ -642,7 +699,7 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
         !make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)UCfg<BITS, BN, RP>::QROW, BM,
                      BITS == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE))
         return LORDS_ERR_CUDA;
-    rc = V::launch(k, (int)tiles, cs, stream);
+    rc = V::launch(k, clusters, cs, stream);
     if (rc != LORDS_OK) return rc;
     st.last_launches = UCfg<BITS, BN, RP>::kConvertInKernel ? 1 : 2;
     return LORDS_OK;

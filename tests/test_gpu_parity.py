@@ -172,6 +172,8 @@ UMMA_SHAPES = [
     (4, 300, 1536, 16, 100, 128, True),
     (3, 384, 1280, 48, 300, 256, False),
     (4, 256, 1024, 8, 257, 256, True),   # a second token tile with one token in it
+    (4, 1024, 512, 16, 600, 32, False),  # more tiles than resident CTAs: the last wave is filled with split tiles
+    (3, 1100, 512, 32, 620, 32, True),
 ]
 
 
@@ -188,7 +190,7 @@ def test_umma_kernel_shapes(lords, bits, m, n, r, M, bn, mixed):
 
 
 @pytest.mark.parametrize("bits,m,n,r,M,bn", [(4, 256, 512, 32, 16, 0), (3, 131, 384, 7, 9, 0), (4, 140, 256, 16, 33, 32),
-                                             (3, 256, 512, 48, 200, 256)])
+                                             (3, 256, 512, 48, 200, 256), (4, 1280, 256, 8, 500, 32)])
 def test_umma_kernel_integer_case_is_bit_exact(lords, bits, m, n, r, M, bn):
     lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m + M)
     lords.lords_set_option("bn", str(bn))
