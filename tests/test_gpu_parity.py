@@ -255,6 +255,23 @@ def test_config3_prefill_full_size_sampled(lords, path):
     assert np.isfinite(y32).all()
 
 
+# ---- the remaining Llama-3-8B module shapes of the full linear stack (k/v with r = 16, o, gate/up at
+# ---- 4 bits, M in {1, 8, 512}), full size, outputs sampled by row
+
+@pytest.mark.parametrize("name,r,bits,M", [("k", 16, 4, 1), ("v", 16, 4, 8), ("o", 32, 4, 8), ("gate", 32, 4, 1),
+                                            ("up", 32, 4, 8), ("down", 32, 4, 1), ("q", 32, 4, 512),
+                                            ("down", 48, 3, 512), ("k", 16, 4, 512)])
+def test_config4_stack_shapes_full_size_sampled(lords, name, r, bits, M):
+    m, n = gen.LLAMA3_8B_SHAPES[name]
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=7 * len(name) + M)
+    dl, y32, ybf = _run(lords, lay, "auto")
+    assert lords.lords_last_path() in ("decode", "umma")
+    rows = _sampled_rows(m, 256 if M <= 8 else 64, 11)
+    y64 = _oracle(lay, dl.packed_host, rows=rows)
+    check_against_oracle(y32[:, rows], ybf[:, rows], y64)
+    assert np.isfinite(y32).all()
+
+
 def test_host_buffer_entry_point_matches_device_entry(lords):
     import torch
     lay = gen.make_layer(512, 1024, 16, 4, bits=4, seed=12)
