@@ -273,6 +273,74 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
     return res
 
 
+STACK_LAYERS = ["q", "k", "v", "o", "gate", "up", "down"]
+
+
+def time_stack(M, mlp_bits, steps, device):
+    """Full Llama-3-8B linear stack: 32 layers x {q, k, v, o, gate, up, down}, one forward call per
+    module (224 calls) from one CUDA graph.  Attention modules are NF4 (r = 32; r = 16 for k/v); the
+    MLP modules are NF4 r = 32 or NF3 r = 48.  Each of the 224 modules has its own weights (3.5 GB
+    at 4 bits: far beyond L2) and its own activations."""
+    import numpy as np
+    import torch
+    from paper_2601_22716_b200 import binding as lords
+    from paper_2601_22716_b200 import inputs as gen
+
+    protos = {}
+    for idx, name in enumerate(STACK_LAYERS):
+        m, n = gen.LLAMA3_8B_SHAPES[name]
+        mlp = name in ("gate", "up", "down")
+        bits = mlp_bits if mlp else 4
+        r = (48 if bits == 3 else 32) if mlp else (16 if name in ("k", "v") else 32)
+        lay = gen.make_layer(m, n, r, M, bits=bits, seed=idx)
+        packed = lords.lords_pack_codes(lay.codes, bits)
+        protos[name] = (lay, torch.from_numpy(packed).to(device), torch.from_numpy(lay.B.view(np.int16)).to(device),
+                        torch.from_numpy(lay.A.view(np.int16)).to(device), torch.from_numpy(lay.x.view(np.int16)).to(device))
+    calls, byt, flo = [], 0, 0
+    for layer in range(32):
+        for name in STACK_LAYERS:
+            lay, q0, B0, A0, x0 = protos[name]
+            q = q0 if layer == 0 else torch.roll(q0, layer, 0).contiguous()
+            B = B0 if layer == 0 else torch.roll(B0, layer, 0).contiguous()
+            y = torch.zeros((M, lay.m), dtype=torch.int16, device=device)
+            calls.append((lay, q, B, A0.clone(), x0.clone(), y))
+            c = dict(m=lay.m, n=lay.n, bits=lay.bits, r=lay.r, M=M)
+            byt += algorithmic_bytes(c)
+            flo += useful_flops(c)
+
+    def one_pass():
+        for lay, q, B, A, x, y in calls:
+            lords.lords_linear_forward_bits(x, q, B, A, lay.codebook, lay.bits, M, lay.m, lay.n, lay.r, y)
+
+    one_pass()
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        one_pass()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        one_pass()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert lords.lords_poll_status() == 0
+    peaks = measured_peaks()
+    gbs, tfs = byt / (ms * 1e-3) / 1e9, flo / (ms * 1e-3) / 1e12
+    return {"case": f"stack_m{M}_mlp{mlp_bits}bit", "ms_per_pass": ms, "ms_per_token": ms / M, "calls": len(calls),
+            "algorithmic_bytes": byt, "gbs": gbs, "tflops": tfs, "frac_hbm": gbs / peaks["hbm_gbs"],
+            "frac_tensor": tfs / peaks["bf16_tflops"], "steps": steps}
+
+
 def cpu_baseline(case, lay, packed, budget_s=12.0):
     """The oracle as it stands, on the host cores, on a bounded sample of the case."""
     import numpy as np
@@ -358,7 +426,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--case", default=None, help="time only this case (default: headline plus the others)")
     ap.add_argument("--no-extras", action="store_true", help="headline case only")
-    ap.add_argument("--path", default="auto", help="force a kernel path (auto|simt|decode|prefill)")
+    ap.add_argument("--path", default="auto", help="force a kernel path (auto|simt|decode|umma)")
+    ap.add_argument("--stack", action="store_true", help="also time the full Llama-3-8B linear stack (224 modules)")
     args = ap.parse_args()
 
     if args.impl == "reference":
@@ -400,6 +469,12 @@ def main():
                           "gbs": r2["gbs"], "tflops": r2["tflops"], "roofline": r2["roofline"],
                           "copies": r2["copies"], "steps": k})
 
+    stack = []
+    if args.stack and world == 1:
+        for (M, mlp_bits, k) in [(1, 4, 20), (8, 4, 20), (512, 4, 3), (1, 3, 20)]:
+            stack.append(time_stack(M, mlp_bits, k, device))
+            torch.cuda.empty_cache()
+
     if rank == 0:
         hbm = c["bound"] == "hbm"
         value = res["gbs"] if hbm else res["tflops"]
@@ -424,6 +499,8 @@ def main():
                 "ms_per_step": e2e["ms_per_step"]},
             "cpu_baseline": base, "cases": cases,
         }
+        if stack:
+            line["stack"] = stack
         print(json.dumps(line))
     lords.lords_shutdown()
     if world > 1:
