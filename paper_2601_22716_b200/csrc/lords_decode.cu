@@ -638,7 +638,7 @@ template <int BITS, int NTOK, int H> int choose_cluster(int tiles, int ksteps, i
     return cs;
 }
 
-template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem &p, int forced_cs, cudaStream_t stream)
+template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem &p, int forced_cs, int forced_halves, cudaStream_t stream)
 {
     const int qrow = DCfg<BITS, 1>::QROW;
     k.ksteps = (p.n + kStep - 1) / kStep;
@@ -650,7 +650,7 @@ template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem
     double cost1 = 0, cost2 = 0;
     const int cs1 = choose_cluster<BITS, NTOK, 1>(tiles1, k.ksteps, forced_cs, cost1);
     const int cs2 = choose_cluster<BITS, NTOK, 2>(tiles2, k.ksteps, forced_cs, cost2);
-    const bool two = cost2 < cost1;
+    const bool two = forced_halves > 0 ? forced_halves == 2 : cost2 < cost1;
     const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
     if (!make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)qrow,
                      two ? 256u : 128u, BITS == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE) ||
@@ -686,8 +686,8 @@ int launch_decode(const Problem &p, State &st, cudaStream_t stream)
     LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)8 * 32 * 8 * 8, stream));
 #endif
     int rc;
-    if (p.bits == 4) rc = p.M == 1 ? launch_bits_tok<4, 1>(k, p, st.forced_splitk, stream) : launch_bits_tok<4, 2>(k, p, st.forced_splitk, stream);
-    else rc = p.M == 1 ? launch_bits_tok<3, 1>(k, p, st.forced_splitk, stream) : launch_bits_tok<3, 2>(k, p, st.forced_splitk, stream);
+    if (p.bits == 4) rc = p.M == 1 ? launch_bits_tok<4, 1>(k, p, st.forced_splitk, st.forced_halves, stream) : launch_bits_tok<4, 2>(k, p, st.forced_splitk, st.forced_halves, stream);
+    else rc = p.M == 1 ? launch_bits_tok<3, 1>(k, p, st.forced_splitk, st.forced_halves, stream) : launch_bits_tok<3, 2>(k, p, st.forced_splitk, st.forced_halves, stream);
     if (rc != LORDS_OK) return rc;
     st.last_launches = 1;
     st.last_path = "decode";
