@@ -31,7 +31,7 @@
  *     the call; the library neither retains nor frees them.  x/y aliasing is undefined.
  *   - the tensor-core kernels are launched with programmatic dependent launch: they may begin while
  *     the previous kernel on `stream` is still draining, and until that kernel has finished they
- *     read only the weights (Qpacked, A); x is read, and y written, after it.  So the weights must
+ *     read only the weights (Qpacked, B, A); x is read, and y written, after it.  So the weights must
  *     not be produced by work that is still in flight on `stream` when a forward call is made
  *     (synchronise the stream once after loading or updating weights); activations may be.
  *   - forward calls validate on the host, enqueue work on `stream` and return
