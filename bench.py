@@ -117,6 +117,23 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(ms, device, world):
+    """A job's step time is that of its slowest rank: MAX-reduce the per-rank device time."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(per_rank_value, world):
+    """Replicas only: every rank processes the same amount of work, so the job's throughput is the
+    per-rank throughput (at the slowest rank's time) times the number of ranks."""
+    return per_rank_value * world
+
+
 def make_case_layers(case, copies, device):
     """One host-seeded layer per case; the other weight copies are row-rotations of it
     (distinct HBM addresses, same statistics), built on the device."""
@@ -206,11 +223,7 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
     e1.record()
     barrier()
     clocks = sampler.stop() if sampler is not None else None
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), device, world)
     ms_per_step = ms / steps
     assert lords.lords_poll_status() == 0
 
@@ -233,11 +246,7 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
             e2e_step()
         e1.record()
         barrier()
-        ems = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ems], dtype=torch.float64, device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
+        ems = max_over_ranks(e0.elapsed_time(e1), device, world)
         e2e = {"ms_per_step": ems / e2e_steps, "h2d_bytes_per_step": copies * M * n * 2,
                "d2h_bytes_per_step": copies * M * m * 2}
 
@@ -260,7 +269,7 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
     roof["us_per_launch"] = us_per_launch
     res = {
         "case": case, "path": path, "copies": copies, "ms_per_step": ms_per_step, "us_per_call": us_per_launch,
-        "gbs": gbs * world, "tflops": tfs * world, "roofline": roof, "clocks": clocks,
+        "gbs": whole_job_value(gbs, world), "tflops": whole_job_value(tfs, world), "roofline": roof, "clocks": clocks,
         "launches_per_call": launches_per_call, "gpu_launches": steps * calls * launches_per_call,
         "graph": graph is not None,
     }
