@@ -420,9 +420,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                                       lane_addr + kWCol + (uint32_t)((h * S + s) * kWSlotCols));
             // one settling point for both products of the step: the B-operand stores become visible
             // to the tensor core's (async-proxy) reads, the TMEM stores complete
+            if (stamper) DSTAMP(1 + g, it, 5);
             fence_proxy_async_smem();
+            if (stamper) DSTAMP(1 + g, it, 6);
             tmem_wait_st();
             tc_fence_before_sync();
+            if (stamper) DSTAMP(1 + g, it, 7);
             __syncwarp();
             if (lane == 0) {
 #pragma unroll
