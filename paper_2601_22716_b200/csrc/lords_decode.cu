@@ -199,8 +199,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     // The cluster shares one tile of 128 * H rows; rank r takes the r-th slice of its k-steps.
     const int csize = (int)cluster_nctarank(), rank = (int)cluster_ctarank();
     const int tile = (int)blockIdx.x / csize;
-    const int ks_a = (int)((long long)rank * p.ksteps / csize);
-    const int ks_b = (int)((long long)(rank + 1) * p.ksteps / csize);
+    const int ks_a = rank * p.ksteps / csize;          // rank < 16 and ksteps < 2^24: no overflow
+    const int ks_b = (rank + 1) * p.ksteps / csize;
     const int total = ks_b - ks_a;
     const int N = NTOK * p.r_pad;
 
@@ -446,6 +446,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             for (int c = 0; c < kNMax / 8; ++c)
                 bq[c] = (i < p.m && c * 8 < p.r) ? __ldg(reinterpret_cast<const uint4 *>(p.B + (size_t)i * p.r) + c)
                                                  : make_uint4(0, 0, 0, 0);
+            // second half of the split-phase cluster barrier (every CTA of the cluster has initialised
+            // its barriers): taken here, where its latency hides behind the wait for the last MMAs
+            if (csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
             float yt[NTOK];
 #pragma unroll
             for (int t = 0; t < NTOK; ++t) yt[t] = 0.0f;
@@ -492,7 +495,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                     for (int t = 0; t < NTOK; ++t) store_out(p.y, p.y_f32, (size_t)t * p.m + i, yt[t]);
             } else {
                 // a CTA that gave up still arrives (with zeros), so the leader never waits in vain
-                asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 #pragma unroll
                 for (int t = 0; t < NTOK; ++t)
                     st_cluster_f32(map_to_rank(red0 + ((rank * NTOK + t) * kTileRows + row_in_tile) * 4, 0), yt[t]);
