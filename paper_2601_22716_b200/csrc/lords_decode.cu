@@ -13,20 +13,19 @@
 // leader adds the partials in rank order -- deterministic, no float atomics, no trip through
 // global memory.
 //
-// Warp roles (20 warps):
-//   0..15  two worker groups of eight warps take k-steps alternately.  For its k-step a group
-//          (a) turns the factor tile A[:, k-step] (TMA, shared memory) in place into the fp16 B
-//              operand A_kj * x_tj, and
-//          (b) dequantises: a warp owns 32 rows (H = 2: all 128 columns of the k-step; H = 1: one
-//              64-column half); a thread reads its row's packed codes from shared memory, looks every
-//              code pair up in a lane-private fp16x2 level table and stores the levels straight into
-//              TMEM as the A operand (tcgen05.st).
+// Warp roles (28 warps):
+//   0..15  two worker groups of eight warps take k-steps alternately and dequantise: a warp owns 32
+//          rows (H = 2: all 128 columns of the k-step; H = 1: one 64-column half); a thread reads its
+//          row's packed codes from shared memory, looks every code pair up in a lane-private fp16x2
+//          level table and stores the levels straight into TMEM as the A operand (tcgen05.st).
 //          Group 0 also runs the epilogue.
-//   16,17  MMA issuers: D[128 x N] += W[128 x 16] * AX[N x 16]^T with A from TMEM and B from shared
+//   16..23 two converter groups of four warps take k-steps alternately: they turn the factor tile
+//          A[:, k-step] (TMA, shared memory) in place into the fp16 B operand A_kj * x_tj.
+//   24,25  MMA issuers: D[128 x N] += W[128 x 16] * AX[N x 16]^T with A from TMEM and B from shared
 //          memory, eight per k-step; one issuer per 128-row half (H = 2) or per k-step parity (H = 1).
-//   18     TMA producer of the packed code tiles (HBM stream, deep ring); it also initialises the
+//   26     TMA producer of the packed code tiles (HBM stream, deep ring); it also initialises the
 //          barriers and starts the stream before the rest of the CTA has finished its set-up.
-//   19     TMA producer of the factor tiles.
+//   27     TMA producer of the factor tiles and of the k-step's slice of x.
 //
 // Every wait is bounded; on expiry the role records LORDS_ERR_TIMEOUT and leaves its loop, so
 // the kernel always reaches its final barrier and frees its TMEM.
@@ -46,11 +45,14 @@ namespace {
 using namespace ptx;
 
 constexpr int kWorkWarps = 16;                         // worker warps: two groups of eight
-constexpr int kIssuerWarp0 = kWorkWarps;               // 16, 17: one per half (H == 2) or per k-step parity (H == 1)
-constexpr int kTmaQWarp = kIssuerWarp0 + 2;            // 18
-constexpr int kTmaAWarp = kTmaQWarp + 1;               // 19
-constexpr int kWarps = kTmaAWarp + 1;                  // 20
-constexpr int kThreads = kWarps * 32;                  // 640
+constexpr int kConvWarp0 = kWorkWarps;                 // 16..23: converters of the factor tiles
+constexpr int kConvGroupWarps = 4;
+constexpr int kConvGroups = 2;
+constexpr int kIssuerWarp0 = kConvWarp0 + kConvGroups * kConvGroupWarps;   // 24, 25: one per half (H == 2) or per k-step parity (H == 1)
+constexpr int kTmaQWarp = kIssuerWarp0 + 2;            // 26
+constexpr int kTmaAWarp = kTmaQWarp + 1;               // 27
+constexpr int kWarps = kTmaAWarp + 1;                  // 28
+constexpr int kThreads = kWarps * 32;                  // 896
 constexpr int kNMax = 64;                              // accumulator columns per half (N = M * r_pad)
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kWCol = 2 * kNMax;                  // W ring starts behind the accumulators
@@ -72,11 +74,12 @@ template <int BITS, int H> struct DCfg {
     static constexpr int S_TMEM = (512 - (int)kWCol) / (H * kWSlotCols);
     static constexpr int S = S_TMEM < 4 ? S_TMEM : 4;          // W / factor ring depth (4 / 3)
     static constexpr int AXSTAGE = kAtoms * kAtomBytes;
+    static constexpr int XSTAGE = 2 * kStep * 2;               // the k-step's slice of x, two tokens (bf16)
     static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;   // one entry per code pair
     static constexpr int LUT_BYTES = LUT_ENTRIES * 128;        // 32 lane-private copies
     static constexpr int RED_BYTES = kClusterMax * 2 * TILE_ROWS * 4;   // the cluster's partials, [rank][token][row]
     static constexpr int BAR_BYTES = 512;
-    static constexpr int SMEM = LUT_BYTES /*alignment slack*/ + LUT_BYTES + SQ * QSTAGE + S * AXSTAGE + RED_BYTES + BAR_BYTES;
+    static constexpr int SMEM = LUT_BYTES /*alignment slack*/ + LUT_BYTES + SQ * QSTAGE + S * (AXSTAGE + XSTAGE) + RED_BYTES + BAR_BYTES;
     // the code ring's depth is a multiple of the group count, so each of its barriers is used by
     // one group alone, which then sees every phase of it
     static_assert(SQ % GROUPS == 0, "code ring depth must be a multiple of the group count");
@@ -176,20 +179,22 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     const uint32_t lut = (raw + C::LUT_BYTES - 1) & ~(uint32_t)(C::LUT_BYTES - 1);   // table-size aligned: entry offsets OR in
     const uint32_t q0 = lut + C::LUT_BYTES;
     const uint32_t ax0 = q0 + SQ * C::QSTAGE;          // multiple of 1024
-    const uint32_t red0 = ax0 + S * C::AXSTAGE;        // [kClusterMax][NTOK][rows] floats: the cluster's partials (leader's copy is used)
+    const uint32_t xs0 = ax0 + S * C::AXSTAGE;         // x slices of the k-steps in flight, [stage][token][128] bf16
+    const uint32_t red0 = xs0 + S * C::XSTAGE;         // [kClusterMax][NTOK][rows] floats: the cluster's partials (leader's copy is used)
     const uint32_t bars = red0 + C::RED_BYTES;
     // mbarriers, 8 bytes each, in one run so that a warp can initialise them lane-parallel
     constexpr int kBarQFull = 0;                            // SQ, 1 arrival + TMA bytes
     constexpr int kBarQEmpty = kBarQFull + SQ;              // SQ, the warps of one group
     constexpr int kBarAFull = kBarQEmpty + SQ;              // S, 1 arrival + TMA bytes
-    constexpr int kBarReady = kBarAFull + S;                // H * S: the warps of one group (W slot and B operand written)
+    constexpr int kBarAxReady = kBarAFull + S;              // S: the warps of one converter group (B operand written)
+    constexpr int kBarReady = kBarAxReady + S;              // H * S: the warps of one worker group (W slot written)
     constexpr int kBarMmaDone = kBarReady + H * S;          // S, one commit per half
     constexpr int kBarAccFull = kBarMmaDone + S;            // 2: one per issuer
     constexpr int kBarReduce = kBarAccFull + 2;             // 1: every epilogue warp of every CTA of the cluster
     constexpr int kBarCount = kBarReduce + 1;
     static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
     const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
-    const uint32_t bar_a_full = bars + 8 * kBarAFull, bar_ready = bars + 8 * kBarReady;
+    const uint32_t bar_a_full = bars + 8 * kBarAFull, bar_ax_ready = bars + 8 * kBarAxReady, bar_ready = bars + 8 * kBarReady;
     const uint32_t bar_mma_done = bars + 8 * kBarMmaDone, bar_acc_full = bars + 8 * kBarAccFull;
     const uint32_t bar_reduce = bars + 8 * kBarReduce;
     const uint32_t tmem_slot = bars + 8 * kBarCount;
@@ -216,7 +221,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         for (int b = lane; b < kBarCount; b += 32) {
             uint32_t count = 1;
             if (b >= kBarQEmpty && b < kBarAFull) count = kGroupWarps;
-            else if (b >= kBarReady && b < kBarMmaDone) count = kGroupWarps;
+            else if (b >= kBarAxReady && b < kBarReady) count = kConvGroupWarps;
+            else if (b >= kBarReady && b < kBarMmaDone) count = kGroupWarps / H;   // the warps that fill this half's W slot
             else if (b >= kBarMmaDone && b < kBarAccFull) count = H;   // H == 1: the step's one issuer
             else if (b == kBarReduce) count = (uint32_t)(4 * H * csize);
             mbar_init(bars + 8 * b, count);
@@ -275,17 +281,28 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     if (warp == kTmaQWarp) {
         // all done above
     } else if (warp == kTmaAWarp) {
-        // ------------------------------------------------------------------ factor tiles A[:, k-step]
+        // ------------------------------------------------------------------ factor tiles A[:, k-step] and x[:, k-step]
         if (lane == 0) {
-            const uint32_t tx = (uint32_t)(kAtoms * p.r_pad * 128);
+            // x may be the previous launch's output: everything before this line only touched weights.
+            // Nothing of this launch reaches global memory before its MMAs have run, and those need
+            // the B operand made from these loads, so this one wait orders the whole launch behind
+            // the previous one.
+            DSTAMP(6, 0, 3);
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            DSTAMP(6, 0, 4);
+            const uint32_t tx_a = (uint32_t)(kAtoms * p.r_pad * 128);
             for (int it = 0; it < total; ++it) {
-                const int s = it % S;
+                const int s = it % S, j0 = (ks_a + it) * kStep;
                 if (it >= S && !mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1))) { failed = true; break; }
                 const uint32_t bar = bar_a_full + 8 * s;
-                mbar_expect_tx(bar, tx);
+                const uint32_t xbytes = (uint32_t)(2 * (p.n - j0 < kStep ? p.n - j0 : kStep));   // a multiple of 64
+                mbar_expect_tx(bar, tx_a + NTOK * xbytes);
 #pragma unroll
                 for (int at = 0; at < kAtoms; ++at)
-                    tma_load_2d(ax0 + s * C::AXSTAGE + at * kAtomBytes, &p.tm_a, (ks_a + it) * kStep + at * 64, 0, bar);
+                    tma_load_2d(ax0 + s * C::AXSTAGE + at * kAtomBytes, &p.tm_a, j0 + at * 64, 0, bar);
+#pragma unroll
+                for (int t = 0; t < NTOK; ++t)
+                    bulk_load(xs0 + s * C::XSTAGE + t * (kStep * 2), p.x + (size_t)t * p.n + j0, xbytes, bar);
             }
         }
     } else if (warp >= kIssuerWarp0) {
@@ -307,7 +324,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         for (int it = first; it < total; it += kStride) {
             const int s = it % S;
             if (j == 0 && lane == 0) DSTAMP(0, it, 0);
-            if (!mbar_wait(bar_ready + 8 * (h * S + s), (uint32_t)((it / S) & 1))) { failed = true; break; }
+            if (!mbar_wait(bar_ax_ready + 8 * s, (uint32_t)((it / S) & 1)) ||
+                !mbar_wait(bar_ready + 8 * (h * S + s), (uint32_t)((it / S) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (j == 0 && lane == 0) DSTAMP(0, it, 1);
             if (lane == 0) {
@@ -323,54 +341,20 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             }
             __syncwarp();
         }
-    } else {
-        // ------------------------------------------------------------------ worker warps
-        // warp wg of a group: lane quadrant q; H == 2: row half h, all 128 columns of the k-step;
-        // H == 1: the one row half, column half ch
-        const int g = warp / kGroupWarps, wg = warp % kGroupWarps, q = warp & 3;
-        const int h = H == 2 ? (wg >> 2) : 0, ch = H == 2 ? 0 : (wg >> 2);
-        const int row_in_tile = h * 128 + q * 32 + lane;
-        uint32_t tmem_base;
-        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-        const uint32_t lut_lane = lut + 4u * (uint32_t)lane;
-        const bool stamper = wg == 0 && lane == 0 && g < 2;
-        // B-operand share of this lane: the 16-byte chunk c16 (8 columns) of rows rsub + kRowStep * i
-        const int c16 = lane & 7, rsub = wg * 4 + (lane >> 3);
-        constexpr int kRowStep = 4 * kGroupWarps;                        // 32
-        constexpr int kRowIters = (kNMax + kRowStep - 1) / kRowStep;     // 2
-
-        uint4 xr[NTOK][kAtoms];
-        auto load_x = [&](int ks) {
-#pragma unroll
-            for (int t = 0; t < NTOK; ++t)
-#pragma unroll
-                for (int at = 0; at < kAtoms; ++at) {
-                    const int j = ks * kStep + at * 64 + c16 * 8;
-                    xr[t][at] = j < p.n ? __ldg(reinterpret_cast<const uint4 *>(p.x + (size_t)t * p.n + j))
-                                        : make_uint4(0, 0, 0, 0);
-                }
-        };
-        // x may be the previous launch's output: everything above this line only touched weights
-        if (tid == 0) DSTAMP(6, 0, 3);
-        asm volatile("griddepcontrol.wait;" ::: "memory");
-        if (tid == 0) DSTAMP(6, 0, 4);
-        if (g < total) load_x(ks_a + g);
-
-        for (int it = g; it < total; it += kGroups) {
-            const int sq = it % SQ, s = it % S;
-            if (stamper) DSTAMP(1 + g, it, 0);
-            // order matters for the factor ring when its depth is odd: the MMA of step it - S being
-            // complete implies the factor tile of step it - S had landed, so the phase of a_full
-            // waited on next is the one for this step
-            bool ok = true;
-            if (it >= S) ok = mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1));
-            if (ok) ok = mbar_wait(bar_a_full + 8 * s, (uint32_t)((it / S) & 1));
-            if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-            tc_fence_after_sync();
-            if (stamper) DSTAMP(1 + g, it, 1);
-
-            // (a) B operand: A_kj * x_tj as fp16, in place (token 0) and behind it (token 1)
+    } else if (warp >= kConvWarp0) {
+        // ------------------------------------------------------------------ converters
+        // B operand: A_kj * x_tj as fp16, in place (token 0) and behind it (token 1).  A lane owns the
+        // 16-byte chunk c16 (8 columns) of rows rsub + kRowStep * i of both 64-column atoms.
+        const int cgp = (warp - kConvWarp0) / kConvGroupWarps, cw = (warp - kConvWarp0) % kConvGroupWarps;
+        const int c16 = lane & 7, rsub = cw * 4 + (lane >> 3);
+        constexpr int kRowStep = 4 * kConvGroupWarps;          // 16
+        constexpr int kRowIters = kNMax / kRowStep;            // 4
+        const bool cstamper = cw == 0 && lane == 0 && cgp == 0;
+        for (int it = cgp; it < total; it += kConvGroups) {
+            const int s = it % S;
+            if (cstamper) DSTAMP(4, it, 0);
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full + 8 * s, (uint32_t)((it / S) & 1)))) { failed = true; break; }
+            if (cstamper) DSTAMP(4, it, 1);
 #pragma unroll
             for (int at = 0; at < kAtoms; ++at) {
                 const uint32_t atom = ax0 + s * C::AXSTAGE + at * kAtomBytes;
@@ -383,7 +367,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 float xf[NTOK][8];
 #pragma unroll
                 for (int t = 0; t < NTOK; ++t) {
-                    const uint32_t xw[4] = {xr[t][at].x, xr[t][at].y, xr[t][at].z, xr[t][at].w};
+                    // columns past n hold nothing the copy wrote: take zero there
+                    const bool in = (ks_a + it) * kStep + at * 64 + c16 * 8 < p.n;
+                    const uint4 xv = in ? lds_v4(xs0 + s * C::XSTAGE + t * (kStep * 2) + at * 128 + c16 * 16) : make_uint4(0, 0, 0, 0);
+                    const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         xf[t][2 * e] = __uint_as_float(xw[e] << 16);
@@ -410,26 +397,45 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                     }
                 }
             }
-            if (it + kGroups < total) load_x(ks_a + it + kGroups);   // the group's next k-step
-            if (stamper) DSTAMP(1 + g, it, 2);
+            // the stores above become visible to the tensor core's (async-proxy) reads
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_ax_ready + 8 * s);
+            if (cstamper) DSTAMP(4, it, 2);
+        }
+    } else {
+        // ------------------------------------------------------------------ worker warps
+        // warp wg of a group: lane quadrant q; H == 2: row half h, all 128 columns of the k-step;
+        // H == 1: the one row half, column half ch
+        const int g = warp / kGroupWarps, wg = warp % kGroupWarps, q = warp & 3;
+        const int h = H == 2 ? (wg >> 2) : 0, ch = H == 2 ? 0 : (wg >> 2);
+        const int row_in_tile = h * 128 + q * 32 + lane;
+        uint32_t tmem_base;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t lut_lane = lut + 4u * (uint32_t)lane;
+        const bool stamper = wg == 0 && lane == 0 && g < 2;
 
-            // (b) codes -> levels -> TMEM
+        for (int it = g; it < total; it += kGroups) {
+            const int sq = it % SQ, s = it % S;
+            if (stamper) DSTAMP(1 + g, it, 0);
+            // the W slot is free once the MMAs of step it - S have completed
+            if (it >= S && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1)))) { failed = true; break; }
+            tc_fence_after_sync();
+            if (stamper) DSTAMP(1 + g, it, 1);
+
+            // codes -> levels -> TMEM
             if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1)))) { failed = true; break; }
             if (stamper) DSTAMP(1 + g, it, 4);
             dequant_row_to_tmem<BITS, C::COLS>(q0 + sq * C::QSTAGE + row_in_tile * C::QROW, row_in_tile, ch, lut_lane,
                                       lane_addr + kWCol + (uint32_t)((h * S + s) * kWSlotCols));
-            // one settling point for both products of the step: the B-operand stores become visible
-            // to the tensor core's (async-proxy) reads, the TMEM stores complete
             if (stamper) DSTAMP(1 + g, it, 5);
-            fence_proxy_async_smem();
-            if (stamper) DSTAMP(1 + g, it, 6);
             tmem_wait_st();
             tc_fence_before_sync();
             if (stamper) DSTAMP(1 + g, it, 7);
             __syncwarp();
             if (lane == 0) {
-#pragma unroll
-                for (int hh = 0; hh < H; ++hh) mbar_arrive(bar_ready + 8 * (hh * S + s));
+                mbar_arrive(bar_ready + 8 * (h * S + s));
                 mbar_arrive(bar_q_empty + 8 * sq);
             }
             if (stamper) DSTAMP(1 + g, it, 3);

@@ -74,6 +74,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, int 
         ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
+// Untiled bulk copy global -> this CTA's shared memory; both addresses 16-byte aligned, bytes a
+// multiple of 16; completion is counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const void *tmap)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
