@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     constexpr int kBarReady = kBarAxReady + S;              // H * S: the warps of one worker group (W slot written)
     constexpr int kBarMmaDone = kBarReady + H * S;          // S, one commit per half
     constexpr int kBarAccFull = kBarMmaDone + S;            // 2: one per issuer
-    constexpr int kBarReduce = kBarAccFull + 2;             // 1: every epilogue warp of every CTA of the cluster
+    constexpr int kBarReduce = kBarAccFull + 2;             // 1: counts the bytes of the cluster's partial sums (leader's copy is used)
     constexpr int kBarCount = kBarReduce + 1;
     static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
     const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
@@ -224,11 +224,13 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             else if (b >= kBarAxReady && b < kBarReady) count = kConvGroupWarps;
             else if (b >= kBarReady && b < kBarMmaDone) count = kGroupWarps / H;   // the warps that fill this half's W slot
             else if (b >= kBarMmaDone && b < kBarAccFull) count = H;   // H == 1: the step's one issuer
-            else if (b == kBarReduce) count = (uint32_t)(4 * H * csize);
             mbar_init(bars + 8 * b, count);
         }
         fence_mbar_init();
         __syncwarp();
+        // the leader's reduce barrier counts the bytes of the cluster's partial sums (its one
+        // arrival is this one); the stores may come before or after, the phase ends when both are in
+        if (rank == 0 && lane == 0 && csize > 1) mbar_expect_tx(bar_reduce, (uint32_t)(csize * NTOK * kTileRows * 4));
         asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");   // barriers exist; does not wait for the others
         // split-phase cluster barrier: arrive now (this CTA's reduce barrier exists and the fence above
         // has published it cluster-wide, so a relaxed arrival is enough); the wait is in the epilogue,
@@ -501,11 +503,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                     for (int t = 0; t < NTOK; ++t) store_out(p.y, p.y_f32, (size_t)t * p.m + i, yt[t]);
             } else {
                 // a CTA that gave up still arrives (with zeros), so the leader never waits in vain
+                const uint32_t leader_bar = map_to_rank(bar_reduce, 0);
 #pragma unroll
                 for (int t = 0; t < NTOK; ++t)
-                    st_cluster_f32(map_to_rank(red0 + ((rank * NTOK + t) * kTileRows + row_in_tile) * 4, 0), yt[t]);
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(map_to_rank(bar_reduce, 0));
+                    st_async_cluster_f32(map_to_rank(red0 + ((rank * NTOK + t) * kTileRows + row_in_tile) * 4, 0), yt[t], leader_bar);
                 if (stamper) DSTAMP(5, 0, 3);
                 if (rank == 0) {
                     if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0))) failed = true;
