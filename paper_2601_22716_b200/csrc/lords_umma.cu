@@ -219,11 +219,14 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             uint32_t count = 1;
             if (b >= kBarQEmpty && b < kBarSFull) count = kWorkWarps;
             else if (b >= kBarSEmpty && b < kBarAccFull) count = kGroupWarps;   // s_empty and w_full
-            else if (b == kBarReduce) count = BN == 16 ? (uint32_t)(4 * csize) : (uint32_t)(4 * (BN / (BN >= 64 ? BN / 4 : 16)));
+            else if (b == kBarReduce) count = BN == 16 ? 1u : (uint32_t)(4 * (BN / (BN >= 64 ? BN / 4 : 16)));
             mbar_init(bars + 8 * b, count);
         }
         fence_mbar_init();
         __syncwarp();
+        // BN == 16: the leader's reduce barrier counts the bytes of the cluster's partial sums (its one
+        // arrival is this one); the stores may come before or after, the phase ends when both are in
+        if (BN == 16 && rank == 0 && lane == 0 && csize > 1) mbar_expect_tx(bar_reduce, (uint32_t)(csize * 16 * BM * 4));
         asm volatile("bar.arrive 1, %0;" ::"n"(kThreads) : "memory");   // barriers exist; does not wait for the others
         // split-phase cluster barrier: the fence above has published this CTA's barriers cluster-wide,
         // a relaxed arrival is enough; the wait is in the epilogue before the first remote access
@@ -453,6 +456,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         const int cg = warp >> 2;
         if (cg * CPG < BN && !failed) {
             bool ok = true;
+            // BN == 16, k-range split over the cluster: the second half of the split-phase cluster barrier
+            // (every CTA has initialised its barriers) is taken here, behind the wait for the last MMAs
+            if (BN == 16 && csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
             if (total > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, 0));
             tc_fence_after_sync();
             const int i = row0 + row;
@@ -501,12 +507,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                     tmem_ld_32x16(lane_addr, v);
                     tmem_wait_ld();
                 }
-                asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+                const uint32_t leader_bar = map_to_rank(bar_reduce, 0);
 #pragma unroll
                 for (int c = 0; c < 16; ++c)
-                    st_cluster_f32(map_to_rank(red0 + (uint32_t)(((rank * 16 + c) * BM + row) * 4), 0), __uint_as_float(v[c]));
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(map_to_rank(bar_reduce, 0));
+                    st_async_cluster_f32(map_to_rank(red0 + (uint32_t)(((rank * 16 + c) * BM + row) * 4), 0), __uint_as_float(v[c]), leader_bar);
                 if (rank == 0) {
                     if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0))) failed = true;
                     else if (i < p.m) {
