@@ -76,10 +76,20 @@ template <int BITS, int H> struct DCfg {
     static constexpr int AXSTAGE = kAtoms * kAtomBytes;
     static constexpr int XSTAGE = 2 * kStep * 2;               // the k-step's slice of x, two tokens (bf16)
     static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;   // one entry per code pair
-    static constexpr int LUT_BYTES = LUT_ENTRIES * 128;        // 32 lane-private copies
+    // 32 lane-private copies of every entry (word = lane, so the lookups of a warp never conflict).
+    // 4-bit: an entry every 256 bytes and the table on a 64 KB boundary, which lets one byte
+    // permute build a lookup address: byte 0 = 4 * lane, byte 1 = the code pair's byte, bytes 2..3 =
+    // the table's base.  3-bit: an entry every 128 bytes, offsets OR-ed into the table-size-aligned base.
+    static constexpr int LUT_STRIDE = BITS == 4 ? 256 : 128;
+    static constexpr int LUT_BYTES = LUT_ENTRIES * LUT_STRIDE;
     static constexpr int RED_BYTES = kClusterMax * 2 * TILE_ROWS * 4;   // the cluster's partials, [rank][token][row]
     static constexpr int BAR_BYTES = 512;
-    static constexpr int SMEM = LUT_BYTES /*alignment slack*/ + LUT_BYTES + SQ * QSTAGE + S * (AXSTAGE + XSTAGE) + RED_BYTES + BAR_BYTES;
+    // 4-bit: the buffers are laid out around the table, some before its 64 KB boundary, the rest
+    // behind it, inside the largest shared-memory window a CTA can have; AX_LOW of the factor stages
+    // sit in the lower part
+    static constexpr int AX_LOW = BITS == 4 ? (H == 1 ? 2 : 1) : S;
+    static constexpr int SMEM = BITS == 4 ? 232448
+                                          : LUT_BYTES /*alignment slack*/ + LUT_BYTES + SQ * QSTAGE + S * (AXSTAGE + XSTAGE) + RED_BYTES + BAR_BYTES;
     // the code ring's depth is a multiple of the group count, so each of its barriers is used by
     // one group alone, which then sees every phase of it
     static_assert(SQ % GROUPS == 0, "code ring depth must be a multiple of the group count");
@@ -141,9 +151,9 @@ __device__ __forceinline__ void dequant_row_to_tmem(uint32_t qrow, int row, int 
             for (int wi = 0; wi < 8; ++wi)
 #pragma unroll
                 for (int b = 0; b < 4; ++b) {
-                    // byte b of the word holds two codes; entry offset = byte * 128
-                    const uint32_t sh = b == 0 ? (w[wi] << 7) : (w[wi] >> (8 * b - 7));
-                    out[wi * 4 + b] = lds_u32((sh & 0x7F80u) | lut_lane);
+                    // byte b of the word holds two codes, its entry sits at byte * 256: the address is
+                    // the table's lane address with that byte as byte 1
+                    out[wi * 4 + b] = lds_u32(__byte_perm(w[wi], lut_lane, 0x7604u | (uint32_t)(b << 4)));
                 }
             tmem_st_32x32(taddr + half * 32, out);
         }
@@ -176,12 +186,32 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     constexpr int S = C::S, SQ = C::SQ, kTileRows = C::TILE_ROWS, kGroups = C::GROUPS, kGroupWarps = C::GROUP_WARPS;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t lut = (raw + C::LUT_BYTES - 1) & ~(uint32_t)(C::LUT_BYTES - 1);   // table-size aligned: entry offsets OR in
-    const uint32_t q0 = lut + C::LUT_BYTES;
-    const uint32_t ax0 = q0 + SQ * C::QSTAGE;          // multiple of 1024
-    const uint32_t xs0 = ax0 + S * C::AXSTAGE;         // x slices of the k-steps in flight, [stage][token][128] bf16
-    const uint32_t red0 = xs0 + S * C::XSTAGE;         // [kClusterMax][NTOK][rows] floats: the cluster's partials (leader's copy is used)
-    const uint32_t bars = red0 + C::RED_BYTES;
+    const uint32_t lut = (raw + C::LUT_BYTES - 1) & ~(uint32_t)(C::LUT_BYTES - 1);   // table-size aligned
+    // q0: code ring; ax_lo / ax_hi: factor stages 0 .. AX_LOW-1 and AX_LOW .. S-1 (tile bases are
+    // multiples of 1024); xs0: x slices of the k-steps in flight, [stage][token][128] bf16;
+    // red0: [kClusterMax][NTOK][rows] floats, the cluster's partials (leader's copy is used)
+    constexpr int kAxLow = C::AX_LOW;
+    uint32_t q0, ax_lo, ax_hi, xs0, red0, bars;
+    bool fits = true;
+    if constexpr (BITS == 4) {
+        ax_lo = (raw + 1023u) & ~1023u;
+        xs0 = ax_lo + kAxLow * C::AXSTAGE;
+        red0 = xs0 + ((S * C::XSTAGE + 1023) & ~1023);
+        bars = red0 + C::RED_BYTES;
+        q0 = lut + C::LUT_BYTES;
+        ax_hi = q0 + SQ * C::QSTAGE;
+        fits = bars + C::BAR_BYTES <= lut && ax_hi + (S - kAxLow) * C::AXSTAGE <= raw + (uint32_t)C::SMEM;
+    } else {
+        q0 = lut + C::LUT_BYTES;
+        ax_lo = q0 + SQ * C::QSTAGE;
+        ax_hi = ax_lo;
+        xs0 = ax_lo + S * C::AXSTAGE;
+        red0 = xs0 + S * C::XSTAGE;
+        bars = red0 + C::RED_BYTES;
+    }
+    auto ax_stage = [&](int s) -> uint32_t {
+        return s < kAxLow ? ax_lo + (uint32_t)(s * C::AXSTAGE) : ax_hi + (uint32_t)((s - kAxLow) * C::AXSTAGE);
+    };
     // mbarriers, 8 bytes each, in one run so that a warp can initialise them lane-parallel
     constexpr int kBarQFull = 0;                            // SQ, 1 arrival + TMA bytes
     constexpr int kBarQEmpty = kBarQFull + SQ;              // SQ, the warps of one group
@@ -211,6 +241,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
 
     if (tid == 0) DSTAMP(7, 0, 0);
     bool failed = false;
+    if (!fits) {
+        // the shared-memory window does not hold the layout (cannot happen with the window the host
+        // asks for; checked because every address below depends on it)
+        if (tid == 0) atomicExch(p.status, LORDS_ERR_CUDA);
+        return;
+    }
 
     if (warp == kTmaQWarp && lane == 0) DSTAMP(6, 0, 0);
     if (warp == kTmaQWarp) {
@@ -265,7 +301,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 const int lo = BITS == 4 ? (entry & 15) : (entry & 7);
                 const int hi = BITS == 4 ? (entry >> 4) : (entry >> 3);
                 const __half2 v = __floats2half2_rn(p.levels[lo], p.levels[hi]);
-                sts_u32(lut + 4u * (uint32_t)(entry * 32 + lane), *reinterpret_cast<const uint32_t *>(&v));
+                sts_u32(lut + (uint32_t)(entry * C::LUT_STRIDE + 4 * lane), *reinterpret_cast<const uint32_t *>(&v));
             }
             if (tid == 0) DSTAMP(7, 0, 5);
         }
@@ -301,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 mbar_expect_tx(bar, tx_a + NTOK * xbytes);
 #pragma unroll
                 for (int at = 0; at < kAtoms; ++at)
-                    tma_load_2d(ax0 + s * C::AXSTAGE + at * kAtomBytes, &p.tm_a, j0 + at * 64, 0, bar);
+                    tma_load_2d(ax_stage(s) + at * kAtomBytes, &p.tm_a, j0 + at * 64, 0, bar);
 #pragma unroll
                 for (int t = 0; t < NTOK; ++t)
                     bulk_load(xs0 + s * C::XSTAGE + t * (kStep * 2), p.x + (size_t)t * p.n + j0, xbytes, bar);
@@ -320,7 +356,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         const uint32_t idesc = (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);  // fp16 x fp16 -> fp32, K-major
         const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
-        const uint32_t ax_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((ax0 & 0x3FFFFu) >> 4);
+        const uint32_t desc_lo = (uint32_t)umma_desc_sw128(0, 1024, 16);
         const uint32_t acc = tmem_base + (uint32_t)(j * kNMax);
         const int first = H == 2 ? 0 : j;
         for (int it = first; it < total; it += kStride) {
@@ -332,7 +368,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             if (j == 0 && lane == 0) DSTAMP(0, it, 1);
             if (lane == 0) {
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)((h * S + s) * kWSlotCols);
-                const uint32_t b_lo = ax_lo0 + (uint32_t)(s * (C::AXSTAGE >> 4));
+                const uint32_t b_lo = desc_lo | ((ax_stage(s) & 0x3FFFFu) >> 4);
 #pragma unroll
                 for (int k = 0; k < kStep / 16; ++k)
                     umma_f16_ts(acc, wslot + k * 8, umma_desc_pack(b_lo + (k >> 2) * (kAtomBytes >> 4) + (k & 3) * 2, desc_hi),
@@ -359,7 +395,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             if (cstamper) DSTAMP(4, it, 1);
 #pragma unroll
             for (int at = 0; at < kAtoms; ++at) {
-                const uint32_t atom = ax0 + s * C::AXSTAGE + at * kAtomBytes;
+                const uint32_t atom = ax_stage(s) + at * kAtomBytes;
                 uint4 av[kRowIters];
 #pragma unroll
                 for (int i = 0; i < kRowIters; ++i) {
