@@ -72,11 +72,17 @@ static int forward_common(const void *x, const uint8_t *q, const void *B, const 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
     // Dispatch.  Each tensor-core path declines (LORDS_ERR_UNSUPPORTED) shapes outside its rules;
-    // "auto" tries the decode kernel (M <= 2), then the scale-MMA kernel, then the CUDA-core path.
+    // "auto" tries the decode kernels (M <= 2, then 3 <= M <= 16), then the scale-MMA kernel, then the
+    // CUDA-core path.
     if (st.forced_path == 0 || st.forced_path == 2) {
         rc = launch_decode(p, st, s);
         if (rc != LORDS_ERR_UNSUPPORTED && rc != LORDS_ERR_WORKSPACE) return rc;
         if (st.forced_path == 2) return rc;
+    }
+    if (st.forced_path == 0 || st.forced_path == 4) {
+        rc = launch_decode16(p, st, s);
+        if (rc != LORDS_ERR_UNSUPPORTED && rc != LORDS_ERR_WORKSPACE) return rc;
+        if (st.forced_path == 4) return rc;
     }
     if (st.forced_path == 0 || st.forced_path == 3) {
         rc = launch_umma(p, st, s);
@@ -302,6 +308,7 @@ int lords_set_option(const char *key, const char *value)
         else if (std::strcmp(value, "simt") == 0) st.forced_path = 1;
         else if (std::strcmp(value, "decode") == 0) st.forced_path = 2;
         else if (std::strcmp(value, "umma") == 0 || std::strcmp(value, "prefill") == 0) st.forced_path = 3;
+        else if (std::strcmp(value, "decode16") == 0) st.forced_path = 4;
         else return LORDS_ERR_OPTION;
         return LORDS_OK;
     }

@@ -35,7 +35,7 @@ struct State {
     uint8_t *stage_x = nullptr;     // device staging for the host-buffer entry point
     uint8_t *stage_y = nullptr;
     size_t stage_x_bytes = 0, stage_y_bytes = 0;
-    int forced_path = 0;            // 0 auto, 1 simt, 2 decode (reassociated form), 3 umma (scale-MMA form)
+    int forced_path = 0;            // 0 auto, 1 simt, 2 decode (reassociated form), 3 umma (scale-MMA form), 4 decode16
     int forced_splitk = 0;          // 0 auto
     int forced_halves = 0;          // 0 auto; else the tile height of the decode kernel in 128-row halves (1, 2)
     int forced_bn = 0;              // 0 auto; else the token tile of the scale-MMA kernel (32, 64, 128, 256)
@@ -65,5 +65,9 @@ int launch_umma(const Problem &p, State &st, cudaStream_t stream);
 // Tensor-core decode path (M <= 2), reassociated form with the scale factors folded into the
 // activation operand.  LORDS_ERR_UNSUPPORTED for shapes outside its rules.
 int launch_decode(const Problem &p, State &st, cudaStream_t stream);
+
+// Tensor-core decode path for 3 .. 16 tokens, scale-MMA form with 128-column k-steps.
+// LORDS_ERR_UNSUPPORTED for shapes outside its rules.
+int launch_decode16(const Problem &p, State &st, cudaStream_t stream);
 
 }  // namespace lords

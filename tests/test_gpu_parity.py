@@ -159,6 +159,73 @@ def test_decode_kernel_declines_what_it_cannot_run(lords):
         lords.lords_set_option("path", "auto")
 
 
+# ---- the decode kernel for 3 .. 16 tokens (scale-MMA form, 128-column k-steps), forced ----------------
+
+DECODE16_SHAPES = [
+    # bits, m, n, r, M, mixed
+    (4, 384, 1024, 32, 5, True),
+    (4, 512, 4096, 32, 8, False),
+    (4, 300, 1088, 8, 3, True),       # ragged rows; n = 8.5 k-steps; r padded to 16
+    (4, 1000, 2048, 24, 16, True),    # r padded to 32, a full token tile
+    (4, 64, 8192, 16, 7, False),      # one tile, the largest cluster
+    (4, 20000, 128, 16, 4, False),    # more tiles than resident clusters, one k-step each
+    (4, 256, 64, 8, 9, True),         # half a k-step
+    (3, 260, 1152, 48, 16, True),
+    (3, 256, 128, 16, 3, False),
+    (3, 2048, 4096, 32, 8, False),
+]
+
+
+@pytest.mark.parametrize("bits,m,n,r,M,mixed", DECODE16_SHAPES)
+def test_decode16_kernel_shapes(lords, bits, m, n, r, M, mixed):
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=3 * m + n + r + M, mixed_sign=mixed)
+    dl, y32, ybf = _run(lords, lay, "decode16")
+    assert lords.lords_last_path() == "decode16" and lords.lords_last_launch_count() == 1
+    y64 = _oracle(lay, dl.packed_host)
+    check_against_oracle(y32, ybf, y64)
+
+
+@pytest.mark.parametrize("bits,m,n,r,M", [(4, 700, 2048, 32, 8), (4, 256, 512, 16, 16), (3, 384, 1024, 48, 3),
+                                          (3, 131, 384, 7, 9)])
+def test_decode16_kernel_integer_case_is_bit_exact(lords, bits, m, n, r, M):
+    lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m + M)
+    dl, y32, ybf = _run(lords, lay, "decode16")
+    assert lords.lords_last_path() == "decode16"
+    y64 = _oracle(lay, dl.packed_host)
+    assert np.array_equal(y32.astype(np.float64), y64)
+    assert np.array_equal(ybf, oracle.round_bf16(y64))
+
+
+@pytest.mark.parametrize("cluster", [1, 3, 7, 100])
+def test_decode16_kernel_cluster_split_is_deterministic(lords, cluster):
+    lay = gen.make_layer(600, 3072, 32, 6, bits=4, seed=19)
+    lords.lords_set_option("splitk", str(cluster))
+    lords.lords_set_option("path", "decode16")
+    try:
+        dl = DeviceLayer(lay)
+        y32, ybf = dl.forward()
+        y32b, ybfb = dl.forward()
+    finally:
+        lords.lords_set_option("splitk", "0")
+        lords.lords_set_option("path", "auto")
+    assert lords.lords_last_path() == "decode16"
+    assert np.array_equal(y32, y32b) and np.array_equal(ybf, ybfb)
+    check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
+
+
+def test_decode16_kernel_declines_what_it_cannot_run(lords):
+    lords.lords_set_option("path", "decode16")
+    try:
+        for lay in (gen.make_layer(256, 256, 4, 2, bits=4, seed=0),       # two tokens: the other decode kernel's
+                    gen.make_layer(256, 256, 48, 4, bits=4, seed=0),      # 4-bit with r > 32
+                    gen.make_layer(256, 256, 4, 17, bits=4, seed=0)):     # more than one token tile
+            with pytest.raises(lords.LordsError) as ei:
+                DeviceLayer(lay).forward()
+            assert ei.value.status == -11
+    finally:
+        lords.lords_set_option("path", "auto")
+
+
 # ---- the scale-MMA kernel, forced; token tiles forced too so that every instantiation runs ----------
 
 UMMA_SHAPES = [
@@ -265,7 +332,7 @@ def test_config4_stack_shapes_full_size_sampled(lords, name, r, bits, M):
     m, n = gen.LLAMA3_8B_SHAPES[name]
     lay = gen.make_layer(m, n, r, M, bits=bits, seed=7 * len(name) + M)
     dl, y32, ybf = _run(lords, lay, "auto")
-    assert lords.lords_last_path() in ("decode", "umma")
+    assert lords.lords_last_path() in ("decode", "decode16", "umma")
     rows = _sampled_rows(m, 256 if M <= 8 else 64, 11)
     y64 = _oracle(lay, dl.packed_host, rows=rows)
     check_against_oracle(y32[:, rows], ybf[:, rows], y64)
@@ -292,4 +359,4 @@ def test_four_bit_entry_point_and_launch_count(lords):
     torch.cuda.synchronize()
     assert np.array_equal(y.cpu().numpy().view(np.uint16), ybf)
     assert lords.lords_last_launch_count() >= 1
-    assert lords.lords_last_path() in ("simt", "decode", "umma")
+    assert lords.lords_last_path() in ("simt", "decode", "decode16", "umma")
