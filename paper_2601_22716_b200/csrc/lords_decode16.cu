@@ -11,7 +11,7 @@
 // tile, and a thread-block cluster that splits a tile's k-range and adds the partial sums in the
 // leader's shared memory in rank order (deterministic, no atomics).
 //
-// Warp roles (26 warps):
+// Warp roles (27 warps):
 //   0..15  two worker groups of eight warps take k-steps alternately: a warp owns 32 rows and one
 //          64-column half; a thread reads its 64 columns of S from TMEM (as fp16 pairs), looks its code
 //          pairs up in a lane-private fp16x2 level table, multiplies and stores W^ straight into TMEM
@@ -19,11 +19,11 @@
 //   16..19 converters: the activation tile x[16 tokens x 128 columns] arrives as bf16 and is turned
 //          into fp16 in place.
 //   20,21  main-MMA issuers, one per k-step parity.
-//   22     scale-MMA issuer.
-//   23     TMA producer of the packed code tiles; it also initialises the barriers and starts the
+//   22,23  scale-MMA issuers, one per k-step parity (= per S buffer).
+//   24     TMA producer of the packed code tiles; it also initialises the barriers and starts the
 //          weight stream before the rest of the CTA has finished its set-up.
-//   24     TMA producer of the factor tiles A[:, k-step].
-//   25     TMA producer of the activation tiles.
+//   25     TMA producer of the B tile (once) and of the factor tiles A[:, k-step].
+//   26     TMA producer of the activation tiles.
 //
 // Every wait is bounded; on expiry the role records LORDS_ERR_TIMEOUT and leaves its loop, so the
 // kernel always reaches its final barrier and frees its TMEM.
@@ -45,12 +45,12 @@ constexpr int kGroupWarps = 8;
 constexpr int kConvWarp0 = kWorkWarps;                 // 16..19
 constexpr int kConvWarps = 4;
 constexpr int kIssuerWarp0 = kConvWarp0 + kConvWarps;  // 20, 21
-constexpr int kScaleWarp = kIssuerWarp0 + 2;           // 22
-constexpr int kTmaQWarp = kScaleWarp + 1;              // 23
-constexpr int kTmaAWarp = kTmaQWarp + 1;               // 24
-constexpr int kTmaXWarp = kTmaAWarp + 1;               // 25
-constexpr int kWarps = kTmaXWarp + 1;                  // 26
-constexpr int kThreads = kWarps * 32;                  // 832
+constexpr int kScaleWarp0 = kIssuerWarp0 + 2;          // 22, 23
+constexpr int kTmaQWarp = kScaleWarp0 + 2;             // 24
+constexpr int kTmaAWarp = kTmaQWarp + 1;               // 25
+constexpr int kTmaXWarp = kTmaAWarp + 1;               // 26
+constexpr int kWarps = kTmaXWarp + 1;                  // 27
+constexpr int kThreads = kWarps * 32;                  // 864
 constexpr int kRows = 128;                             // W^ rows per CTA = UMMA M
 constexpr int kStep = 128;                             // in-feature columns per k-step
 constexpr int kTok = 16;                               // token tile = UMMA N of the main MMA
@@ -100,7 +100,8 @@ template <int BITS, int RP> struct XCfg {
     static constexpr int kBarMmaDone = kBarReady + WS;     // WS: main MMAs of the k-step done (commit): frees W slot and x tile
     static constexpr int kBarAccFull = kBarMmaDone + WS;   // 2: one per main issuer
     static constexpr int kBarReduce = kBarAccFull + 2;     // 1: counts the bytes of the cluster's partial sums
-    static constexpr int kBarCount = kBarReduce + 1;
+    static constexpr int kBarBFull = kBarReduce + 1;       // 1: 1 arrival + TMA bytes of the B tile
+    static constexpr int kBarCount = kBarBFull + 1;
     static_assert(8 * kBarCount + 8 <= BAR_BYTES, "barrier area");
     static_assert(SQ % 2 == 0 && SD % 2 == 0, "one worker group per barrier of these rings");
 };
@@ -109,6 +110,7 @@ struct alignas(64) Dec16Params {
     CUtensorMap tm_q;     // u8 [m][n*bits/8], box {QROW, 128}
     CUtensorMap tm_a;     // bf16 [r][n], box {64, r_pad}, 128-byte swizzle
     CUtensorMap tm_x;     // bf16 [M][n], box {64, 16}, 128-byte swizzle (rows past M read as zero)
+    CUtensorMap tm_b;     // bf16 [m][r], box {64, 128}, 128-byte swizzle (ranks past r read as zero); used if r % 8 == 0
     const uint16_t *B;    // bf16 [m][r]
     float levels[16];
     int M, m, n, r, r_pad;
@@ -116,7 +118,19 @@ struct alignas(64) Dec16Params {
     void *y;
     int y_f32;
     int *status;
+#ifdef LORDS_TRACE
+    long long *trace;     // [8 roles][32 iterations][8 events] clock64 stamps of one CTA (debug builds only)
+#endif
 };
+
+#ifdef LORDS_TRACE
+#define XSTAMP(role, it, ev)                                                                         \
+    do {                                                                                             \
+        if (blockIdx.x == 0 && (it) < 32) p.trace[((role) * 32 + (it)) * 8 + (ev)] = clock64(); \
+    } while (0)
+#else
+#define XSTAMP(role, it, ev) do { } while (0)
+#endif
 
 __device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float v)
 {
@@ -194,6 +208,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     const uint32_t bar_s_full = bars + 8 * C::kBarSFull, bar_s_empty = bars + 8 * C::kBarSEmpty;
     const uint32_t bar_ready = bars + 8 * C::kBarReady, bar_mma_done = bars + 8 * C::kBarMmaDone;
     const uint32_t bar_acc_full = bars + 8 * C::kBarAccFull, bar_reduce = bars + 8 * C::kBarReduce;
+    const uint32_t bar_b_full = bars + 8 * C::kBarBFull;
+    const bool b_by_tma = (p.r & 7) == 0;      // rows of B are 16-byte multiples: the tile comes by TMA
     const uint32_t tmem_slot = bars + 8 * C::kBarCount;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -207,6 +223,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     const int total = ks_b - ks_a;
 
     bool failed = false;
+    if (tid == 0) XSTAMP(7, 0, 0);
     if (!fits) {
         // the shared-memory window does not hold the layout (cannot happen with the window the host
         // asks for; checked because every address below depends on it)
@@ -241,6 +258,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                 const int sq = it % SQ;
                 if (it >= SQ && !mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1))) { failed = true; break; }
                 const uint32_t bar = bar_q_full + 8 * sq;
+                XSTAMP(3, it, 0);
                 mbar_expect_tx(bar, (uint32_t)C::QSTAGE);
                 tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (ks_a + it) * C::QROW, row0, bar);
             }
@@ -250,7 +268,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             tmem_alloc(tmem_slot, kTmemCols);
             tmem_relinquish();
         } else if (warp == kTmaAWarp) {
-            if (lane == 0) tma_prefetch_desc(&p.tm_a);
+            if (lane == 0) {
+                tma_prefetch_desc(&p.tm_a);
+                if (b_by_tma) tma_prefetch_desc(&p.tm_b);
+            }
         } else if (warp == kTmaXWarp) {
             if (lane == 0) tma_prefetch_desc(&p.tm_x);
         } else if (warp < kWorkWarps) {
@@ -264,8 +285,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                 const __half2 v = __floats2half2_rn(p.levels[lo], p.levels[hi]);
                 sts_u32(lut + (uint32_t)(entry * C::LUT_STRIDE + 4 * lane), *reinterpret_cast<const uint32_t *>(&v));
             }
-            // B tile: 128 rows x 64 ranks (zero padded) bf16, K-major, 128-byte swizzle
-            if (tid < 256) {
+            // B tile: 128 rows x 64 ranks (zero padded) bf16, K-major, 128-byte swizzle: by TMA (below)
+            // or, when a row of B is not a multiple of 16 bytes, element by element here
+            if (!b_by_tma && tid < 256) {
                 const int rr = tid >> 1, half = tid & 1;
                 const int i = row0 + rr;
 #pragma unroll
@@ -298,6 +320,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     } else if (warp == kTmaAWarp) {
         // ------------------------------------------------------------------ factor tiles A[:, k-step] (weights)
         if (lane == 0) {
+            if (b_by_tma) {
+                mbar_expect_tx(bar_b_full, (uint32_t)kBTileBytes);
+                tma_load_2d(b_tile, &p.tm_b, 0, row0, bar_b_full);
+            }
             const uint32_t tx = (uint32_t)(2 * p.r_pad * 128);
             for (int it = 0; it < total; ++it) {
                 const int sa = it % SA;
@@ -315,7 +341,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             // x may be the previous launch's output: everything before this line only touched weights.
             // Nothing of this launch reaches global memory before its main MMAs have run, and those
             // need these tiles, so this one wait orders the whole launch behind the previous one.
+            XSTAMP(6, 0, 3);
             asm volatile("griddepcontrol.wait;" ::: "memory");
+            XSTAMP(6, 0, 4);
             for (int it = 0; it < total; ++it) {
                 const int sx = it % WS;
                 if (it >= WS && !mbar_wait(bar_mma_done + 8 * sx, (uint32_t)((it / WS - 1) & 1))) { failed = true; break; }
@@ -326,33 +354,37 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                     tma_load_2d(x0 + sx * kXStage + at * kXAtom, &p.tm_x, (ks_a + it) * kStep + at * 64, 0, bar);
             }
         }
-    } else if (warp == kScaleWarp) {
-        // ------------------------------------------------------------------ scale-MMA issuer
-        // S of k-step `it` goes into S buffer it % SD as soon as the factor tile has landed and the
-        // workers have read the buffer's previous content.  Two MMAs of N = 64 per 16 ranks, one per
-        // 64-column atom of the factor tile.
+    } else if (warp >= kScaleWarp0) {
+        // ------------------------------------------------------------------ scale-MMA issuers
+        // Issuer j takes the k-steps of parity j, i.e. S buffer j.  S of k-step `it` goes into its
+        // buffer as soon as the factor tile has landed and the workers have read the buffer's previous content.  One MMA of N = 128 per 16 ranks: its B
+        // operand (MN-major) spans the two 64-column atoms of the factor tile, one atom size apart.
         uint32_t tmem_base;
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
-        constexpr uint32_t idesc_s = umma_idesc_f16(1, 0, 1, kRows, 64);     // bf16, B operand MN-major, N = 64
+        constexpr uint32_t idesc_s = umma_idesc_f16(1, 0, 1, kRows, kStep);   // bf16, B operand MN-major, N = 128
         const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
-        const uint32_t lbo_lo = (uint32_t)umma_desc_sw128(0, 1024, 16);
-        const uint32_t b_lo = lbo_lo | ((b_tile & 0x3FFFFu) >> 4);
-        const uint32_t a_lo0 = lbo_lo | ((a0 & 0x3FFFFu) >> 4);
+        const uint32_t b_lo = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((b_tile & 0x3FFFFu) >> 4);
+        const uint32_t a_lo0 = (uint32_t)umma_desc_sw128(0, 1024, (uint32_t)C::AATOM) | ((a0 & 0x3FFFFu) >> 4);
         const int rsteps = p.r_pad / 16;
-        for (int it = 0; it < total; ++it) {
+        const int sj = warp - kScaleWarp0;
+        static_assert(SD == 2 && SA % 2 == 0, "one scale issuer per S buffer; each factor-ring barrier belongs to one of them");
+        if (b_by_tma && sj < total && !mbar_wait(bar_b_full, 0)) failed = true;
+        for (int it = sj; it < total && !failed; it += 2) {
             const int sa = it % SA, sd = it % SD;
+            if (lane == 0) XSTAMP(4, it, 0);
             if (!mbar_wait(bar_a_full + 8 * sa, (uint32_t)((it / SA) & 1))) { failed = true; break; }
+            if (lane == 0) XSTAMP(4, it, 1);
             if (it >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((it / SD - 1) & 1))) { failed = true; break; }
             tc_fence_after_sync();
+            if (lane == 0) XSTAMP(4, it, 2);
             if (lane == 0) {
                 const uint32_t a_lo = a_lo0 + (uint32_t)(sa * (C::ASTAGE >> 4));
-#pragma unroll
-                for (int at = 0; at < 2; ++at)
-                    for (int k = 0; k < rsteps; ++k)
-                        umma_f16_ss(tmem_base + kSCol + (uint32_t)(sd * kStep + at * 64), umma_desc_pack(b_lo + k * 2, desc_hi),
-                                    umma_desc_pack(a_lo + at * (C::AATOM >> 4) + k * 128, desc_hi), idesc_s, k > 0);
+                for (int k = 0; k < rsteps; ++k)
+                    umma_f16_ss(tmem_base + kSCol + (uint32_t)(sd * kStep), umma_desc_pack(b_lo + k * 2, desc_hi),
+                                umma_desc_pack(a_lo + k * 128, desc_hi), idesc_s, k > 0);
                 umma_commit(bar_s_full + 8 * sd);
                 umma_commit(bar_a_done + 8 * sa);
+                XSTAMP(4, it, 3);
             }
             __syncwarp();
         }
@@ -369,9 +401,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         const uint32_t acc = tmem_base + (uint32_t)(j * 32);
         for (int it = j; it < total; it += 2) {
             const int ws = it % WS;
+            if (j == 0 && lane == 0) XSTAMP(0, it, 0);
             if (!mbar_wait(bar_x_ready + 8 * ws, (uint32_t)((it / WS) & 1)) ||
                 !mbar_wait(bar_ready + 8 * ws, (uint32_t)((it / WS) & 1))) { failed = true; break; }
             tc_fence_after_sync();
+            if (j == 0 && lane == 0) XSTAMP(0, it, 1);
             if (lane == 0) {
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)(ws * 64);
                 const uint32_t x_lo = x_lo0 + (uint32_t)(ws * (kXStage >> 4));
@@ -381,6 +415,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                                 idesc_m, (it == j && k == 0) ? 0u : 1u);
                 umma_commit(bar_mma_done + 8 * ws);
                 if (it + 2 >= total) umma_commit(bar_acc_full + 8 * j);
+                if (j == 0) XSTAMP(0, it, 2);
             }
             __syncwarp();
         }
@@ -419,10 +454,13 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         const uint32_t lut_lane = lut + 4u * (uint32_t)lane;
 
+        const bool stamper = wg == 0 && lane == 0;
         for (int it = g; it < total; it += 2) {
             const int sq = it % SQ, sd = it % SD, ws = it % WS;
+            if (stamper) XSTAMP(1 + g, it, 0);
             if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * sd, (uint32_t)((it / SD) & 1)))) { failed = true; break; }
             tc_fence_after_sync();
+            if (stamper) XSTAMP(1 + g, it, 1);
             // this thread's 64 columns of S, as 32 fp16 pairs
             uint32_t sp[32];
 #pragma unroll
@@ -439,11 +477,14 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s_empty + 8 * sd);      // S is in registers: the buffer may be refilled
+            if (stamper) XSTAMP(1 + g, it, 2);
             if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1)))) { failed = true; break; }
+            if (stamper) XSTAMP(1 + g, it, 3);
             dequant_half_row<BITS>(q0 + sq * C::QSTAGE + row * C::QROW, row, ch, lut_lane, sp);
             // the W slot is free once the MMAs of step it - WS have completed
             if (it >= WS && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * ws, (uint32_t)((it / WS - 1) & 1)))) { failed = true; break; }
             tc_fence_after_sync();
+            if (stamper) XSTAMP(1 + g, it, 4);
             tmem_st_32x32(lane_addr + kWCol + (uint32_t)(ws * 64 + ch * 32), sp);
             tmem_wait_st();
             tc_fence_before_sync();
@@ -452,6 +493,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                 mbar_arrive(bar_ready + 8 * ws);
                 mbar_arrive(bar_q_empty + 8 * sq);
             }
+            if (stamper) XSTAMP(1 + g, it, 5);
         }
 
         // Epilogue (group 0, column half 0: one thread per row): the two accumulators -> this CTA's
@@ -464,6 +506,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
 #pragma unroll
             for (int t = 0; t < kTok; ++t) yt[t] = 0.0f;
             bool ok = true;
+            if (stamper) XSTAMP(5, 0, 0);
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 if (ok && j < total) {       // issuer j had a k-step
@@ -483,6 +526,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
 #pragma unroll
                 for (int t = 0; t < kTok; ++t) yt[t] = 0.0f;
             }
+            if (stamper) XSTAMP(5, 0, 1);
             if (csize == 1) {
                 if (ok && i < p.m)
 #pragma unroll
@@ -494,26 +538,35 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
 #pragma unroll
                 for (int t = 0; t < kTok; ++t)
                     st_async_cluster_f32(map_to_rank(red0 + (uint32_t)(((rank * kTok + t) * kRows + row) * 4), 0), yt[t], leader_bar);
+                if (stamper) XSTAMP(5, 0, 2);
                 if (rank == 0) {
-                    if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0))) failed = true;
+                    const bool got = __all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0));
+                    if (stamper) XSTAMP(5, 0, 3);
+                    if (!got) failed = true;
                     else if (i < p.m) {
-#pragma unroll 1
-                        for (int t = 0; t < kTok; ++t) {
-                            if (t >= p.M) break;
-                            float a = 0.0f;
-                            for (int rr = 0; rr < csize; ++rr)
-                                a += __uint_as_float(lds_u32(red0 + (uint32_t)(((rr * kTok + t) * kRows + row) * 4)));
-                            store_out(p.y, p.y_f32, (size_t)t * p.m + i, a);
-                        }
+                        // rank order for every token; the sixteen sums run side by side
+                        float a[kTok];
+#pragma unroll
+                        for (int t = 0; t < kTok; ++t) a[t] = 0.0f;
+                        for (int rr = 0; rr < csize; ++rr)
+#pragma unroll
+                            for (int t = 0; t < kTok; ++t)
+                                a[t] += __uint_as_float(lds_u32(red0 + (uint32_t)(((rr * kTok + t) * kRows + row) * 4)));
+#pragma unroll
+                        for (int t = 0; t < kTok; ++t)
+                            if (t < p.M) store_out(p.y, p.y_f32, (size_t)t * p.m + i, a[t]);
                     }
+                    if (stamper) XSTAMP(5, 0, 4);
                 }
             }
         }
     }
 
+    if (tid == 0) XSTAMP(7, 0, 1);
     if (failed) atomicExch(p.status, LORDS_ERR_TIMEOUT);
     tc_fence_before_sync();
     __syncthreads();
+    if (tid == 0) XSTAMP(7, 0, 2);
     if (warp == kIssuerWarp0) {
         tc_fence_after_sync();
         uint32_t tmem_base;
@@ -624,6 +677,13 @@ template <int BITS, int RP> int launch_variant(Dec16Params &k, const Problem &p,
         !make_map_2d(&k.tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.x, (uint64_t)p.n, (uint64_t)p.M, 64, (uint32_t)kTok,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return LORDS_ERR_CUDA;
+    if ((p.r & 7) == 0) {
+        if (!make_map_2d(&k.tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.B, (uint64_t)p.r, (uint64_t)p.m, 64, (uint32_t)kRows,
+                         CU_TENSOR_MAP_SWIZZLE_128B))
+            return LORDS_ERR_CUDA;
+    } else {
+        k.tm_b = k.tm_a;      // not used: the kernel builds the B tile element by element
+    }
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
     V::fill(cfg, attr, cs, tiles, stream);
@@ -652,6 +712,10 @@ int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
     k.ksteps = (p.n + kStep - 1) / kStep;
     k.y = p.y; k.y_f32 = p.y_f32;
     k.status = st.status_word;
+#ifdef LORDS_TRACE
+    k.trace = reinterpret_cast<long long *>(st.workspace + st.workspace_bytes - (size_t)8 * 32 * 8 * 8);
+    LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)8 * 32 * 8 * 8, stream));
+#endif
     int rc;
     if (p.bits == 4) rc = launch_variant<4, 32>(k, p, st.forced_splitk, stream);
     else rc = k.r_pad <= 32 ? launch_variant<3, 32>(k, p, st.forced_splitk, stream) : launch_variant<3, 64>(k, p, st.forced_splitk, stream);
