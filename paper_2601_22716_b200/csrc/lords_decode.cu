@@ -547,11 +547,18 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 if (rank == 0) {
                     if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0))) failed = true;
                     else if (i < p.m) {
+                        // all partials are read first (the loads overlap), then added in rank order
+                        float v[NTOK][kClusterMax];
+#pragma unroll
+                        for (int t = 0; t < NTOK; ++t)
+#pragma unroll
+                            for (int rr = 0; rr < kClusterMax; ++rr)
+                                v[t][rr] = rr < csize ? __uint_as_float(lds_u32(red0 + ((rr * NTOK + t) * kTileRows + row_in_tile) * 4)) : 0.0f;
 #pragma unroll
                         for (int t = 0; t < NTOK; ++t) {
                             float a = 0.0f;
-                            for (int rr = 0; rr < csize; ++rr)
-                                a += __uint_as_float(lds_u32(red0 + ((rr * NTOK + t) * kTileRows + row_in_tile) * 4));
+#pragma unroll
+                            for (int rr = 0; rr < kClusterMax; ++rr) a += v[t][rr];
                             store_out(p.y, p.y_f32, (size_t)t * p.m + i, a);
                         }
                     }
