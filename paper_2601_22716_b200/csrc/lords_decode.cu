@@ -578,6 +578,13 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         tmem_dealloc(tmem_base, kTmemCols);
     }
+    // No CTA of the cluster leaves before the leader has received every partial sum: the asynchronous
+    // stores of a CTA must not be in flight when it exits (with programmatic dependent launch a CTA
+    // of the next launch can take over the SM at once).
+    if (csize > 1) {
+        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,

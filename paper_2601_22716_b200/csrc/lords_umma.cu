@@ -538,6 +538,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         tmem_dealloc(tmem_base, kTmemCols);
     }
+    // BN == 16 with a split k-range: no CTA of the cluster leaves before the leader has received
+    // every partial sum (the asynchronous stores of a CTA must not be in flight when it exits)
+    if (BN == 16 && csize > 1) {
+        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
 }
 
 // x bf16 -> fp16 (exact for every bf16 value inside fp16's normal range), 8 elements per thread.
