@@ -186,14 +186,15 @@ int lords_last_cuda_error(void);
 
 /*
  * Measurement switches.  Keys: "path" = "auto" | "simt" | "decode" (reassociated-form kernel,
- * M <= 2) | "umma" (scale-MMA kernel; "prefill" is an alias);
+ * M <= 2) | "decode16" (scale-MMA form with 128-column k-steps, 3 <= M <= 16) | "umma" (scale-MMA
+ * kernel for any M; "prefill" is an alias);
  * "splitk" = "0" (auto) or a positive integer (CTAs sharing one tile's k-range); "bn" = "0" (auto)
  * or the token tile 32, 64, 128, 256 of the scale-MMA kernel for M > 16; "halves" = "0" (auto), "1"
  * or "2": tile height of the decode kernel in 128-row halves.  Unknown keys: LORDS_ERR_OPTION.
  */
 int lords_set_option(const char *key, const char *value);
 
-/* Name of the path the most recent forward call dispatched to ("simt", "decode", "umma"). */
+/* Name of the path the most recent forward call dispatched to ("simt", "decode", "decode16", "umma"). */
 const char *lords_last_path(void);
 
 /* Number of kernels the most recent forward call launched. */
