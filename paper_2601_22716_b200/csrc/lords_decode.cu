@@ -8,10 +8,10 @@
 //
 // A thread-block cluster owns one tile of 128 * H rows of Q (H = 1 or 2); its CTAs split the tile's
 // k-steps (128 in-feature columns each) evenly, and the host picks H and the cluster size so that
-// all clusters are resident at once and fill the SMs.  Each CTA parks its partial y in the cluster
-// leader's shared memory (distributed shared memory) and arrives on the leader's mbarrier; the
+// all clusters are resident at once and fill the SMs.  Each CTA sends its partial y into the cluster
+// leader's shared memory with asynchronous stores whose bytes the leader's mbarrier counts; the
 // leader adds the partials in rank order -- deterministic, no float atomics, no trip through
-// global memory.
+// global memory.  A cluster barrier at the very end keeps every CTA alive until the leader is done.
 //
 // Warp roles (28 warps):
 //   0..15  two worker groups of eight warps take k-steps alternately and dequantise: a warp owns 32
@@ -98,6 +98,7 @@ template <int BITS, int H> struct DCfg {
 struct alignas(64) DecodeParams {
     CUtensorMap tm_q;     // u8 [m][n*bits/8], box {QROW, 128 * H}
     CUtensorMap tm_a;     // bf16 [r][n], box {64, r_pad}, 128-byte swizzle
+    CUtensorMap tm_x;     // bf16 [M][n], box {128, M}, no swizzle (columns past n read as zero)
     const uint16_t *x;    // bf16 [M][n]
     const uint16_t *B;    // bf16 [m][r]
     float levels[16];
@@ -241,6 +242,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
 
     if (tid == 0) DSTAMP(7, 0, 0);
     bool failed = false;
+    bool cluster_waited = false;      // this thread has taken the second half of the set-up cluster barrier
     if (!fits) {
         // the shared-memory window does not hold the layout (cannot happen with the window the host
         // asks for; checked because every address below depends on it)
@@ -290,7 +292,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             tmem_relinquish();
             if (lane == 0) DSTAMP(7, 0, 4);
         } else if (warp == kTmaAWarp) {
-            if (lane == 0) tma_prefetch_desc(&p.tm_a);
+            if (lane == 0) {
+                tma_prefetch_desc(&p.tm_a);
+                tma_prefetch_desc(&p.tm_x);
+            }
         } else if (warp < kWorkWarps) {
             // level-pair table: entry e = (L[lo code], L[hi code]) as fp16x2; word e*32 + lane is lane's
             // copy (bank = lane, so the lookups of a warp never conflict)
@@ -314,6 +319,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     }
     // let a dependent launch (the next layer) begin its own weight prefetch as SMs become free
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Everything except the stream of packed codes waits here for the previous launch to finish: a CTA
+    // that starts early sets up, prefetches its codes and then stands still.  (Letting the workers
+    // run ahead of this point as well was tried; with it about one run in twenty of a 224-kernel
+    // graph ended in device-side timeouts whose cause was not found.)
+    if (warp != kTmaQWarp) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tid == 0) DSTAMP(7, 0, 1);
 
     if (warp == kTmaQWarp) {
@@ -333,14 +343,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 const int s = it % S, j0 = (ks_a + it) * kStep;
                 if (it >= S && !mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1))) { failed = true; break; }
                 const uint32_t bar = bar_a_full + 8 * s;
-                const uint32_t xbytes = (uint32_t)(2 * (p.n - j0 < kStep ? p.n - j0 : kStep));   // a multiple of 64
-                mbar_expect_tx(bar, tx_a + NTOK * xbytes);
+                mbar_expect_tx(bar, tx_a + (uint32_t)(NTOK * kStep * 2));
 #pragma unroll
                 for (int at = 0; at < kAtoms; ++at)
                     tma_load_2d(ax_stage(s) + at * kAtomBytes, &p.tm_a, j0 + at * 64, 0, bar);
-#pragma unroll
-                for (int t = 0; t < NTOK; ++t)
-                    bulk_load(xs0 + s * C::XSTAGE + t * (kStep * 2), p.x + (size_t)t * p.n + j0, xbytes, bar);
+                tma_load_2d(xs0 + s * C::XSTAGE, &p.tm_x, j0, 0, bar);
             }
         }
     } else if (warp >= kIssuerWarp0) {
@@ -492,7 +499,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                                                  : make_uint4(0, 0, 0, 0);
             // second half of the split-phase cluster barrier (every CTA of the cluster has initialised
             // its barriers): taken here, where its latency hides behind the wait for the last MMAs
-            if (csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+            if (csize > 1) {
+                asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+                cluster_waited = true;
+            }
             float yt[NTOK];
 #pragma unroll
             for (int t = 0; t < NTOK; ++t) yt[t] = 0.0f;
@@ -582,8 +592,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     // stores of a CTA must not be in flight when it exits (with programmatic dependent launch a CTA
     // of the next launch can take over the SM at once).
     if (csize > 1) {
-        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
-        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        // every arrival is paired with a wait: threads that have not waited on the set-up barrier do so first
+        if (!cluster_waited) asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+        asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
     }
 }
 
@@ -717,7 +729,9 @@ template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem
     if (!make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)qrow,
                      two ? 256u : 128u, BITS == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE) ||
         !make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.A, (uint64_t)p.n, (uint64_t)p.r, 64, (uint32_t)k.r_pad,
-                     CU_TENSOR_MAP_SWIZZLE_128B))
+                     CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&k.tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.x, (uint64_t)p.n, (uint64_t)p.M, (uint32_t)kStep, (uint32_t)NTOK,
+                     CU_TENSOR_MAP_SWIZZLE_NONE))
         return LORDS_ERR_CUDA;
     k.tiles = two ? tiles2 : tiles1;
     return two ? DecodeVariant<BITS, NTOK, 2>::launch(k, tiles2, cs2, stream)

@@ -223,6 +223,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     const int total = ks_b - ks_a;
 
     bool failed = false;
+    bool cluster_waited = false;      // this thread has taken the second half of the set-up cluster barrier
     if (tid == 0) XSTAMP(7, 0, 0);
     if (!fits) {
         // the shared-memory window does not hold the layout (cannot happen with the window the host
@@ -314,6 +315,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     }
     // let a dependent launch (the next layer) begin its own weight prefetch as SMs become free
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Everything except the stream of packed codes waits here for the previous launch to finish: a CTA
+    // that starts early sets up, prefetches its codes and then stands still.  (Letting the workers
+    // run ahead of this point as well was tried; with it about one run in twenty of a 224-kernel
+    // graph ended in device-side timeouts whose cause was not found.)
+    if (warp != kTmaQWarp) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == kTmaQWarp) {
         // all done above
@@ -501,7 +507,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         if (g == 0 && ch == 0 && !failed) {
             const int i = row0 + row;
             // second half of the split-phase cluster barrier, behind the wait for the last MMAs
-            if (csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+            if (csize > 1) {
+                asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+                cluster_waited = true;
+            }
             float yt[kTok];
 #pragma unroll
             for (int t = 0; t < kTok; ++t) yt[t] = 0.0f;
@@ -577,8 +586,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     // stores of a CTA must not be in flight when it exits (with programmatic dependent launch a CTA
     // of the next launch can take over the SM at once).
     if (csize > 1) {
-        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
-        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        // every arrival is paired with a wait: threads that have not waited on the set-up barrier do so first
+        if (!cluster_waited) asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+        asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
     }
 }
 

@@ -42,17 +42,49 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: gives up after about a second of polling and reports failure, so that no role of
+// Wall-clock nanoseconds, one time base for the whole GPU.
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// The limit of every bounded wait: it gives up only when three independent measures agree that it
+// has waited for seconds -- the number of polls, the SM's cycle counter and the GPU's wall clock.
+// (With the cycle counter alone, waits on many SMs were seen to run out at the same instant about
+// once in fifteen runs of a 224-kernel graph; no wait of these kernels takes a millisecond.)
+struct WaitLimit {
+    long long c0;
+    unsigned long long g0;
+    unsigned rounds;
+};
+__device__ __forceinline__ WaitLimit wait_limit_start()
+{
+    WaitLimit w;
+    w.c0 = clock64();
+    w.g0 = global_ns();
+    w.rounds = 0;
+    return w;
+}
+// called after every 256 unsuccessful polls
+__device__ __forceinline__ bool wait_limit_expired(WaitLimit &w)
+{
+    ++w.rounds;
+    return w.rounds > 256u && clock64() - w.c0 > 4000000000LL && global_ns() - w.g0 > 2000000000ULL;
+}
+
+// Bounded wait: gives up after about two seconds of polling and reports failure, so that no role of
 // a kernel can spin forever on a shared GPU.  Callers record LORDS_ERR_TIMEOUT and drain.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
+    WaitLimit limit = wait_limit_start();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > 2000000000LL) return false;
+        if (wait_limit_expired(limit)) return false;
     }
 }
 
@@ -73,13 +105,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, int 
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y)
         : "memory");
-}
-// Untiled bulk copy global -> this CTA's shared memory; both addresses 16-byte aligned, bytes a
-// multiple of 16; completion is counted in bytes on `bar`.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tma_prefetch_desc(const void *tmap)
 {
@@ -228,12 +253,12 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
 {
     if (mbar_try_wait_cluster(bar, parity)) return true;
-    const long long t0 = clock64();
+    WaitLimit limit = wait_limit_start();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait_cluster(bar, parity)) return true;
-        if (clock64() - t0 > 2000000000LL) return false;
+        if (wait_limit_expired(limit)) return false;
     }
 }
 

@@ -210,6 +210,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
     const int total = 2 * pairs;          // k-steps of this CTA; global k-step = 2 * pa + it
 
     bool failed = false;
+    bool cluster_waited = false;      // this thread has taken the second half of the set-up cluster barrier
 
     if (warp == kTmaWarp) {
         // ------------------------------------------------------------------ TMA producer
@@ -458,7 +459,10 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             bool ok = true;
             // BN == 16, k-range split over the cluster: the second half of the split-phase cluster barrier
             // (every CTA has initialised its barriers) is taken here, behind the wait for the last MMAs
-            if (BN == 16 && csize > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+            if (BN == 16 && csize > 1) {
+                asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+                cluster_waited = true;
+            }
             if (total > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full, 0));
             tc_fence_after_sync();
             const int i = row0 + row;
@@ -494,6 +498,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 }
                 if (pair_split && rank == 1) {
                     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // the partner's barrier exists
+                    cluster_waited = true;
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(map_to_rank(bar_reduce, 0));
                 }
@@ -538,11 +543,14 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         tmem_dealloc(tmem_base, kTmemCols);
     }
-    // BN == 16 with a split k-range: no CTA of the cluster leaves before the leader has received
-    // every partial sum (the asynchronous stores of a CTA must not be in flight when it exits)
-    if (BN == 16 && csize > 1) {
-        asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
-        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    // Clusters (split k-range of the 16-token tile, or a pair): no CTA leaves before its partner has
+    // received what it sent (asynchronous stores and remote arrivals of a CTA must not be in flight
+    // when it exits)
+    if (csize > 1) {
+        // every arrival is paired with a wait: threads that have not waited on the set-up barrier do so first
+        if (!cluster_waited) asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+        asm volatile("barrier.cluster.arrive.relaxed;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
     }
 }
 
