@@ -25,7 +25,7 @@
 //          memory, eight per k-step; one issuer per 128-row half (H = 2) or per k-step parity (H = 1).
 //   26     TMA producer of the packed code tiles (HBM stream, deep ring); it also initialises the
 //          barriers and starts the stream before the rest of the CTA has finished its set-up.
-//   27     TMA producer of the factor tiles and of the k-step's slice of x.
+//   27     TMA producer of the factor tiles and of the k-step's slice of x (two tensor maps, one barrier).
 //
 // Every wait is bounded; on expiry the role records LORDS_ERR_TIMEOUT and leaves its loop, so
 // the kernel always reaches its final barrier and frees its TMEM.
@@ -331,10 +331,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     } else if (warp == kTmaAWarp) {
         // ------------------------------------------------------------------ factor tiles A[:, k-step] and x[:, k-step]
         if (lane == 0) {
-            // x may be the previous launch's output: everything before this line only touched weights.
-            // Nothing of this launch reaches global memory before its MMAs have run, and those need
-            // the B operand made from these loads, so this one wait orders the whole launch behind
-            // the previous one.
+            // x may be the previous launch's output.  (This warp has already waited above with the
+            // others; the wait is repeated where the dependency is.)
             DSTAMP(6, 0, 3);
             asm volatile("griddepcontrol.wait;" ::: "memory");
             DSTAMP(6, 0, 4);

@@ -344,9 +344,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     } else if (warp == kTmaXWarp) {
         // ------------------------------------------------------------------ activation tiles x[:, k-step]
         if (lane == 0) {
-            // x may be the previous launch's output: everything before this line only touched weights.
-            // Nothing of this launch reaches global memory before its main MMAs have run, and those
-            // need these tiles, so this one wait orders the whole launch behind the previous one.
+            // x may be the previous launch's output.  (This warp has already waited above with the
+            // others; the wait is repeated where the dependency is.)
             XSTAMP(6, 0, 3);
             asm volatile("griddepcontrol.wait;" ::: "memory");
             XSTAMP(6, 0, 4);
