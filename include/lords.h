@@ -189,8 +189,7 @@ int lords_last_cuda_error(void);
  * M <= 2) | "decode16" (scale-MMA form with 128-column k-steps, 3 <= M <= 16) | "umma" (scale-MMA
  * kernel for any M; "prefill" is an alias);
  * "splitk" = "0" (auto) or a positive integer (CTAs sharing one tile's k-range); "bn" = "0" (auto)
- * or the token tile 32, 64, 128, 256 of the scale-MMA kernel for M > 16; "halves" = "0" (auto), "1"
- * or "2": tile height of the decode kernel in 128-row halves.  Unknown keys: LORDS_ERR_OPTION.
+ * or the token tile 32, 64, 128, 256 of the scale-MMA kernel for M > 16.  Unknown keys: LORDS_ERR_OPTION.
  */
 int lords_set_option(const char *key, const char *value);
 

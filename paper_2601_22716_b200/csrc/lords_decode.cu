@@ -37,6 +37,7 @@
 
 #include "lords_internal.h"
 #include "lords_ptx.cuh"
+#include "lords_tc_common.cuh"
 
 namespace lords {
 
@@ -108,28 +109,7 @@ struct alignas(64) DecodeParams {
     void *y;
     int y_f32;
     int *status;
-#ifdef LORDS_TRACE
-    long long *trace;     // [8 roles][32 iterations][8 events] clock64 stamps of one CTA (debug builds only)
-#endif
 };
-
-#ifdef LORDS_TRACE
-#ifndef LORDS_TRACE_CTA
-#define LORDS_TRACE_CTA 0
-#endif
-#define DSTAMP(role, it, ev)                                                                         \
-    do {                                                                                             \
-        if (blockIdx.x == LORDS_TRACE_CTA && (it) < 32) p.trace[((role) * 32 + (it)) * 8 + (ev)] = clock64(); \
-    } while (0)
-#else
-#define DSTAMP(role, it, ev) do { } while (0)
-#endif
-
-__device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float v)
-{
-    if (y_f32) static_cast<float *>(y)[idx] = v;
-    else static_cast<__nv_bfloat16 *>(y)[idx] = __float2bfloat16_rn(v);
-}
 
 // One row of one k-step (128 codes): packed codes (shared memory) -> fp16 level pairs -> 64 TMEM columns.
 // 4-bit rows are 64 bytes and arrive 64-byte-swizzled (16-byte chunk c of row i sits at chunk
@@ -239,8 +219,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     const int ks_b = (rank + 1) * p.ksteps / csize;
     const int total = ks_b - ks_a;
     const int N = NTOK * p.r_pad;
+    const int *status = p.status;
 
-    if (tid == 0) DSTAMP(7, 0, 0);
     bool failed = false;
     bool cluster_waited = false;      // this thread has taken the second half of the set-up cluster barrier
     if (!fits) {
@@ -250,7 +230,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         return;
     }
 
-    if (warp == kTmaQWarp && lane == 0) DSTAMP(6, 0, 0);
     if (warp == kTmaQWarp) {
         // ------------------------------------------------------------------ code tiles (HBM stream)
         // This warp initialises every barrier, releases the rest of the CTA and starts the stream of
@@ -275,13 +254,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         // right before the first access to the leader's shared memory
         asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
         if (lane == 0) {
-            DSTAMP(7, 0, 3);
             tma_prefetch_desc(&p.tm_q);
             for (int it = 0; it < total; ++it) {
                 const int sq = it % SQ;
-                if (it >= SQ && !mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1))) { failed = true; break; }
+                if (it >= SQ && !mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1), status)) { failed = true; break; }
                 const uint32_t bar = bar_q_full + 8 * sq;
-                DSTAMP(3, it, 0);
                 mbar_expect_tx(bar, (uint32_t)C::QSTAGE);
                 tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (ks_a + it) * C::QROW, tile * kTileRows, bar);
             }
@@ -290,7 +267,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         if (warp == kIssuerWarp0) {
             tmem_alloc(tmem_slot, kTmemCols);
             tmem_relinquish();
-            if (lane == 0) DSTAMP(7, 0, 4);
         } else if (warp == kTmaAWarp) {
             if (lane == 0) {
                 tma_prefetch_desc(&p.tm_a);
@@ -308,44 +284,47 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 const __half2 v = __floats2half2_rn(p.levels[lo], p.levels[hi]);
                 sts_u32(lut + (uint32_t)(entry * C::LUT_STRIDE + 4 * lane), *reinterpret_cast<const uint32_t *>(&v));
             }
-            if (tid == 0) DSTAMP(7, 0, 5);
         }
         tc_fence_before_sync();
-        if (tid == 0) DSTAMP(6, 0, 1);
         asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");   // table, TMEM address and barriers are in place
         tc_fence_after_sync();
-        if (tid == 0) DSTAMP(6, 0, 2);
         asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");   // see above
     }
     // let a dependent launch (the next layer) begin its own weight prefetch as SMs become free
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    // Everything except the stream of packed codes waits here for the previous launch to finish: a CTA
-    // that starts early sets up, prefetches its codes and then stands still.  (Letting the workers
-    // run ahead of this point as well was tried; with it about one run in twenty of a 224-kernel
-    // graph ended in device-side timeouts whose cause was not found.)
-    if (warp != kTmaQWarp) asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (tid == 0) DSTAMP(7, 0, 1);
+    griddep_launch_dependents();
+    // Everything except the two streams of weights (packed codes, first factor tiles) waits here for
+    // the previous launch to finish: a CTA that starts early sets up, prefetches and then stands still,
+    // so every bounded wait below begins behind the dependency point.
+    if (warp != kTmaQWarp && warp != kTmaAWarp) griddep_wait();
 
     if (warp == kTmaQWarp) {
         // all done above
     } else if (warp == kTmaAWarp) {
         // ------------------------------------------------------------------ factor tiles A[:, k-step] and x[:, k-step]
         if (lane == 0) {
-            // x may be the previous launch's output.  (This warp has already waited above with the
-            // others; the wait is repeated where the dependency is.)
-            DSTAMP(6, 0, 3);
-            asm volatile("griddepcontrol.wait;" ::: "memory");
-            DSTAMP(6, 0, 4);
             const uint32_t tx_a = (uint32_t)(kAtoms * p.r_pad * 128);
-            for (int it = 0; it < total; ++it) {
+            // one barrier per stage counts the bytes of the factor tile and of the x slice
+            auto load_a = [&](int it) {
                 const int s = it % S, j0 = (ks_a + it) * kStep;
-                if (it >= S && !mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1))) { failed = true; break; }
                 const uint32_t bar = bar_a_full + 8 * s;
                 mbar_expect_tx(bar, tx_a + (uint32_t)(NTOK * kStep * 2));
 #pragma unroll
                 for (int at = 0; at < kAtoms; ++at)
                     tma_load_2d(ax_stage(s) + at * kAtomBytes, &p.tm_a, j0 + at * 64, 0, bar);
-                tma_load_2d(xs0 + s * C::XSTAGE, &p.tm_x, j0, 0, bar);
+            };
+            auto load_x = [&](int it) {
+                const int s = it % S;
+                tma_load_2d(xs0 + s * C::XSTAGE, &p.tm_x, (ks_a + it) * kStep, 0, bar_a_full + 8 * s);
+            };
+            // the factors are weights: the first stages are filled before the dependency point
+            const int pre = total < S ? total : S;
+            for (int it = 0; it < pre; ++it) load_a(it);
+            griddep_wait();   // x may be the previous launch's output
+            for (int it = 0; it < pre; ++it) load_x(it);
+            for (int it = S; it < total; ++it) {
+                if (!mbar_wait(bar_mma_done + 8 * (it % S), (uint32_t)((it / S - 1) & 1), status)) { failed = true; break; }
+                load_a(it);
+                load_x(it);
             }
         }
     } else if (warp >= kIssuerWarp0) {
@@ -366,11 +345,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         const int first = H == 2 ? 0 : j;
         for (int it = first; it < total; it += kStride) {
             const int s = it % S;
-            if (j == 0 && lane == 0) DSTAMP(0, it, 0);
-            if (!mbar_wait(bar_ax_ready + 8 * s, (uint32_t)((it / S) & 1)) ||
-                !mbar_wait(bar_ready + 8 * (h * S + s), (uint32_t)((it / S) & 1))) { failed = true; break; }
+            if (!mbar_wait(bar_ax_ready + 8 * s, (uint32_t)((it / S) & 1), status) ||
+                !mbar_wait(bar_ready + 8 * (h * S + s), (uint32_t)((it / S) & 1), status)) { failed = true; break; }
             tc_fence_after_sync();
-            if (j == 0 && lane == 0) DSTAMP(0, it, 1);
             if (lane == 0) {
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)((h * S + s) * kWSlotCols);
                 const uint32_t b_lo = desc_lo | ((ax_stage(s) & 0x3FFFFu) >> 4);
@@ -380,7 +357,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                                 idesc, (it == first && k == 0) ? 0u : 1u);
                 umma_commit(bar_mma_done + 8 * s);
                 if (it + kStride >= total) umma_commit(bar_acc_full + 8 * j);
-                if (j == 0) DSTAMP(0, it, 2);
             }
             __syncwarp();
         }
@@ -392,12 +368,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         const int c16 = lane & 7, rsub = cw * 4 + (lane >> 3);
         constexpr int kRowStep = 4 * kConvGroupWarps;          // 16
         constexpr int kRowIters = kNMax / kRowStep;            // 4
-        const bool cstamper = cw == 0 && lane == 0 && cgp == 0;
         for (int it = cgp; it < total; it += kConvGroups) {
             const int s = it % S;
-            if (cstamper) DSTAMP(4, it, 0);
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full + 8 * s, (uint32_t)((it / S) & 1)))) { failed = true; break; }
-            if (cstamper) DSTAMP(4, it, 1);
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full + 8 * s, (uint32_t)((it / S) & 1), status))) { failed = true; break; }
 #pragma unroll
             for (int at = 0; at < kAtoms; ++at) {
                 const uint32_t atom = ax_stage(s) + at * kAtomBytes;
@@ -410,9 +383,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 float xf[NTOK][8];
 #pragma unroll
                 for (int t = 0; t < NTOK; ++t) {
-                    // columns past n hold nothing the copy wrote: take zero there
-                    const bool in = (ks_a + it) * kStep + at * 64 + c16 * 8 < p.n;
-                    const uint4 xv = in ? lds_v4(xs0 + s * C::XSTAGE + t * (kStep * 2) + at * 128 + c16 * 16) : make_uint4(0, 0, 0, 0);
+                    // columns past n were filled with zeros by the tensor-map copy
+                    const uint4 xv = lds_v4(xs0 + s * C::XSTAGE + t * (kStep * 2) + at * 128 + c16 * 16);
                     const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
@@ -444,7 +416,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_ax_ready + 8 * s);
-            if (cstamper) DSTAMP(4, it, 2);
         }
     } else {
         // ------------------------------------------------------------------ worker warps
@@ -457,44 +428,52 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         const uint32_t lut_lane = lut + 4u * (uint32_t)lane;
-        const bool stamper = wg == 0 && lane == 0 && g < 2;
 
         for (int it = g; it < total; it += kGroups) {
             const int sq = it % SQ, s = it % S;
-            if (stamper) DSTAMP(1 + g, it, 0);
             // the W slot is free once the MMAs of step it - S have completed
-            if (it >= S && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1)))) { failed = true; break; }
+            if (it >= S && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1), status))) { failed = true; break; }
             tc_fence_after_sync();
-            if (stamper) DSTAMP(1 + g, it, 1);
 
             // codes -> levels -> TMEM
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1)))) { failed = true; break; }
-            if (stamper) DSTAMP(1 + g, it, 4);
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1), status))) { failed = true; break; }
             dequant_row_to_tmem<BITS, C::COLS>(q0 + sq * C::QSTAGE + row_in_tile * C::QROW, row_in_tile, ch, lut_lane,
                                       lane_addr + kWCol + (uint32_t)((h * S + s) * kWSlotCols));
-            if (stamper) DSTAMP(1 + g, it, 5);
             tmem_wait_st();
             tc_fence_before_sync();
-            if (stamper) DSTAMP(1 + g, it, 7);
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(bar_ready + 8 * (h * S + s));
                 mbar_arrive(bar_q_empty + 8 * sq);
             }
-            if (stamper) DSTAMP(1 + g, it, 3);
         }
 
         // Epilogue (group 0): z (TMEM) . B row -> this CTA's partial y, parked in the cluster
         // leader's shared memory; the leader adds the cluster's partials in rank order.
-        if (g == 0 && ch == 0 && !failed) {
+        if (g == 0 && ch == 0) {
             const int i = tile * kTileRows + row_in_tile;
-            if (stamper) DSTAMP(5, 0, 0);
             // B row first, so its latency hides behind the wait for the last MMAs
             uint4 bq[kNMax / 8];
+            if ((p.r & 7) == 0) {
 #pragma unroll
-            for (int c = 0; c < kNMax / 8; ++c)
-                bq[c] = (i < p.m && c * 8 < p.r) ? __ldg(reinterpret_cast<const uint4 *>(p.B + (size_t)i * p.r) + c)
-                                                 : make_uint4(0, 0, 0, 0);
+                for (int c = 0; c < kNMax / 8; ++c)
+                    bq[c] = (i < p.m && c * 8 < p.r) ? __ldg(reinterpret_cast<const uint4 *>(p.B + (size_t)i * p.r) + c)
+                                                     : make_uint4(0, 0, 0, 0);
+            } else {
+                // ranks that are not a multiple of 8: the rows of B are not 16-byte aligned
+#pragma unroll
+                for (int c = 0; c < kNMax / 8; ++c) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int k = c * 8 + 2 * e;
+                        const uint32_t lo = (i < p.m && k < p.r) ? __ldg(p.B + (size_t)i * p.r + k) : 0u;
+                        const uint32_t hi = (i < p.m && k + 1 < p.r) ? __ldg(p.B + (size_t)i * p.r + k + 1) : 0u;
+                        w[e] = lo | (hi << 16);
+                    }
+                    bq[c] = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
             // second half of the split-phase cluster barrier (every CTA of the cluster has initialised
             // its barriers): taken here, where its latency hides behind the wait for the last MMAs
             if (csize > 1) {
@@ -504,7 +483,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             float yt[NTOK];
 #pragma unroll
             for (int t = 0; t < NTOK; ++t) yt[t] = 0.0f;
-            bool ok = true;
+            bool ok = !failed;
             // H == 2: this half's accumulator.  H == 1: the accumulators of both issuers (the second
             // one only if it had a k-step at all).
             constexpr int kAccs = H == 2 ? 1 : 2;
@@ -512,9 +491,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             for (int a = 0; a < kAccs; ++a) {
                 const int j = H == 2 ? h : a;
                 if (ok && j < total + (H == 2 ? 2 : 0)) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * j, 0));
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * j, 0, status));
                     tc_fence_after_sync();
-                    if (stamper) DSTAMP(5, 0, 1);
                     if (ok) {
 #pragma unroll
                         for (int t = 0; t < NTOK; ++t) {
@@ -539,7 +517,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                     }
                 }
             }
-            if (stamper) DSTAMP(5, 0, 2);
             if (!ok) failed = true;
             if (csize == 1) {
                 if (ok && i < p.m)
@@ -551,9 +528,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
 #pragma unroll
                 for (int t = 0; t < NTOK; ++t)
                     st_async_cluster_f32(map_to_rank(red0 + ((rank * NTOK + t) * kTileRows + row_in_tile) * 4, 0), yt[t], leader_bar);
-                if (stamper) DSTAMP(5, 0, 3);
                 if (rank == 0) {
-                    if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0))) failed = true;
+                    if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0, status))) failed = true;
                     else if (i < p.m) {
                         // all partials are read first (the loads overlap), then added in rank order
                         float v[NTOK][kClusterMax];
@@ -570,7 +546,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                             store_out(p.y, p.y_f32, (size_t)t * p.m + i, a);
                         }
                     }
-                    if (stamper) DSTAMP(5, 0, 4);
                 }
             }
         }
@@ -579,7 +554,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     if (failed) atomicExch(p.status, LORDS_ERR_TIMEOUT);
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0) DSTAMP(7, 0, 2);
     if (warp == kIssuerWarp0) {
         tc_fence_after_sync();
         uint32_t tmem_base;
@@ -597,49 +571,19 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
-}
-
-bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *ptr, uint64_t inner,
-                 uint64_t outer, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swz)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {inner, outer};
-    cuuint64_t strides[1] = {inner * (uint64_t)elem_bytes};
-    cuuint32_t box[2] = {box_inner, box_outer};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // One (code width, tokens, halves) instantiation: its launch attributes, how many clusters of each
 // size the device can hold at once, and the launch itself.
 template <int BITS, int NTOK, int H> struct DecodeVariant {
-    static int prepare()
+    static int prepare(int dev)
     {
-        static bool done = false;
-        if (!done) {
+        static bool done[kMaxDevices] = {};
+        if (!done[dev]) {
             auto kernel = lords_decode_kernel<BITS, NTOK, H>;
             LORDS_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DCfg<BITS, H>::SMEM));
             // cluster sizes above 8 are outside the portable range; they are used only where the
             // occupancy query below says such a cluster fits
             LORDS_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
-            done = true;
+            done[dev] = true;
         }
         return LORDS_OK;
     }
@@ -662,19 +606,19 @@ template <int BITS, int NTOK, int H> struct DecodeVariant {
         cfg.numAttrs = 2;
     }
     // Clusters of `cs` CTAs that can be resident at the same time (0 if such a cluster cannot run).
-    static int max_clusters(int cs)
+    static int max_clusters(int dev, int cs)
     {
-        static int cache[kClusterMax + 1];   // 0 = not asked yet, -1 = cannot run
-        if (cache[cs] == 0) {
+        static int cache[kMaxDevices][kClusterMax + 1];   // 0 = not asked yet, -1 = cannot run
+        if (cache[dev][cs] == 0) {
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute attr[2];
             fill(cfg, attr, cs, 1, nullptr);
             int n = 0;
             const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_decode_kernel<BITS, NTOK, H>, &cfg);
             if (e != cudaSuccess) (void)cudaGetLastError();
-            cache[cs] = (e == cudaSuccess && n >= 1) ? n : -1;
+            cache[dev][cs] = (e == cudaSuccess && n >= 1) ? n : -1;
         }
-        return cache[cs] > 0 ? cache[cs] : 0;
+        return cache[dev][cs] > 0 ? cache[dev][cs] : 0;
     }
     static int launch(const DecodeParams &k, int tiles, int cs, cudaStream_t stream)
     {
@@ -689,19 +633,19 @@ template <int BITS, int NTOK, int H> struct DecodeVariant {
 // Cluster size for `tiles` tiles of `ksteps` k-steps: the largest split that still lets every cluster
 // be resident at once (one wave); 1 when there are more tiles than that.  `cost` receives a relative
 // time estimate, k-steps per CTA x waves x the per-step weight of the tile height.
-template <int BITS, int NTOK, int H> int choose_cluster(int tiles, int ksteps, int forced, double &cost)
+template <int BITS, int NTOK, int H> int choose_cluster(int dev, int tiles, int ksteps, int forced, double &cost)
 {
     using V = DecodeVariant<BITS, NTOK, H>;
     int cs = 1;
     if (forced > 0) {
         cs = forced < kClusterMax ? forced : kClusterMax;
         if (cs > ksteps) cs = ksteps;
-        while (cs > 1 && V::max_clusters(cs) == 0) --cs;
+        while (cs > 1 && V::max_clusters(dev, cs) == 0) --cs;
     } else {
         for (int c = kClusterMax < ksteps ? kClusterMax : ksteps; c > 1; --c)
-            if (V::max_clusters(c) >= tiles) { cs = c; break; }
+            if (V::max_clusters(dev, c) >= tiles) { cs = c; break; }
     }
-    const int resident = V::max_clusters(cs) > 0 ? V::max_clusters(cs) : 1;
+    const int resident = V::max_clusters(dev, cs) > 0 ? V::max_clusters(dev, cs) : 1;
     const int waves = (tiles + resident - 1) / resident;
     const int steps = (ksteps + cs - 1) / cs;
     // a two-half step covers twice the rows in about 1.7 times the time of a one-half step, and every
@@ -710,18 +654,19 @@ template <int BITS, int NTOK, int H> int choose_cluster(int tiles, int ksteps, i
     return cs;
 }
 
-template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem &p, int forced_cs, int forced_halves, cudaStream_t stream)
+template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem &p, const State &st, cudaStream_t stream)
 {
+    const int dev = device_slot(st), forced_cs = st.forced_splitk, forced_halves = 0;
     const int qrow = DCfg<BITS, 1>::QROW;
     k.ksteps = (p.n + kStep - 1) / kStep;
-    int rc = DecodeVariant<BITS, NTOK, 1>::prepare();
-    if (rc == LORDS_OK) rc = DecodeVariant<BITS, NTOK, 2>::prepare();
+    int rc = DecodeVariant<BITS, NTOK, 1>::prepare(dev);
+    if (rc == LORDS_OK) rc = DecodeVariant<BITS, NTOK, 2>::prepare(dev);
     if (rc != LORDS_OK) return rc;
     const int tiles1 = (p.m + 127) / 128, tiles2 = (p.m + 255) / 256;
     if (tiles1 > 65535) return LORDS_ERR_UNSUPPORTED;
     double cost1 = 0, cost2 = 0;
-    const int cs1 = choose_cluster<BITS, NTOK, 1>(tiles1, k.ksteps, forced_cs, cost1);
-    const int cs2 = choose_cluster<BITS, NTOK, 2>(tiles2, k.ksteps, forced_cs, cost2);
+    const int cs1 = choose_cluster<BITS, NTOK, 1>(dev, tiles1, k.ksteps, forced_cs, cost1);
+    const int cs2 = choose_cluster<BITS, NTOK, 2>(dev, tiles2, k.ksteps, forced_cs, cost2);
     const bool two = forced_halves > 0 ? forced_halves == 2 : cost2 < cost1;
     const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
     if (!make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)qrow,
@@ -738,13 +683,13 @@ template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem
 
 }  // namespace
 
-// Rules of this path: 3- or 4-bit codes; M <= 2 with M * ceil16(r) <= 64; r a multiple of 8 (16-byte
-// rows of B); n a multiple of 32 (4-bit) or 128 (3-bit), which makes every TMA row pitch a multiple
-// of 16 bytes.  Anything else: LORDS_ERR_UNSUPPORTED.
+// Rules of this path: 3- or 4-bit codes; M <= 2 with M * ceil16(r) <= 64; n a multiple of 32 (4-bit)
+// or 128 (3-bit), which makes every TMA row pitch a multiple of 16 bytes.  Anything else:
+// LORDS_ERR_UNSUPPORTED.
 int launch_decode(const Problem &p, State &st, cudaStream_t stream)
 {
     if (p.bits != 3 && p.bits != 4) return LORDS_ERR_UNSUPPORTED;
-    if (p.M > 2 || p.r % 8 != 0) return LORDS_ERR_UNSUPPORTED;
+    if (p.M > 2) return LORDS_ERR_UNSUPPORTED;
     const int r_pad = (p.r + 15) / 16 * 16;
     if (p.M * r_pad > kNMax) return LORDS_ERR_UNSUPPORTED;
     if (p.n % (p.bits == 4 ? 32 : 128) != 0) return LORDS_ERR_UNSUPPORTED;
@@ -755,30 +700,13 @@ int launch_decode(const Problem &p, State &st, cudaStream_t stream)
     k.M = p.M; k.m = p.m; k.n = p.n; k.r = p.r; k.r_pad = r_pad;
     k.y = p.y; k.y_f32 = p.y_f32;
     k.status = st.status_word;
-#ifdef LORDS_TRACE
-    k.trace = reinterpret_cast<long long *>(st.workspace + st.workspace_bytes - (size_t)8 * 32 * 8 * 8);
-    LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)8 * 32 * 8 * 8, stream));
-#endif
     int rc;
-    if (p.bits == 4) rc = p.M == 1 ? launch_bits_tok<4, 1>(k, p, st.forced_splitk, st.forced_halves, stream) : launch_bits_tok<4, 2>(k, p, st.forced_splitk, st.forced_halves, stream);
-    else rc = p.M == 1 ? launch_bits_tok<3, 1>(k, p, st.forced_splitk, st.forced_halves, stream) : launch_bits_tok<3, 2>(k, p, st.forced_splitk, st.forced_halves, stream);
+    if (p.bits == 4) rc = p.M == 1 ? launch_bits_tok<4, 1>(k, p, st, stream) : launch_bits_tok<4, 2>(k, p, st, stream);
+    else rc = p.M == 1 ? launch_bits_tok<3, 1>(k, p, st, stream) : launch_bits_tok<3, 2>(k, p, st, stream);
     if (rc != LORDS_OK) return rc;
     st.last_launches = 1;
     st.last_path = "decode";
     return LORDS_OK;
 }
-
-#ifdef LORDS_TRACE
-// Debug builds only: copy the traced CTA's clock stamps of the last decode launch to the host.
-extern "C" int lords_debug_read_decode_trace(long long *out)
-{
-    State &st = state();
-    if (!st.initialised) return LORDS_ERR_NOT_INIT;
-    LORDS_CUDA_TRY(cudaDeviceSynchronize());
-    LORDS_CUDA_TRY(cudaMemcpy(out, st.workspace + st.workspace_bytes - (size_t)8 * 32 * 8 * 8, (size_t)8 * 32 * 8 * 8,
-                              cudaMemcpyDeviceToHost));
-    return LORDS_OK;
-}
-#endif
 
 }  // namespace lords

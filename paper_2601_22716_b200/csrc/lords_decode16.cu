@@ -33,6 +33,7 @@
 
 #include "lords_internal.h"
 #include "lords_ptx.cuh"
+#include "lords_tc_common.cuh"
 
 namespace lords {
 
@@ -131,12 +132,6 @@ struct alignas(64) Dec16Params {
 #else
 #define XSTAMP(role, it, ev) do { } while (0)
 #endif
-
-__device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float v)
-{
-    if (y_f32) static_cast<float *>(y)[idx] = v;
-    else static_cast<__nv_bfloat16 *>(y)[idx] = __float2bfloat16_rn(v);
-}
 
 // 64 columns of one row: code pairs -> level pairs, times the matching pairs of S (sp, in and out).
 // 4-bit rows are 64 bytes and arrive 64-byte-swizzled (16-byte chunk c of row i sits at chunk
@@ -592,45 +587,15 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
-}
-
-bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *ptr, uint64_t inner,
-                 uint64_t outer, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swz)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {inner, outer};
-    cuuint64_t strides[1] = {inner * (uint64_t)elem_bytes};
-    cuuint32_t box[2] = {box_inner, box_outer};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // One (code width, rank slot) instantiation: launch attributes, resident clusters per size, launch.
 template <int BITS, int RP> struct Dec16Variant {
-    static int prepare()
+    static int prepare(int dev)
     {
-        static bool done = false;
-        if (!done) {
+        static bool done[kMaxDevices] = {};
+        if (!done[dev]) {
             LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_decode16_kernel<BITS, RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 XCfg<BITS, RP>::SMEM));
-            done = true;
+            done[dev] = true;
         }
         return LORDS_OK;
     }
@@ -652,27 +617,28 @@ template <int BITS, int RP> struct Dec16Variant {
         cfg.numAttrs = 2;
     }
     // Clusters of `cs` CTAs that can be resident at the same time (0 if such a cluster cannot run).
-    static int max_clusters(int cs)
+    static int max_clusters(int dev, int cs)
     {
-        static int cache[kClusterMax + 1];   // 0 = not asked yet, -1 = cannot run
-        if (cache[cs] == 0) {
+        static int cache[kMaxDevices][kClusterMax + 1];   // 0 = not asked yet, -1 = cannot run
+        if (cache[dev][cs] == 0) {
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute attr[2];
             fill(cfg, attr, cs, 1, nullptr);
             int n = 0;
             const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_decode16_kernel<BITS, RP>, &cfg);
             if (e != cudaSuccess) (void)cudaGetLastError();
-            cache[cs] = (e == cudaSuccess && n >= 1) ? n : -1;
+            cache[dev][cs] = (e == cudaSuccess && n >= 1) ? n : -1;
         }
-        return cache[cs] > 0 ? cache[cs] : 0;
+        return cache[dev][cs] > 0 ? cache[dev][cs] : 0;
     }
 };
 
-template <int BITS, int RP> int launch_variant(Dec16Params &k, const Problem &p, int forced_cs, cudaStream_t stream)
+template <int BITS, int RP> int launch_variant(Dec16Params &k, const Problem &p, const State &st, cudaStream_t stream)
 {
     using V = Dec16Variant<BITS, RP>;
     using C = XCfg<BITS, RP>;
-    int rc = V::prepare();
+    const int dev = device_slot(st), forced_cs = st.forced_splitk;
+    int rc = V::prepare(dev);
     if (rc != LORDS_OK) return rc;
     const int tiles = (p.m + kRows - 1) / kRows;
     if (tiles > 65535) return LORDS_ERR_UNSUPPORTED;
@@ -681,10 +647,10 @@ template <int BITS, int RP> int launch_variant(Dec16Params &k, const Problem &p,
     const int lim = kClusterMax < k.ksteps ? kClusterMax : k.ksteps;
     if (forced_cs > 0) {
         cs = forced_cs < lim ? forced_cs : lim;
-        while (cs > 1 && V::max_clusters(cs) == 0) --cs;
+        while (cs > 1 && V::max_clusters(dev, cs) == 0) --cs;
     } else {
         for (int c = lim; c > 1; --c)
-            if (V::max_clusters(c) >= tiles) { cs = c; break; }
+            if (V::max_clusters(dev, c) >= tiles) { cs = c; break; }
     }
     const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
     if (!make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)C::QROW, (uint32_t)kRows,
@@ -734,8 +700,8 @@ int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
     LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)8 * 32 * 8 * 8, stream));
 #endif
     int rc;
-    if (p.bits == 4) rc = launch_variant<4, 32>(k, p, st.forced_splitk, stream);
-    else rc = k.r_pad <= 32 ? launch_variant<3, 32>(k, p, st.forced_splitk, stream) : launch_variant<3, 64>(k, p, st.forced_splitk, stream);
+    if (p.bits == 4) rc = launch_variant<4, 32>(k, p, st, stream);
+    else rc = k.r_pad <= 32 ? launch_variant<3, 32>(k, p, st, stream) : launch_variant<3, 64>(k, p, st, stream);
     if (rc != LORDS_OK) return rc;
     st.last_launches = 1;
     st.last_path = "decode16";

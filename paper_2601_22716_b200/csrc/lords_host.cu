@@ -227,12 +227,11 @@ int lords_shutdown(void)
         if (st.stage_x) cudaFree(st.stage_x);
         if (st.stage_y) cudaFree(st.stage_y);
     }
-    int fp = st.forced_path, fs = st.forced_splitk, fb = st.forced_bn, fh = st.forced_halves;
+    int fp = st.forced_path, fs = st.forced_splitk, fb = st.forced_bn;
     st = State();
     st.forced_path = fp;
     st.forced_splitk = fs;
     st.forced_bn = fb;
-    st.forced_halves = fh;
     return LORDS_OK;
 }
 
@@ -317,11 +316,6 @@ int lords_set_option(const char *key, const char *value)
         long v = std::strtol(value, &end, 10);
         if (end == value || *end != '\0' || v < 0 || v > 1024) return LORDS_ERR_OPTION;
         st.forced_splitk = (int)v;
-        return LORDS_OK;
-    }
-    if (std::strcmp(key, "halves") == 0) {
-        if (std::strcmp(value, "0") != 0 && std::strcmp(value, "1") != 0 && std::strcmp(value, "2") != 0) return LORDS_ERR_OPTION;
-        st.forced_halves = value[0] - '0';
         return LORDS_OK;
     }
     if (std::strcmp(key, "bn") == 0) {

@@ -37,7 +37,6 @@ struct State {
     size_t stage_x_bytes = 0, stage_y_bytes = 0;
     int forced_path = 0;            // 0 auto, 1 simt, 2 decode (reassociated form), 3 umma (scale-MMA form), 4 decode16
     int forced_splitk = 0;          // 0 auto
-    int forced_halves = 0;          // 0 auto; else the tile height of the decode kernel in 128-row halves (1, 2)
     int forced_bn = 0;              // 0 auto; else the token tile of the scale-MMA kernel (32, 64, 128, 256)
     int last_cuda_error = 0;
     int last_launches = 0;

@@ -50,43 +50,58 @@ __device__ __forceinline__ unsigned long long global_ns()
     return t;
 }
 
-// The limit of every bounded wait: it gives up only when three independent measures agree that it
-// has waited for seconds -- the number of polls, the SM's cycle counter and the GPU's wall clock.
-// (With the cycle counter alone, waits on many SMs were seen to run out at the same instant about
-// once in fifteen runs of a 224-kernel graph; no wait of these kernels takes a millisecond.)
+// The limit of every bounded wait.  No wait of these kernels that starts after the kernel's own
+// dependency point lasts longer than the kernel itself (tens of microseconds), so a wait that has
+// polled for kWaitLimitNs of wall-clock time is taken as lost; it also ends at once when the
+// library's status word shows that some other role has already given up, so one give-up drains the
+// whole grid instead of letting every wait run to its own limit.
+constexpr unsigned long long kWaitLimitNs = 50ull * 1000 * 1000;
+constexpr unsigned kWaitSleepNs = 40;
 struct WaitLimit {
-    long long c0;
     unsigned long long g0;
     unsigned rounds;
 };
 __device__ __forceinline__ WaitLimit wait_limit_start()
 {
     WaitLimit w;
-    w.c0 = clock64();
     w.g0 = global_ns();
     w.rounds = 0;
     return w;
 }
-// called after every 256 unsuccessful polls
-__device__ __forceinline__ bool wait_limit_expired(WaitLimit &w)
+// called after every 64 unsuccessful tries; `status` is the library's device status word (may be null)
+__device__ __forceinline__ bool wait_limit_expired(WaitLimit &w, const int *status)
 {
     ++w.rounds;
-    return w.rounds > 256u && clock64() - w.c0 > 4000000000LL && global_ns() - w.g0 > 2000000000ULL;
+    if (status != nullptr && *reinterpret_cast<const volatile int *>(status) != 0) return true;
+    return w.rounds > 4u && global_ns() - w.g0 > kWaitLimitNs;
 }
 
-// Bounded wait: gives up after about two seconds of polling and reports failure, so that no role of
-// a kernel can spin forever on a shared GPU.  Callers record LORDS_ERR_TIMEOUT and drain.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Bounded wait: gives up after kWaitLimitNs of polling (or as soon as the status word is set) and
+// reports failure, so that no role of a kernel can spin forever on a shared GPU.  Callers record
+// LORDS_ERR_TIMEOUT and drain.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const int *status = nullptr)
 {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity) || mbar_try_wait(bar, parity)) return true;
+    // a waiting warp sleeps between its tries, so that it does not take issue slots from the warps
+    // it is waiting for
     WaitLimit limit = wait_limit_start();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 256; ++i)
+        for (int i = 0; i < 64; ++i) {
+            __nanosleep(kWaitSleepNs);
             if (mbar_try_wait(bar, parity)) return true;
-        if (wait_limit_expired(limit)) return false;
+        }
+        if (wait_limit_expired(limit, status)) return false;
     }
 }
+
+// ---- programmatic dependent launch ----------------------------------------------------------------
+// Lets the next kernel of the stream begin (its CTAs start as resources free up).
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// Returns when the previous kernel of the stream has finished and its writes are visible.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 // ---- proxies / fences -------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem()
@@ -125,6 +140,22 @@ __device__ __forceinline__ void tmem_relinquish()
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
 {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// The same three for a CTA pair (cta_group::2): one warp of EACH of the two CTAs executes them, and
+// every tcgen05 instruction of such a kernel names cta_group::2.
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(cols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 
 // 32 lanes x 32 consecutive 32-bit columns: thread l of the warp receives lane (base_lane + l).
@@ -235,6 +266,13 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
+// Arrival on an mbarrier of another CTA of the cluster without a cluster-scope release: for hand-offs
+// whose data does not travel through generic memory (tensor memory written with tcgen05.st and fenced
+// with tcgen05 fences; shared memory of the arriving CTA itself, fenced for the async proxy).
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
@@ -250,15 +288,17 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     return ok != 0;
 }
 // Bounded like mbar_wait, with acquire at cluster scope (the arrivals come from other CTAs).
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const int *status = nullptr)
 {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     WaitLimit limit = wait_limit_start();
     for (;;) {
 #pragma unroll 1
-        for (int i = 0; i < 256; ++i)
+        for (int i = 0; i < 64; ++i) {
+            __nanosleep(kWaitSleepNs);
             if (mbar_try_wait_cluster(bar, parity)) return true;
-        if (wait_limit_expired(limit)) return false;
+        }
+        if (wait_limit_expired(limit, status)) return false;
     }
 }
 
@@ -325,6 +365,40 @@ __device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, ui
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// CTA-pair forms (cta_group::2), issued by one thread of the pair's even-ranked CTA.
+// D[tmem, 256 rows: 128 lanes in each CTA] (+)= A[tmem of each CTA] * B[smem: rows 0..N/2-1 in the even
+// CTA, N/2..N-1 in the odd one, at the same shared-memory offset]
+__device__ __forceinline__ void umma_pair_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive once on the barrier at the same shared-memory offset in every CTA of `cta_mask` (bit = rank
+// in the cluster) when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_pair_commit(uint32_t bar, uint16_t cta_mask)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(cta_mask) : "memory");
+}
+
+// Two fp32 products in one instruction: {a.x * b.x, a.y * b.y}, round to nearest even.
+__device__ __forceinline__ float2 mul_f32x2(float2 a, float2 b)
+{
+    unsigned long long ua, ub, ud;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ua) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ub) : "f"(b.x), "f"(b.y));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(ud) : "l"(ua), "l"(ub));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(ud));
+    return d;
 }
 
 }  // namespace ptx

@@ -25,6 +25,7 @@
 
 #include "lords_internal.h"
 #include "lords_ptx.cuh"
+#include "lords_tc_common.cuh"
 
 namespace lords {
 
@@ -102,12 +103,6 @@ struct alignas(64) UmmaParams {
 #else
 #define USTAMP(role, it, ev) do { } while (0)
 #endif
-
-__device__ __forceinline__ void store_out(void *y, int y_f32, size_t idx, float v)
-{
-    if (y_f32) static_cast<float *>(y)[idx] = v;
-    else static_cast<__nv_bfloat16 *>(y)[idx] = __float2bfloat16_rn(v);
-}
 
 // The 32 columns (chunk c of the 128-column code stage) of one row: codes -> level pairs, times the
 // matching pairs of S, as 16 fp16x2 words.
@@ -572,44 +567,14 @@ __global__ void lords_x_to_f16_kernel(const uint4 *__restrict__ x, uint4 *__rest
     x16[e] = make_uint4(out[0], out[1], out[2], out[3]);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
-}
-
-bool make_map_2d(CUtensorMap *map, CUtensorMapDataType dt, int elem_bytes, const void *ptr, uint64_t inner,
-                 uint64_t outer, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swz)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {inner, outer};
-    cuuint64_t strides[1] = {inner * (uint64_t)elem_bytes};
-    cuuint32_t box[2] = {box_inner, box_outer};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int BITS, int BN, int RP> struct UmmaVariant {
-    static int prepare()
+    static int prepare(int dev)
     {
-        static bool done = false;
-        if (!done) {
+        static bool done[kMaxDevices] = {};
+        if (!done[dev]) {
             LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_umma_kernel<BITS, BN, RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 UCfg<BITS, BN, RP>::SMEM));
-            done = true;
+            done[dev] = true;
         }
         return LORDS_OK;
     }
@@ -631,19 +596,19 @@ template <int BITS, int BN, int RP> struct UmmaVariant {
         cfg.numAttrs = 2;
     }
     // Clusters of `cs` CTAs that can be resident at the same time (0 if such a cluster cannot run).
-    static int max_clusters(int cs)
+    static int max_clusters(int dev, int cs)
     {
-        static int cache[kClusterMax + 1];   // 0 = not asked yet, -1 = cannot run
-        if (cache[cs] == 0) {
+        static int cache[kMaxDevices][kClusterMax + 1];   // 0 = not asked yet, -1 = cannot run
+        if (cache[dev][cs] == 0) {
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute attr[2];
             fill(cfg, attr, cs, 1, nullptr);
             int n = 0;
             const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_umma_kernel<BITS, BN, RP>, &cfg);
             if (e != cudaSuccess) (void)cudaGetLastError();
-            cache[cs] = (e == cudaSuccess && n >= 1) ? n : -1;
+            cache[dev][cs] = (e == cudaSuccess && n >= 1) ? n : -1;
         }
-        return cache[cs] > 0 ? cache[cs] : 0;
+        return cache[dev][cs] > 0 ? cache[dev][cs] : 0;
     }
     static int launch(const UmmaParams &k, int tiles, int cs, cudaStream_t stream)
     {
@@ -658,7 +623,8 @@ template <int BITS, int BN, int RP> struct UmmaVariant {
 template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Problem &p, State &st, cudaStream_t stream)
 {
     using V = UmmaVariant<BITS, BN, RP>;
-    int rc = V::prepare();
+    const int dev = device_slot(st);
+    int rc = V::prepare(dev);
     if (rc != LORDS_OK) return rc;
     k.tok_tiles = (p.M + BN - 1) / BN;
     const int row_tiles = (p.m + BM - 1) / BM;
@@ -673,7 +639,7 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
         int lim = want < kClusterMax ? (int)want : kClusterMax;
         if (lim > k.npairs) lim = k.npairs;
         for (int c = lim; c > 1; --c)
-            if (V::max_clusters(c) >= (forced ? 1 : tiles)) { cs = c; break; }
+            if (V::max_clusters(dev, c) >= (forced ? 1 : tiles)) { cs = c; break; }
     }
 
     // Pair mode (BN > 16): when the tiles need more than one wave of CTAs, idle slots of the last wave
@@ -683,7 +649,7 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
     int clusters = (int)tiles;
     size_t pair_bytes = 0;
     if (BN > 16 && k.npairs >= 2) {
-        const long long resident = 2LL * V::max_clusters(2);
+        const long long resident = 2LL * V::max_clusters(dev, 2);
         if (resident > 0 && tiles > resident) {
             const long long waves = (tiles + resident - 1) / resident;
             long long split = waves * resident - tiles;

@@ -118,11 +118,11 @@ def test_options():
 def test_measurement_options_are_validated():
     # known keys with legal values
     for key, value in [("path", "auto"), ("path", "simt"), ("path", "decode"), ("path", "decode16"), ("path", "umma"), ("path", "prefill"),
-                       ("splitk", "0"), ("splitk", "7"), ("bn", "0"), ("bn", "128"), ("halves", "2"), ("halves", "0")]:
+                       ("splitk", "0"), ("splitk", "7"), ("bn", "0"), ("bn", "128")]:
         lords.lords_set_option(key, value)
-    for key, value in [("path", "fast"), ("splitk", "-1"), ("splitk", "x"), ("bn", "48"), ("halves", "3"), ("colour", "blue")]:
+    for key, value in [("path", "fast"), ("splitk", "-1"), ("splitk", "x"), ("bn", "48"), ("halves", "2"), ("colour", "blue")]:
         with pytest.raises(lords.LordsError) as ei:
             lords.lords_set_option(key, value)
         assert ei.value.status == -10
-    for key, value in [("path", "auto"), ("splitk", "0"), ("bn", "0"), ("halves", "0")]:
+    for key, value in [("path", "auto"), ("splitk", "0"), ("bn", "0")]:
         lords.lords_set_option(key, value)
