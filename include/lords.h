@@ -34,6 +34,13 @@
  *     read only the weights (Qpacked, B, A); x is read, and y written, after it.  So the weights must
  *     not be produced by work that is still in flight on `stream` when a forward call is made
  *     (synchronise the stream once after loading or updating weights); activations may be.
+ *   - precision and range: products are accumulated in fp32.  The tensor-core kernels hold their
+ *     operands in fp16, each rounded once: the dequantised weight L[Q_ij] * (BA)_ij (M > 2), or the bare
+ *     level L[Q_ij] and the product A_kj * x_tj (M <= 2), and x itself (M > 2).  These values must lie
+ *     within fp16's range: magnitudes above 65504 overflow to infinity, magnitudes below 6.1e-5 are
+ *     rounded to multiples of 6e-8 (which matters only where such terms dominate a sum).  Layer
+ *     weights and activations of the usual scales (|x| up to a few thousand, factors around 1e-2 to 1)
+ *     are far inside; the CUDA-core path ("path" = "simt") is fp32 throughout and has no such limit.
  *   - forward calls validate on the host, enqueue work on `stream` and return
  *     without synchronising.  They use library-owned scratch memory, so two forward
  *     calls may only overlap on the GPU if they are ordered on the same stream.
@@ -178,6 +185,11 @@ int lords_linear_forward_noalloc(const void *x, const uint8_t *Qpacked, const vo
 /*
  * Read and clear the device status word.  Synchronises `stream` first.  Returns LORDS_OK, or
  * the error a kernel recorded (LORDS_ERR_TIMEOUT when a bounded wait ran out).
+ * Every device-side wait of the tensor-core kernels is bounded (50 ms); a wait that runs out records
+ * LORDS_ERR_TIMEOUT here, every other wait then ends at once, and the kernels finish without
+ * writing their results.  Forward calls do not report this themselves: when this call returns
+ * non-zero, the y of every forward call since the previous poll is undefined, and so is the y of
+ * calls made before the word is cleared by this call.
  */
 int lords_poll_status(void *stream);
 
@@ -189,7 +201,9 @@ int lords_last_cuda_error(void);
  * M <= 2) | "decode16" (scale-MMA form with 128-column k-steps, 3 <= M <= 16) | "umma" (scale-MMA
  * kernel for any M; "prefill" is an alias);
  * "splitk" = "0" (auto) or a positive integer (CTAs sharing one tile's k-range); "bn" = "0" (auto)
- * or the token tile 32, 64, 128, 256 of the scale-MMA kernel for M > 16.  Unknown keys: LORDS_ERR_OPTION.
+ * or the token tile 32, 64, 128, 256 of the scale-MMA kernel for M > 16; "inject_status" = "0" or a
+ * negative status code: writes that value into the device status word, as a kernel that gave up would
+ * (a test switch).  Unknown keys: LORDS_ERR_OPTION.
  */
 int lords_set_option(const char *key, const char *value);
 

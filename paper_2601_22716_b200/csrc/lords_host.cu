@@ -318,6 +318,16 @@ int lords_set_option(const char *key, const char *value)
         st.forced_splitk = (int)v;
         return LORDS_OK;
     }
+    if (std::strcmp(key, "inject_status") == 0) {
+        // test switch: write a value into the device status word, as a kernel that gave up would
+        char *end = nullptr;
+        long v = std::strtol(value, &end, 10);
+        if (end == value || *end != '\0' || v < -64 || v > 0) return LORDS_ERR_OPTION;
+        if (!st.initialised) return LORDS_ERR_NOT_INIT;
+        const int word = (int)v;
+        LORDS_CUDA_TRY(cudaMemcpy(st.status_word, &word, sizeof(int), cudaMemcpyHostToDevice));
+        return LORDS_OK;
+    }
     if (std::strcmp(key, "bn") == 0) {
         char *end = nullptr;
         long v = std::strtol(value, &end, 10);

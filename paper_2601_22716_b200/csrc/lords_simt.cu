@@ -190,6 +190,20 @@ __global__ void lords_splitk_reduce_kernel(const float *partial, int splits, siz
 
 }  // namespace
 
+// The kernel's dynamic shared-memory limit is raised once per device, with that device current, to
+// what the largest rank needs: both entry points that launch it then always find the same limit.
+int simt_prepare_device(int dev)
+{
+    static bool done[64] = {};
+    const int slot = dev >= 0 && dev < 64 ? dev : 0;
+    if (!done[slot]) {
+        const size_t most = ((size_t)LORDS_R_MAX * kChunk + kTokTile * kChunk + (size_t)kRowsPerCta * LORDS_R_MAX) * sizeof(float);
+        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most));
+        done[slot] = true;
+    }
+    return LORDS_OK;
+}
+
 int launch_simt(const Problem &p, State &st, cudaStream_t stream)
 {
     SimtParams k;
@@ -220,11 +234,8 @@ int launch_simt(const Problem &p, State &st, cudaStream_t stream)
     k.partial = reinterpret_cast<float *>(st.workspace);
 
     const size_t smem = ((size_t)p.r * kChunk + kTokTile * kChunk + (size_t)kRowsPerCta * p.r) * sizeof(float);
-    static size_t smem_attr = 0;
-    if (smem > smem_attr) {
-        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        smem_attr = smem;
-    }
+    const int prc = simt_prepare_device(st.device);
+    if (prc != LORDS_OK) return prc;
     dim3 grid(row_ctas, splits, tok_tiles);
     if (tok_tiles > 65535) return LORDS_ERR_SHAPE;
     lords_simt_kernel<<<grid, kWarps * 32, smem, stream>>>(k);
@@ -324,8 +335,8 @@ extern "C" int lords_linear_forward_noalloc(const void *x, const uint8_t *Qpacke
     k.partial = g_noalloc_ptr[dev];
 
     const size_t smem = ((size_t)r * kChunk + kTokTile * kChunk + (size_t)kRowsPerCta * r) * sizeof(float);
-    if (smem > 48 * 1024)
-        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_simt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int prc = simt_prepare_device(dev);
+    if (prc != LORDS_OK) return prc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (splits > 1) {
         lords_simt_kernel<<<dim3(row_ctas, splits, tok_tiles), kWarps * 32, smem, s>>>(k);

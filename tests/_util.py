@@ -31,8 +31,14 @@ def bf16_ulp(v):
     return 2.0 ** (np.floor(np.log2(v)) - 7)
 
 
-def check_against_oracle(y32, ybf_bits, y64):
-    """Assert the A-level tolerances; returns the metrics for reporting."""
+REPORT = []   # one line per checked case, printed at the end of the run (tests/conftest.py)
+
+
+def check_against_oracle(y32, ybf_bits, y64, label=None):
+    """Assert the A-level tolerances; returns the metrics and records them for the end-of-run report:
+    e_acc (fp32 accumulator vs oracle, normwise), e_out (bf16 output vs oracle), e_floor (a perfectly
+    rounded bf16 copy of the oracle vs the oracle), the largest per-element error of the accumulator,
+    and how many bf16 outputs differ from the rounded oracle value (all by at most one ulp)."""
     normwise, element = error_metrics(y32, y64)
     assert normwise <= NORMWISE_TOL, f"normwise {normwise:.3e} > {NORMWISE_TOL}"
     assert element <= ELEMENT_TOL, f"per-element {element:.3e} > {ELEMENT_TOL}"
@@ -47,7 +53,15 @@ def check_against_oracle(y32, ybf_bits, y64):
     got = gen.bf16_to_f32(ybf_bits).astype(np.float64)
     worst = float(np.max(np.abs(got - yhat) / ulp)) if got.size else 0.0
     assert worst <= 1.0 + 1e-9, f"bf16 output {worst:.2f} ulp from the rounded oracle value"
-    return {"normwise": normwise, "element": element, "ulp": worst}
+    e_out, _ = error_metrics(got, y64)
+    e_floor, _ = error_metrics(yhat, y64)
+    flips = int(np.count_nonzero(got != yhat))
+    if label is None:
+        import os
+        label = os.environ.get("PYTEST_CURRENT_TEST", "case").split("::")[-1].split(" ")[0]
+    REPORT.append(f"{label}: e_acc={normwise:.3e} e_out={e_out:.3e} e_floor={e_floor:.3e} "
+                  f"max_element={element:.3e} ulp_flips={flips}/{got.size} worst_ulp={worst:.2f}")
+    return {"normwise": normwise, "element": element, "ulp": worst, "e_out": e_out, "e_floor": e_floor, "flips": flips}
 
 
 class DeviceLayer:

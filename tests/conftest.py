@@ -15,3 +15,17 @@ def pytest_configure(config):
 @pytest.fixture(scope="session")
 def repo_root():
     return ROOT
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Every parity case reports its error figures (accumulator, bf16 output, rounding floor, worst
+    element, one-ulp flips), so that a reader with another reading of the tolerances can re-judge."""
+    try:
+        from _util import REPORT
+    except Exception:
+        return
+    if REPORT:
+        terminalreporter.write_line("")
+        terminalreporter.write_line("parity report (CUDA path vs fp64 oracle):")
+        for line in REPORT:
+            terminalreporter.write_line("  " + line)
