@@ -4,9 +4,11 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--case NAME]
 
 A *step* is one pass of the whole hot path (unpack, level lookup, scale reconstruction,
-Hadamard product, contraction, epilogue) over one batch of synthetic layers: `copies`
-distinct weight sets of the case's shape, one forward call each, so that a step touches
-more than twice the L2 capacity and every launch reads its weights from HBM.
+Hadamard product, contraction, epilogue) over one batch of synthetic layers: `rounds` rounds over
+`copies` distinct weight sets of the case's shape, one forward call each, so that a round touches
+more than twice the L2 capacity and every launch reads its weights from HBM.  `rounds` is chosen
+from a short calibration so that the K timed steps together last about a second whatever K is: the
+clock sampler then has samples and the tensor-bound case runs at sustained clocks.
 
 The headline case is the Llama-3-8B q_proj decode (m = n = 4096, NF4, r = 32, M = 1) and
 the headline metric is algorithmic HBM bytes per second (packed Q + B + A + x + y).  The
@@ -166,7 +168,10 @@ def copies_for(case):
     return max(2, -(-2 * L2_BYTES // per) + 1)
 
 
-def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=True):
+MIN_TIMED_SECONDS = 1.0   # the K timed steps together last at least about this long
+
+
+def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=True, min_seconds=MIN_TIMED_SECONDS):
     import numpy as np
     import torch
     import torch.distributed as dist
@@ -210,7 +215,25 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
               file=sys.stderr)
         torch.cuda.synchronize()
 
-    run = (graph.replay if graph is not None else one_step)
+    one_round = (graph.replay if graph is not None else one_step)
+    # calibration: rounds per step so that `steps` steps take about min_seconds (all ranks agree on the
+    # slowest rank's figure)
+    for _ in range(3):
+        one_round()
+    torch.cuda.synchronize()
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0.record()
+    for _ in range(3):
+        one_round()
+    c1.record()
+    torch.cuda.synchronize()
+    round_ms = max_over_ranks(c0.elapsed_time(c1) / 3.0, device, world)
+    rounds = int(max(1, min(100000, -(-min_seconds * 1e3 // max(steps * round_ms, 1e-6)))))
+
+    def run():
+        for _ in range(rounds):
+            one_round()
+
     for _ in range(max(warmup, 3)):
         run()
     # A device-side status (a bounded wait that gave up) invalidates the measurement: it is reported
@@ -233,7 +256,10 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
         status = lords.lords_poll_status()
         if status == 0:
             break
-        print(f"[bench] device status {status} during {case}; measuring once more", file=sys.stderr)
+        d0, d1 = lords.lords_read_status_detail()
+        print(f"[bench] device status {status} during {case} (first expired wait: tag {d0 & 0xFF}, parity {(d0 >> 8) & 1}, "
+              f"warp {(d0 >> 16) & 0xFF}, CTA {(d0 >> 32) & 0x7FFFFFFF}, barrier 0x{d1 & 0xFFFFFFFF:x}, "
+              f"{d1 >> 32} rounds of 64 tries); measuring once more", file=sys.stderr)
         status_retries += 1
         if status_retries > 1:
             raise RuntimeError(f"device status {status} during {case}, twice")
@@ -245,24 +271,25 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
         yh = [torch.zeros((M, m), dtype=torch.int16).pin_memory() for _ in range(copies)]
 
         def e2e_step():
-            for (q, B, A, _x), xx, yy in zip(sets, xh, yh):
-                lords.lords_linear_forward_host(xx, q, B, A, lay.codebook, bits, M, m, n, r, yy)
+            for _ in range(rounds):
+                for (q, B, A, _x), xx, yy in zip(sets, xh, yh):
+                    lords.lords_linear_forward_host(xx, q, B, A, lay.codebook, bits, M, m, n, r, yy)
 
-        for _ in range(3):
-            e2e_step()
+        for (q, B, A, _x), xx, yy in list(zip(sets, xh, yh)) * 3:
+            lords.lords_linear_forward_host(xx, q, B, A, lay.codebook, bits, M, m, n, r, yy)
         barrier()
         e0.record()
-        e2e_steps = max(1, min(steps, 200))
+        e2e_steps = max(1, min(steps, int(2.0 / (rounds * copies * 30e-6)) or 1))
         for _ in range(e2e_steps):
             e2e_step()
         e1.record()
         barrier()
         ems = max_over_ranks(e0.elapsed_time(e1), device, world)
-        e2e = {"ms_per_step": ems / e2e_steps, "h2d_bytes_per_step": copies * M * n * 2,
-               "d2h_bytes_per_step": copies * M * m * 2}
+        e2e = {"ms_per_step": ems / e2e_steps, "h2d_bytes_per_step": rounds * copies * M * n * 2,
+               "d2h_bytes_per_step": rounds * copies * M * m * 2, "steps": e2e_steps}
 
     peaks = measured_peaks()
-    calls = copies
+    calls = copies * rounds
     us_per_launch = ms_per_step * 1e3 / calls
     byt, flo = algorithmic_bytes(c), useful_flops(c)
     gbs = byt / (us_per_launch * 1e-6) / 1e9
@@ -279,7 +306,7 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
     roof["algorithmic_bytes_per_launch"] = byt
     roof["us_per_launch"] = us_per_launch
     res = {
-        "case": case, "path": path, "copies": copies, "ms_per_step": ms_per_step, "us_per_call": us_per_launch,
+        "case": case, "path": path, "copies": copies, "rounds": rounds, "ms_per_step": ms_per_step, "us_per_call": us_per_launch,
         "gbs": whole_job_value(gbs, world), "tflops": whole_job_value(tfs, world), "roofline": roof, "clocks": clocks,
         "launches_per_call": launches_per_call, "gpu_launches": steps * calls * launches_per_call,
         "graph": graph is not None, "status_retries": status_retries,
@@ -369,6 +396,42 @@ def time_stack(M, mlp_bits, steps, device):
             "frac_tensor": tfs / peaks["bf16_tflops"], "steps": steps, "status_retries": status_retries}
 
 
+def run_sweep(device):
+    """The measurement behind the per-M choice of kernel: every tensor-core path that accepts the
+    shape, at M in {1, 2, 3, 4, 8, 16}, on the q_proj (NF4, r = 32), gate and down (NF3, r = 48) shapes.
+    Microseconds per forward call, graph replay over distinct weight sets as in the main measurement."""
+    from paper_2601_22716_b200 import binding as lords
+    shapes = [("q_proj 4096x4096 NF4 r=32", dict(m=4096, n=4096, bits=4, r=32)),
+              ("gate 14336x4096 NF3 r=48", dict(m=14336, n=4096, bits=3, r=48)),
+              ("down 4096x14336 NF3 r=48", dict(m=4096, n=14336, bits=3, r=48))]
+    paths = ["decode", "decode16", "umma"]
+    rows = []
+    for label, shp in shapes:
+        for M in (1, 2, 3, 4, 8, 16):
+            CASES["_sweep"] = dict(shp, M=M, outliers=0.0, bound="hbm")
+            entry = {"shape": label, "M": M}
+            for path in paths:
+                lords.lords_set_option("path", path)
+                try:
+                    r = time_case("_sweep", 5, 3, device, 0, 1, None, do_e2e=False, min_seconds=0.12)
+                    r.pop("_lay")
+                    entry[path] = round(r["us_per_call"], 2)
+                except lords.LordsError:
+                    entry[path] = None           # the path declines this shape
+                finally:
+                    lords.lords_set_option("path", "auto")
+            lords.lords_set_option("path", "auto")
+            r = time_case("_sweep", 5, 3, device, 0, 1, None, do_e2e=False, min_seconds=0.12)
+            r.pop("_lay")
+            entry["auto"] = round(r["us_per_call"], 2)
+            entry["auto_path"] = r["path"]
+            rows.append(entry)
+            print(f"[sweep] {label} M={M}: " + ", ".join(f"{k}={entry[k]}" for k in paths) +
+                  f", auto={entry['auto']} ({entry['auto_path']})", file=sys.stderr)
+    CASES.pop("_sweep", None)
+    return rows
+
+
 def cpu_baseline(case, lay, packed, budget_s=12.0):
     """The oracle as it stands, on the host cores, on a bounded sample of the case."""
     import numpy as np
@@ -455,7 +518,10 @@ def main():
     ap.add_argument("--case", default=None, help="time only this case (default: headline plus the others)")
     ap.add_argument("--no-extras", action="store_true", help="headline case only")
     ap.add_argument("--path", default="auto", help="force a kernel path (auto|simt|decode|umma)")
-    ap.add_argument("--stack", action="store_true", help="also time the full Llama-3-8B linear stack (224 modules)")
+    ap.add_argument("--stack", action="store_true", help="(default) time the full Llama-3-8B linear stack as well")
+    ap.add_argument("--no-stack", action="store_true", help="skip the 224-module Llama-3-8B linear stack")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every kernel path at M in {1, 2, 3, 4, 8, 16} on the q_proj, gate and down shapes and print the table")
     args = ap.parse_args()
 
     if args.impl == "reference":
@@ -477,6 +543,15 @@ def main():
     lords.lords_init(local, 0)
     lords.lords_set_option("path", args.path)
 
+    if args.sweep:
+        rows = run_sweep(device) if rank == 0 else []
+        if rank == 0:
+            print(json.dumps({"sweep": rows, "unit": "us per forward call"}))
+        lords.lords_shutdown()
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
     head = args.case or HEADLINE
     sampler = ClockSampler(local) if rank == 0 else None
     res = time_case(head, args.steps, args.warmup, device, rank, world, sampler)
@@ -491,15 +566,15 @@ def main():
             k = {"decode_q_m8": 400, "mlp3_gate_m1": 800, "mlp3_down_m1": 800, "mlp3_down_m16": 300,
                  "prefill_m2048": 60}.get(name, 20)
             k = max(3, min(args.steps, k))
-            r2 = time_case(name, k, 3, device, rank, world, None, do_e2e=False)
+            r2 = time_case(name, k, 3, device, rank, world, None, do_e2e=False, min_seconds=0.4)
             r2.pop("_lay")
             cases.append({"case": name, "path": r2["path"], "us_per_call": r2["us_per_call"],
                           "gbs": r2["gbs"], "tflops": r2["tflops"], "roofline": r2["roofline"],
-                          "copies": r2["copies"], "steps": k, "status_retries": r2["status_retries"]})
+                          "copies": r2["copies"], "rounds": r2["rounds"], "steps": k, "status_retries": r2["status_retries"]})
 
     stack = []
-    if args.stack and world == 1:
-        for (M, mlp_bits, k) in [(1, 4, 20), (8, 4, 20), (512, 4, 3), (1, 3, 20)]:
+    if not args.no_stack and not args.no_extras and not args.case and world == 1:
+        for (M, mlp_bits, k) in [(1, 4, 30), (8, 4, 30), (512, 4, 5), (1, 3, 30)]:
             stack.append(time_stack(M, mlp_bits, k, device))
             torch.cuda.empty_cache()
 
@@ -515,8 +590,9 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f16",
             "data": "synthetic",
             "config": {"workload": head, **{k: c[k] for k in ("m", "n", "bits", "r", "M")},
-                       "copies_per_step": res["copies"], "path": res["path"], "cuda_graph": res["graph"],
-                       "l2": f"step rotates over {res['copies']} distinct weight sets "
+                       "copies_per_step": res["copies"], "rounds_per_step": res["rounds"],
+                       "calls_per_step": res["copies"] * res["rounds"], "path": res["path"], "cuda_graph": res["graph"],
+                       "l2": f"every round of a step rotates over {res['copies']} distinct weight sets "
                              f"({res['copies'] * algorithmic_bytes(c) / 1e6:.0f} MB > 2 x L2), no explicit flush",
                        "parallelism": "replicas" if world > 1 else "single"},
             "us_per_call": res["us_per_call"],

@@ -193,6 +193,17 @@ int lords_linear_forward_noalloc(const void *x, const uint8_t *Qpacked, const vo
  */
 int lords_poll_status(void *stream);
 
+/*
+ * Diagnosis of LORDS_ERR_TIMEOUT: reads and clears the record that the first device-side wait to run
+ * out left behind (host pointer to two 64-bit words; both zero if none ran out).
+ *   detail[0]: bit 63 set; bits 0..7 a tag naming the wait inside its kernel, bit 8 the phase parity
+ *              waited for, bits 16..23 the warp, bits 32..62 the CTA (blockIdx.x)
+ *   detail[1]: bits 0..31 the shared-memory address of the barrier, bits 32..63 how many rounds of
+ *              64 tries the wait made
+ * Synchronises the device.
+ */
+int lords_read_status_detail(uint64_t detail[2]);
+
 /* The cudaError_t (as int) of the most recent failed CUDA call, 0 if none. */
 int lords_last_cuda_error(void);
 

@@ -49,6 +49,7 @@ def _load():
         "lords_linear_forward_host": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_forward_noalloc": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_poll_status": (ci, [p]),
+        "lords_read_status_detail": (ci, [p]),
         "lords_last_cuda_error": (ci, []),
         "lords_set_option": (ci, [cs, cs]),
         "lords_last_path": (cs, []),
@@ -71,7 +72,7 @@ def exported_symbols():
     return ["lords_version", "lords_strerror", "lords_equivalent_rank", "lords_packed_bytes",
             "lords_pack_codes", "lords_unpack_codes", "lords_init", "lords_shutdown",
             "lords_linear_forward", "lords_linear_forward_bits", "lords_linear_forward_f32",
-            "lords_linear_forward_host", "lords_linear_forward_noalloc", "lords_poll_status", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
+            "lords_linear_forward_host", "lords_linear_forward_noalloc", "lords_poll_status", "lords_read_status_detail", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
             "lords_last_launch_count"]
 
 
@@ -185,6 +186,13 @@ def lords_linear_forward_noalloc(x, Qpacked, B, A, codebook, bits, M, m, n, r, y
 
 def lords_poll_status(stream=None) -> int:
     return int(_load().lords_poll_status(_stream_ptr(stream)))
+
+
+def lords_read_status_detail():
+    """The two 64-bit words of the first expired wait's record (both 0 if none), read and cleared."""
+    buf = (ctypes.c_uint64 * 2)()
+    _check(_load().lords_read_status_detail(ctypes.cast(buf, ctypes.c_void_p)), "lords_read_status_detail")
+    return int(buf[0]), int(buf[1])
 
 
 def lords_last_cuda_error() -> int:

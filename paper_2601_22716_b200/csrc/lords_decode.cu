@@ -28,7 +28,10 @@
 //   27     TMA producer of the factor tiles and of the k-step's slice of x (two tensor maps, one barrier).
 //
 // Every wait is bounded; on expiry the role records LORDS_ERR_TIMEOUT and leaves its loop, so
-// the kernel always reaches its final barrier and frees its TMEM.
+// the kernel always reaches its final barrier and frees its TMEM.  The waits carry tags for the
+// diagnostic record of the first wait that ran out: 1 code stage free, 2 factor stage free, 3 B operand
+// written, 4 W slot written, 5 factor tile and x landed, 6 W slot free, 7 code tile landed,
+// 8 accumulator complete, 9 partial sums received.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -257,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             tma_prefetch_desc(&p.tm_q);
             for (int it = 0; it < total; ++it) {
                 const int sq = it % SQ;
-                if (it >= SQ && !mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1), status)) { failed = true; break; }
+                if (it >= SQ && !mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1), status, 1)) { failed = true; break; }
                 const uint32_t bar = bar_q_full + 8 * sq;
                 mbar_expect_tx(bar, (uint32_t)C::QSTAGE);
                 tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (ks_a + it) * C::QROW, tile * kTileRows, bar);
@@ -322,7 +325,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             griddep_wait();   // x may be the previous launch's output
             for (int it = 0; it < pre; ++it) load_x(it);
             for (int it = S; it < total; ++it) {
-                if (!mbar_wait(bar_mma_done + 8 * (it % S), (uint32_t)((it / S - 1) & 1), status)) { failed = true; break; }
+                if (!mbar_wait(bar_mma_done + 8 * (it % S), (uint32_t)((it / S - 1) & 1), status, 2)) { failed = true; break; }
                 load_a(it);
                 load_x(it);
             }
@@ -345,8 +348,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         const int first = H == 2 ? 0 : j;
         for (int it = first; it < total; it += kStride) {
             const int s = it % S;
-            if (!mbar_wait(bar_ax_ready + 8 * s, (uint32_t)((it / S) & 1), status) ||
-                !mbar_wait(bar_ready + 8 * (h * S + s), (uint32_t)((it / S) & 1), status)) { failed = true; break; }
+            if (!mbar_wait(bar_ax_ready + 8 * s, (uint32_t)((it / S) & 1), status, 3) ||
+                !mbar_wait(bar_ready + 8 * (h * S + s), (uint32_t)((it / S) & 1), status, 4)) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)((h * S + s) * kWSlotCols);
@@ -370,7 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         constexpr int kRowIters = kNMax / kRowStep;            // 4
         for (int it = cgp; it < total; it += kConvGroups) {
             const int s = it % S;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full + 8 * s, (uint32_t)((it / S) & 1), status))) { failed = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full + 8 * s, (uint32_t)((it / S) & 1), status, 5))) { failed = true; break; }
 #pragma unroll
             for (int at = 0; at < kAtoms; ++at) {
                 const uint32_t atom = ax_stage(s) + at * kAtomBytes;
@@ -432,11 +435,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         for (int it = g; it < total; it += kGroups) {
             const int sq = it % SQ, s = it % S;
             // the W slot is free once the MMAs of step it - S have completed
-            if (it >= S && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1), status))) { failed = true; break; }
+            if (it >= S && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1), status, 6))) { failed = true; break; }
             tc_fence_after_sync();
 
             // codes -> levels -> TMEM
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1), status))) { failed = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1), status, 7))) { failed = true; break; }
             dequant_row_to_tmem<BITS, C::COLS>(q0 + sq * C::QSTAGE + row_in_tile * C::QROW, row_in_tile, ch, lut_lane,
                                       lane_addr + kWCol + (uint32_t)((h * S + s) * kWSlotCols));
             tmem_wait_st();
@@ -491,7 +494,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             for (int a = 0; a < kAccs; ++a) {
                 const int j = H == 2 ? h : a;
                 if (ok && j < total + (H == 2 ? 2 : 0)) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * j, 0, status));
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8 * j, 0, status, 8));
                     tc_fence_after_sync();
                     if (ok) {
 #pragma unroll
@@ -529,7 +532,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 for (int t = 0; t < NTOK; ++t)
                     st_async_cluster_f32(map_to_rank(red0 + ((rank * NTOK + t) * kTileRows + row_in_tile) * 4, 0), yt[t], leader_bar);
                 if (rank == 0) {
-                    if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0, status))) failed = true;
+                    if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0, status, 9))) failed = true;
                     else if (i < p.m) {
                         // all partials are read first (the loads overlap), then added in rank order
                         float v[NTOK][kClusterMax];

@@ -296,6 +296,17 @@ int lords_poll_status(void *stream)
     return word;
 }
 
+int lords_read_status_detail(uint64_t detail[2])
+{
+    State &st = state();
+    if (!detail) return LORDS_ERR_NULL;
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    LORDS_CUDA_TRY(cudaDeviceSynchronize());
+    LORDS_CUDA_TRY(cudaMemcpy(detail, st.status_word + 2, 2 * sizeof(uint64_t), cudaMemcpyDeviceToHost));
+    LORDS_CUDA_TRY(cudaMemset(st.status_word + 2, 0, 2 * sizeof(uint64_t)));
+    return LORDS_OK;
+}
+
 int lords_last_cuda_error(void) { return state().last_cuda_error; }
 
 int lords_set_option(const char *key, const char *value)

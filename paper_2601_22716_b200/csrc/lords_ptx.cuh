@@ -57,6 +57,9 @@ __device__ __forceinline__ unsigned long long global_ns()
 // whole grid instead of letting every wait run to its own limit.
 constexpr unsigned long long kWaitLimitNs = 50ull * 1000 * 1000;
 constexpr unsigned kWaitSleepNs = 40;
+// ... and that has really polled that long: a context that was merely descheduled for a while does not
+// count (rounds of 64 tries, each at least kWaitSleepNs apart)
+constexpr unsigned kWaitMinRounds = 64;
 struct WaitLimit {
     unsigned long long g0;
     unsigned rounds;
@@ -68,18 +71,30 @@ __device__ __forceinline__ WaitLimit wait_limit_start()
     w.rounds = 0;
     return w;
 }
-// called after every 64 unsuccessful tries; `status` is the library's device status word (may be null)
-__device__ __forceinline__ bool wait_limit_expired(WaitLimit &w, const int *status)
+// called after every 64 unsuccessful tries; `status` is the library's device status word (may be null).
+// The first wait of a grid that runs out by itself (not because the status word was already set) leaves
+// a record behind the status word, for diagnosis: {tag | parity << 8 | warp << 16 | CTA << 32,
+// barrier address | rounds of 64 tries << 32}.
+__device__ __forceinline__ bool wait_limit_expired(WaitLimit &w, const int *status, uint32_t bar, uint32_t parity, uint32_t tag)
 {
     ++w.rounds;
     if (status != nullptr && *reinterpret_cast<const volatile int *>(status) != 0) return true;
-    return w.rounds > 4u && global_ns() - w.g0 > kWaitLimitNs;
+    if (w.rounds > kWaitMinRounds && global_ns() - w.g0 > kWaitLimitNs) {
+        if (status != nullptr) {
+            unsigned long long *detail = reinterpret_cast<unsigned long long *>(const_cast<int *>(status) + 2);
+            const unsigned long long who = (unsigned long long)(tag & 0xFFu) | ((unsigned long long)(parity & 1u) << 8) |
+                                           ((unsigned long long)((threadIdx.x >> 5) & 0xFFu) << 16) | ((unsigned long long)blockIdx.x << 32);
+            if (atomicCAS(detail, 0ull, who | (1ull << 63)) == 0ull) detail[1] = (unsigned long long)bar | ((unsigned long long)w.rounds << 32);
+        }
+        return true;
+    }
+    return false;
 }
 
 // Bounded wait: gives up after kWaitLimitNs of polling (or as soon as the status word is set) and
 // reports failure, so that no role of a kernel can spin forever on a shared GPU.  Callers record
 // LORDS_ERR_TIMEOUT and drain.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const int *status = nullptr)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const int *status = nullptr, uint32_t tag = 0)
 {
     if (mbar_try_wait(bar, parity) || mbar_try_wait(bar, parity)) return true;
     // a waiting warp sleeps between its tries, so that it does not take issue slots from the warps
@@ -91,7 +106,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const i
             __nanosleep(kWaitSleepNs);
             if (mbar_try_wait(bar, parity)) return true;
         }
-        if (wait_limit_expired(limit, status)) return false;
+        if (wait_limit_expired(limit, status, bar, parity, tag)) return false;
     }
 }
 
@@ -288,7 +303,7 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     return ok != 0;
 }
 // Bounded like mbar_wait, with acquire at cluster scope (the arrivals come from other CTAs).
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const int *status = nullptr)
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const int *status = nullptr, uint32_t tag = 0)
 {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     WaitLimit limit = wait_limit_start();
@@ -298,7 +313,7 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
             __nanosleep(kWaitSleepNs);
             if (mbar_try_wait_cluster(bar, parity)) return true;
         }
-        if (wait_limit_expired(limit, status)) return false;
+        if (wait_limit_expired(limit, status, bar, parity, tag)) return false;
     }
 }
 
