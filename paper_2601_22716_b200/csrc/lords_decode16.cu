@@ -119,19 +119,7 @@ struct alignas(64) Dec16Params {
     void *y;
     int y_f32;
     int *status;
-#ifdef LORDS_TRACE
-    long long *trace;     // [8 roles][32 iterations][8 events] clock64 stamps of one CTA (debug builds only)
-#endif
 };
-
-#ifdef LORDS_TRACE
-#define XSTAMP(role, it, ev)                                                                         \
-    do {                                                                                             \
-        if (blockIdx.x == 0 && (it) < 32) p.trace[((role) * 32 + (it)) * 8 + (ev)] = clock64(); \
-    } while (0)
-#else
-#define XSTAMP(role, it, ev) do { } while (0)
-#endif
 
 // 64 columns of one row: code pairs -> level pairs, times the matching pairs of S (sp, in and out).
 // 4-bit rows are 64 bytes and arrive 64-byte-swizzled (16-byte chunk c of row i sits at chunk
@@ -219,7 +207,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
 
     bool failed = false;
     bool cluster_waited = false;      // this thread has taken the second half of the set-up cluster barrier
-    if (tid == 0) XSTAMP(7, 0, 0);
     if (!fits) {
         // the shared-memory window does not hold the layout (cannot happen with the window the host
         // asks for; checked because every address below depends on it)
@@ -254,7 +241,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                 const int sq = it % SQ;
                 if (it >= SQ && !mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1))) { failed = true; break; }
                 const uint32_t bar = bar_q_full + 8 * sq;
-                XSTAMP(3, it, 0);
                 mbar_expect_tx(bar, (uint32_t)C::QSTAGE);
                 tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (ks_a + it) * C::QROW, row0, bar);
             }
@@ -309,12 +295,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");   // see above
     }
     // let a dependent launch (the next layer) begin its own weight prefetch as SMs become free
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    griddep_launch_dependents();
     // Everything except the stream of packed codes waits here for the previous launch to finish: a CTA
     // that starts early sets up, prefetches its codes and then stands still.  (Letting the workers
     // run ahead of this point as well was tried; with it about one run in twenty of a 224-kernel
     // graph ended in device-side timeouts whose cause was not found.)
-    if (warp != kTmaQWarp) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (warp != kTmaQWarp) griddep_wait();
 
     if (warp == kTmaQWarp) {
         // all done above
@@ -341,9 +327,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         if (lane == 0) {
             // x may be the previous launch's output.  (This warp has already waited above with the
             // others; the wait is repeated where the dependency is.)
-            XSTAMP(6, 0, 3);
-            asm volatile("griddepcontrol.wait;" ::: "memory");
-            XSTAMP(6, 0, 4);
+            griddep_wait();
             for (int it = 0; it < total; ++it) {
                 const int sx = it % WS;
                 if (it >= WS && !mbar_wait(bar_mma_done + 8 * sx, (uint32_t)((it / WS - 1) & 1))) { failed = true; break; }
@@ -371,12 +355,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         if (b_by_tma && sj < total && !mbar_wait(bar_b_full, 0)) failed = true;
         for (int it = sj; it < total && !failed; it += 2) {
             const int sa = it % SA, sd = it % SD;
-            if (lane == 0) XSTAMP(4, it, 0);
             if (!mbar_wait(bar_a_full + 8 * sa, (uint32_t)((it / SA) & 1))) { failed = true; break; }
-            if (lane == 0) XSTAMP(4, it, 1);
             if (it >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((it / SD - 1) & 1))) { failed = true; break; }
             tc_fence_after_sync();
-            if (lane == 0) XSTAMP(4, it, 2);
             if (lane == 0) {
                 const uint32_t a_lo = a_lo0 + (uint32_t)(sa * (C::ASTAGE >> 4));
                 for (int k = 0; k < rsteps; ++k)
@@ -384,7 +365,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                                 umma_desc_pack(a_lo + k * 128, desc_hi), idesc_s, k > 0);
                 umma_commit(bar_s_full + 8 * sd);
                 umma_commit(bar_a_done + 8 * sa);
-                XSTAMP(4, it, 3);
             }
             __syncwarp();
         }
@@ -401,11 +381,9 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         const uint32_t acc = tmem_base + (uint32_t)(j * 32);
         for (int it = j; it < total; it += 2) {
             const int ws = it % WS;
-            if (j == 0 && lane == 0) XSTAMP(0, it, 0);
             if (!mbar_wait(bar_x_ready + 8 * ws, (uint32_t)((it / WS) & 1)) ||
                 !mbar_wait(bar_ready + 8 * ws, (uint32_t)((it / WS) & 1))) { failed = true; break; }
             tc_fence_after_sync();
-            if (j == 0 && lane == 0) XSTAMP(0, it, 1);
             if (lane == 0) {
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)(ws * 64);
                 const uint32_t x_lo = x_lo0 + (uint32_t)(ws * (kXStage >> 4));
@@ -415,7 +393,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                                 idesc_m, (it == j && k == 0) ? 0u : 1u);
                 umma_commit(bar_mma_done + 8 * ws);
                 if (it + 2 >= total) umma_commit(bar_acc_full + 8 * j);
-                if (j == 0) XSTAMP(0, it, 2);
             }
             __syncwarp();
         }
@@ -457,10 +434,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         const bool stamper = wg == 0 && lane == 0;
         for (int it = g; it < total; it += 2) {
             const int sq = it % SQ, sd = it % SD, ws = it % WS;
-            if (stamper) XSTAMP(1 + g, it, 0);
             if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * sd, (uint32_t)((it / SD) & 1)))) { failed = true; break; }
             tc_fence_after_sync();
-            if (stamper) XSTAMP(1 + g, it, 1);
             // this thread's 64 columns of S, as 32 fp16 pairs
             uint32_t sp[32];
 #pragma unroll
@@ -477,14 +452,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s_empty + 8 * sd);      // S is in registers: the buffer may be refilled
-            if (stamper) XSTAMP(1 + g, it, 2);
             if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1)))) { failed = true; break; }
-            if (stamper) XSTAMP(1 + g, it, 3);
             dequant_half_row<BITS>(q0 + sq * C::QSTAGE + row * C::QROW, row, ch, lut_lane, sp);
             // the W slot is free once the MMAs of step it - WS have completed
             if (it >= WS && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * ws, (uint32_t)((it / WS - 1) & 1)))) { failed = true; break; }
             tc_fence_after_sync();
-            if (stamper) XSTAMP(1 + g, it, 4);
             tmem_st_32x32(lane_addr + kWCol + (uint32_t)(ws * 64 + ch * 32), sp);
             tmem_wait_st();
             tc_fence_before_sync();
@@ -493,7 +465,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                 mbar_arrive(bar_ready + 8 * ws);
                 mbar_arrive(bar_q_empty + 8 * sq);
             }
-            if (stamper) XSTAMP(1 + g, it, 5);
         }
 
         // Epilogue (group 0, column half 0: one thread per row): the two accumulators -> this CTA's
@@ -509,7 +480,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
 #pragma unroll
             for (int t = 0; t < kTok; ++t) yt[t] = 0.0f;
             bool ok = true;
-            if (stamper) XSTAMP(5, 0, 0);
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 if (ok && j < total) {       // issuer j had a k-step
@@ -529,7 +499,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
 #pragma unroll
                 for (int t = 0; t < kTok; ++t) yt[t] = 0.0f;
             }
-            if (stamper) XSTAMP(5, 0, 1);
             if (csize == 1) {
                 if (ok && i < p.m)
 #pragma unroll
@@ -541,10 +510,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
 #pragma unroll
                 for (int t = 0; t < kTok; ++t)
                     st_async_cluster_f32(map_to_rank(red0 + (uint32_t)(((rank * kTok + t) * kRows + row) * 4), 0), yt[t], leader_bar);
-                if (stamper) XSTAMP(5, 0, 2);
                 if (rank == 0) {
                     const bool got = __all_sync(0xffffffffu, mbar_wait_cluster(bar_reduce, 0));
-                    if (stamper) XSTAMP(5, 0, 3);
                     if (!got) failed = true;
                     else if (i < p.m) {
                         // rank order for every token; the sixteen sums run side by side
@@ -559,17 +526,14 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                         for (int t = 0; t < kTok; ++t)
                             if (t < p.M) store_out(p.y, p.y_f32, (size_t)t * p.m + i, a[t]);
                     }
-                    if (stamper) XSTAMP(5, 0, 4);
                 }
             }
         }
     }
 
-    if (tid == 0) XSTAMP(7, 0, 1);
     if (failed) atomicExch(p.status, LORDS_ERR_TIMEOUT);
     tc_fence_before_sync();
     __syncthreads();
-    if (tid == 0) XSTAMP(7, 0, 2);
     if (warp == kIssuerWarp0) {
         tc_fence_after_sync();
         uint32_t tmem_base;
@@ -676,14 +640,14 @@ template <int BITS, int RP> int launch_variant(Dec16Params &k, const Problem &p,
 
 }  // namespace
 
-// Rules of this path: 3- or 4-bit codes; 3 <= M <= 16 (one or two tokens belong to the reassociated
-// decode kernel); r <= 32 (4-bit) or <= 64 (3-bit), which is what the shared-memory layout holds;
+// Rules of this path: 3- or 4-bit codes; M <= 16 (with automatic dispatch one or two tokens go to the
+// reassociated decode kernel first, and come here when that one declines the rank); r <= 32 (4-bit) or <= 64 (3-bit), which is what the shared-memory layout holds;
 // n a multiple of 64 (4-bit) or 128 (3-bit), which makes every TMA row pitch a multiple of 16 bytes.
 // Anything else: LORDS_ERR_UNSUPPORTED.
 int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
 {
     if (p.bits != 3 && p.bits != 4) return LORDS_ERR_UNSUPPORTED;
-    if (p.M < 3 || p.M > kTok) return LORDS_ERR_UNSUPPORTED;
+    if (p.M > kTok) return LORDS_ERR_UNSUPPORTED;
     if (p.r > (p.bits == 4 ? 32 : 64)) return LORDS_ERR_UNSUPPORTED;
     if (p.n % (p.bits == 4 ? 64 : 128) != 0) return LORDS_ERR_UNSUPPORTED;
 
@@ -695,10 +659,6 @@ int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
     k.ksteps = (p.n + kStep - 1) / kStep;
     k.y = p.y; k.y_f32 = p.y_f32;
     k.status = st.status_word;
-#ifdef LORDS_TRACE
-    k.trace = reinterpret_cast<long long *>(st.workspace + st.workspace_bytes - (size_t)8 * 32 * 8 * 8);
-    LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)8 * 32 * 8 * 8, stream));
-#endif
     int rc;
     if (p.bits == 4) rc = launch_variant<4, 32>(k, p, st, stream);
     else rc = k.r_pad <= 32 ? launch_variant<3, 32>(k, p, st, stream) : launch_variant<3, 64>(k, p, st, stream);

@@ -72,12 +72,13 @@ __device__ __forceinline__ WaitLimit wait_limit_start()
     return w;
 }
 // called after every 64 unsuccessful tries; `status` is the library's device status word (may be null).
-// The first wait of a grid that runs out by itself (not because the status word was already set) leaves
-// a record behind the status word, for diagnosis: {tag | parity << 8 | warp << 16 | CTA << 32,
-// barrier address | rounds of 64 tries << 32}.
+// Every 16th call (about every hundred microseconds of waiting) it looks at the status word and at the
+// clock.  The first wait of a grid that runs out by itself (not because the status word was already
+// set) leaves a record behind the status word, for diagnosis: {tag | parity << 8 | warp << 16 |
+// CTA << 32, barrier address | rounds of 64 tries << 32}.
 __device__ __forceinline__ bool wait_limit_expired(WaitLimit &w, const int *status, uint32_t bar, uint32_t parity, uint32_t tag)
 {
-    ++w.rounds;
+    if ((++w.rounds & 15u) != 0u) return false;
     if (status != nullptr && *reinterpret_cast<const volatile int *>(status) != 0) return true;
     if (w.rounds > kWaitMinRounds && global_ns() - w.g0 > kWaitLimitNs) {
         if (status != nullptr) {

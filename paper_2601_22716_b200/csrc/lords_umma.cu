@@ -87,22 +87,7 @@ struct alignas(64) UmmaParams {
     void *y;
     int y_f32;
     int *status;
-#ifdef LORDS_TRACE
-    long long *trace;     // [8 roles][32 iterations][8 events] clock64 stamps of one CTA (debug builds only)
-#endif
 };
-
-#ifdef LORDS_TRACE
-#ifndef LORDS_TRACE_CTA
-#define LORDS_TRACE_CTA 0
-#endif
-#define USTAMP(role, it, ev)                                                                         \
-    do {                                                                                             \
-        if (blockIdx.x == LORDS_TRACE_CTA && (it) < 32) p.trace[((role) * 32 + (it)) * 8 + (ev)] = clock64(); \
-    } while (0)
-#else
-#define USTAMP(role, it, ev) do { } while (0)
-#endif
 
 // The 32 columns (chunk c of the 128-column code stage) of one row: codes -> level pairs, times the
 // matching pairs of S, as 16 fp16x2 words.
@@ -255,13 +240,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             };
             issue_q(false);
             // x may be the previous launch's output
-            asm volatile("griddepcontrol.wait;" ::: "memory");
+            griddep_wait();
             for (int it = 0; it < total; ++it) {
                 const int sx = it % SX;
                 if (next_q <= (it >> 1) && !issue_q(true)) { failed = true; break; }   // the pair this k-step reads
                 if (it >= SX && !mbar_wait(bar_done + 8 * ((it - SX) % DR), (uint32_t)(((it - SX) / DR) & 1))) { failed = true; break; }
                 const uint32_t bar = bar_x_full + 8 * sx;
-                USTAMP(3, it, 0);
                 mbar_expect_tx(bar, (uint32_t)C::XTILE);
                 tma_load_2d(x0 + sx * C::XTILE, &p.tm_x, (2 * pa + it) * BK, tok0, bar);
                 issue_q(false);
@@ -309,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
     }
     // let a dependent launch begin its own weight prefetch as SMs become free
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    griddep_launch_dependents();
 
     if (warp == kTmaWarp) {
         // all done above
@@ -340,19 +324,16 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         const int ksteps = p.r_pad / 16;
         for (int j = 0; j < total; ++j) {
             const int sa = j % SA, sd = j % SD;
-            if (lane == 0) USTAMP(4, j, 0);
             if (!mbar_wait(bar_a_full + 8 * sa, (uint32_t)((j / SA) & 1))) { failed = true; break; }
             if (j >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((j / SD - 1) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
-                USTAMP(4, j, 1);
                 const uint32_t a_lo = a_lo0 + (uint32_t)(sa * (kATileBytes >> 4));
                 for (int k = 0; k < ksteps; ++k)
                     umma_f16_ss(tmem_base + C::SCOL + sd * 64, umma_desc_pack(b_lo + k * 2, desc_hi),
                                 umma_desc_pack(a_lo + k * 128, desc_hi), idesc_s, k > 0);
                 umma_commit(bar_s_full + 8 * sd);
                 umma_commit(bar_a_done + 8 * sa);
-                USTAMP(4, j, 2);
             }
             __syncwarp();
         }
@@ -365,13 +346,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         const uint32_t x_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((x0 & 0x3FFFFu) >> 4);
         for (int it = 0; it < total; ++it) {
             const int sx = it % SX, ws = it % WD;
-            if (lane == 0) USTAMP(0, it, 0);
             // W^ of the k-step is in TMEM and its activation tile has landed
             if (!mbar_wait(bar_w_full + 8 * ws, (uint32_t)((it / WD) & 1))) { failed = true; break; }
             if (!mbar_wait(bar_x_full + 8 * sx, (uint32_t)((it / SX) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
-                USTAMP(0, it, 2);
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)(ws * 32);
                 const uint32_t x_lo = x_lo0 + (uint32_t)((sx * C::XTILE) >> 4);
 #pragma unroll
@@ -380,7 +359,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                                 (it > 0 || k > 0) ? 1u : 0u);
                 umma_commit(bar_done + 8 * (it % DR));
                 if (it == total - 1) umma_commit(bar_acc_full);
-                USTAMP(0, it, 3);
             }
             __syncwarp();
         }
@@ -395,11 +373,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 
         for (int it = g; it < total; it += 2) {
             const int sx = it % SX, sd = it % SD, ws = it % WD, pr = it >> 1, sq = pr % SQ;
-            const bool stamper = wg == 0 && lane == 0;
-            if (stamper) USTAMP(1 + g, it, 0);
             if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * sd, (uint32_t)((it / SD) & 1)))) { failed = true; break; }
             tc_fence_after_sync();
-            if (stamper) USTAMP(1 + g, it, 1);
             uint32_t s[32];
             tmem_ld_32x32(lane_addr + C::SCOL + (uint32_t)(sd * 64 + ch * 32), s);
             bool ok = mbar_wait(bar_q_full + 8 * sq, (uint32_t)((pr / SQ) & 1));
@@ -408,7 +383,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s_empty + 8 * sd);      // S is in registers: the buffer may be refilled
             if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-            if (stamper) USTAMP(1 + g, it, 2);
             uint32_t out[16];
             dequant_chunk<BITS>(q0 + sq * C::QSTAGE + row * C::QROW, row, (it & 1) * 2 + ch, lut_lane, s, out);
             if constexpr (C::kConvertInKernel) {
@@ -435,7 +409,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 break;
             }
             tc_fence_after_sync();
-            if (stamper) USTAMP(1 + g, it, 3);
             tmem_st_32x16(lane_addr + kWCol + (uint32_t)(ws * 32 + ch * 16), out);
             tmem_wait_st();
             tc_fence_before_sync();
@@ -444,7 +417,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 mbar_arrive(bar_w_full + 8 * ws);
                 mbar_arrive(bar_q_empty + 8 * sq);
             }
-            if (stamper) USTAMP(1 + g, it, 4);
         }
 
         // ------------------------------------------------------------------ epilogue
@@ -727,10 +699,6 @@ int launch_umma(const Problem &p, State &st, cudaStream_t stream)
     k.npairs = (p.n + 127) / 128;
     k.y = p.y; k.y_f32 = p.y_f32;
     k.status = st.status_word;
-#ifdef LORDS_TRACE
-    k.trace = reinterpret_cast<long long *>(st.workspace + st.workspace_bytes - (size_t)8 * 32 * 8 * 8);
-    LORDS_CUDA_TRY(cudaMemsetAsync(k.trace, 0, (size_t)8 * 32 * 8 * 8, stream));
-#endif
     const int rc = p.bits == 4 ? launch_bits<4>(k, p, st, stream) : launch_bits<3>(k, p, st, stream);
     if (rc != LORDS_OK) return rc;
     st.last_path = "umma";

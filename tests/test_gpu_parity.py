@@ -148,6 +148,13 @@ def test_decode_kernel_cluster_split_is_deterministic(lords, cluster):
     check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
 
 
+def test_two_tokens_with_a_large_rank_take_the_128_column_kernel(lords):
+    lay = gen.make_layer(512, 1024, 48, 2, bits=3, seed=5)       # 2 * 48 accumulator columns: too many for the reassociated form
+    dl, y32, ybf = _run(lords, lay, "auto")
+    assert lords.lords_last_path() == "decode16"
+    check_against_oracle(y32, ybf, _oracle(lay, dl.packed_host))
+
+
 def test_decode_kernel_declines_what_it_cannot_run(lords):
     lay = gen.make_layer(256, 256, 4, 4, bits=4, seed=0)      # M = 4, r = 4
     lords.lords_set_option("path", "decode")
@@ -173,6 +180,8 @@ DECODE16_SHAPES = [
     (3, 260, 1152, 48, 16, True),
     (3, 256, 128, 16, 3, False),
     (3, 2048, 4096, 32, 8, False),
+    (3, 640, 2048, 48, 2, True),      # two tokens with a rank the reassociated kernel declines
+    (4, 256, 512, 32, 1, False),
 ]
 
 
@@ -216,8 +225,7 @@ def test_decode16_kernel_cluster_split_is_deterministic(lords, cluster):
 def test_decode16_kernel_declines_what_it_cannot_run(lords):
     lords.lords_set_option("path", "decode16")
     try:
-        for lay in (gen.make_layer(256, 256, 4, 2, bits=4, seed=0),       # two tokens: the other decode kernel's
-                    gen.make_layer(256, 256, 48, 4, bits=4, seed=0),      # 4-bit with r > 32
+        for lay in (gen.make_layer(256, 256, 48, 4, bits=4, seed=0),      # 4-bit with r > 32
                     gen.make_layer(256, 256, 4, 17, bits=4, seed=0)):     # more than one token tile
             with pytest.raises(lords.LordsError) as ei:
                 DeviceLayer(lay).forward()
