@@ -48,6 +48,8 @@ def _load():
         lib.lords_oracle_forward.argtypes = [p, p, p, p, p, ci, i64, i64, i64, i64, p, i64, p, ci]
         lib.lords_oracle_round_bf16.restype = None
         lib.lords_oracle_round_bf16.argtypes = [p, i64, p]
+        lib.lords_oracle_quantize.restype = ci
+        lib.lords_oracle_quantize.argtypes = [p, p, p, p, ci, i64, i64, i64, p, p, p, p]
         lib.lords_oracle_equivalent_rank.restype = i64
         lib.lords_oracle_equivalent_rank.argtypes = [i64, i64, i64]
         _lib = lib
@@ -140,3 +142,26 @@ def round_bf16(v: np.ndarray) -> np.ndarray:
 
 def equivalent_rank(rows: int, cols: int, blk: int) -> int:
     return int(_load().lords_oracle_equivalent_rank(rows, cols, blk))
+
+
+def quantize(W, B, A, codebook, bits: int, details: bool = False):
+    """Alg. 1 step 2.1: codes uint8 [m, n] = argmin_c (S * L[c] - W)^2 with S = B A, lowest code on ties.
+    W, B, A are bf16 bit patterns.  With details=True also returns (runner-up codes, gap, magnitude)."""
+    W = _c(W, np.uint16); B = _c(B, np.uint16); A = _c(A, np.uint16); codebook = _c(codebook, np.float32)
+    m, n = W.shape
+    r = B.shape[1]
+    assert B.shape == (m, r) and A.shape == (r, n) and codebook.size == 2**bits
+    codes = np.empty((m, n), dtype=np.uint8)
+    if details:
+        runner = np.empty((m, n), dtype=np.uint8)
+        gap = np.empty((m, n), dtype=np.float64)
+        mag = np.empty((m, n), dtype=np.float64)
+        rc = _load().lords_oracle_quantize(_ptr(W), _ptr(B), _ptr(A), _ptr(codebook), bits, m, n, r,
+                                           _ptr(codes), _ptr(runner), _ptr(gap), _ptr(mag))
+    else:
+        rc = _load().lords_oracle_quantize(_ptr(W), _ptr(B), _ptr(A), _ptr(codebook), bits, m, n, r,
+                                           _ptr(codes), None, None, None)
+    if rc != 0:
+        raise ValueError(f"oracle quantize failed: {rc}")
+    return (codes, runner, gap, mag) if details else codes
+

@@ -31,6 +31,13 @@
  * closed-form answer, pack known-answer bytes, and the rank rule of Table 7.
  * Not pinned: a forward output on real model weights -- the paper prints no
  * worked numeric example of the forward path ("parity unpinned" for that only).
+ *
+ * The step before the path, the quantisation step of Alg. 1 (step 2.1), is stated here too
+ * (lords_oracle_quantize): Q_ij = argmin over the levels v of (S_ij v - W_ij)^2 with S = BA, every
+ * level tried in turn in fp64.  The paper does not say which level wins a tie: the lowest code does.
+ * Pins: the codes of an exactly representable W^ are recovered; no other level has a smaller error
+ * (an independent array-wise check); exact midpoints go to the lower code; negating S and W together
+ * changes nothing; for S > 0 the code does not decrease as W grows.
  */
 #include <math.h>
 #include <stdint.h>
@@ -234,3 +241,57 @@ int64_t lords_oracle_equivalent_rank(int64_t rows, int64_t cols, int64_t blk)
     if (rows < 1 || cols < 1 || blk < 1) return ORACLE_ERR_ARG;
     return (rows * cols) / (blk * (rows + cols));
 }
+
+/*
+ * Quantisation step (Alg. 1, step 2.1; Sec. 3.3 "nearest-neighbor search in the look-up table"):
+ *   Q_ij = argmin_{c} (S_ij * L[c] - W_ij)^2,  S = B A (Eq. 3),  ties -> the lowest code.
+ * W, B, A are bf16 bit patterns (W: m x n), widened exactly; all arithmetic fp64.
+ *   codes_out  : m*n bytes, one code per byte
+ *   runner_out : (may be NULL) the best code among the others (lowest code on ties)
+ *   gap_out    : (may be NULL) |S L[runner] - W| - |S L[best] - W| >= 0: by how much the choice was clear
+ *   mag_out    : (may be NULL) |S| * max|L| + |W|: the magnitude the gap is to be compared with
+ */
+int lords_oracle_quantize(const uint16_t *W, const uint16_t *B, const uint16_t *A, const float *codebook, int bits,
+                          int64_t m, int64_t n, int64_t r, uint8_t *codes_out, uint8_t *runner_out, double *gap_out,
+                          double *mag_out)
+{
+    if (!W || !B || !A || !codebook || !codes_out || m < 0 || n < 0 || r < 1) return ORACLE_ERR_ARG;
+    if (bits != 2 && bits != 3 && bits != 4) return ORACLE_ERR_ARG;
+    const int levels = 1 << bits;
+    double lmax = 0.0;
+    for (int c = 0; c < levels; ++c)
+        if (fabs((double)codebook[c]) > lmax) lmax = fabs((double)codebook[c]);
+    int rc = ORACLE_OK;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < m; ++i) {
+        double *S_row = (double *)malloc((size_t)(n > 0 ? n : 1) * sizeof(double));
+        if (!S_row) {
+#pragma omp critical
+            rc = ORACLE_ERR_NOMEM;
+            continue;
+        }
+        scale_row(B, A, n, r, i, S_row);
+        for (int64_t j = 0; j < n; ++j) {
+            const double w = bf16_to_f64(W[i * n + j]);
+            int best = -1, runner = -1;
+            double e_best = 0.0, e_runner = 0.0;
+            for (int c = 0; c < levels; ++c) {
+                const double d = S_row[j] * (double)codebook[c] - w;
+                const double e = d * d;
+                if (best < 0 || e < e_best) {
+                    runner = best; e_runner = e_best;
+                    best = c; e_best = e;
+                } else if (runner < 0 || e < e_runner) {
+                    runner = c; e_runner = e;
+                }
+            }
+            codes_out[i * n + j] = (uint8_t)best;
+            if (runner_out) runner_out[i * n + j] = (uint8_t)runner;
+            if (gap_out) gap_out[i * n + j] = sqrt(e_runner) - sqrt(e_best);
+            if (mag_out) mag_out[i * n + j] = fabs(S_row[j]) * lmax + fabs(w);
+        }
+        free(S_row);
+    }
+    return rc;
+}
+

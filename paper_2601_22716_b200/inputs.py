@@ -196,3 +196,14 @@ def make_integer_layer(m: int, n: int, r: int, M: int, bits: int = 4, seed: int 
         xf[t, cols] = vals[torch.randint(0, 4, (nnz_per_token,), generator=g)]
     return LayerInputs(m=m, n=n, r=r, M=M, bits=bits, codes=codes, B=bf16_bits(Bf), A=bf16_bits(Af),
                        x=bf16_bits(xf), codebook=int_codebook(bits), meta={"seed": seed, "integer": True})
+
+
+def make_weight(m: int, n: int, seed: int = 0, *, sigma: float = 0.05) -> np.ndarray:
+    """A weight matrix to quantise: bf16 bit patterns of N(0, sigma^2), m x n (out x in).
+
+    With the scale factors of ``make_layer`` (S = B*A around 0.1 for r = 32) the ratios W / S spread over
+    and a little beyond the level range [-1, 1], as weights divided by their block scales do.
+    """
+    g = _gen(seed)
+    return bf16_bits(torch.randn(m, n, generator=g) * sigma)
+

@@ -236,3 +236,71 @@ def test_nf_codebook_properties(bits):
     assert cb[0] == -1.0 and cb[-1] == 1.0
     assert np.count_nonzero(cb == 0.0) == 1
     assert np.count_nonzero(cb < 0) == 2 ** (bits - 1) - 1 and np.count_nonzero(cb > 0) == 2 ** (bits - 1)
+
+
+# ---------------------------------------------------------------- quantisation step (Alg. 1, step 2.1)
+
+def test_quantize_recovers_the_codes_of_a_representable_weight():
+    """W = L[Q] * S exactly (small integers everywhere): the error of the true code is zero and every
+    other level is off by at least |S|, so the codes come back -- except where S = 0, where every level
+    ties and the lowest code wins."""
+    import torch
+    lay = gen.make_integer_layer(48, 96, 5, 1, bits=4, seed=3)
+    S = _f64(lay.B) @ _f64(lay.A)
+    S[::7, ::5] = 0.0                                   # some exact zeros in S: knock out the rows of B that feed them
+    Bz = _f64(lay.B).copy()
+    Bz[::7, :] = 0.0
+    S = Bz @ _f64(lay.A)
+    W = lay.codebook.astype(np.float64)[lay.codes] * S
+    Wb = gen.bf16_bits(torch.from_numpy(W.astype(np.float32)))
+    assert np.array_equal(_f64(Wb), W)                  # representable: nothing was rounded
+    got = oracle.quantize(Wb, gen.bf16_bits(torch.from_numpy(Bz.astype(np.float32))), lay.A, lay.codebook, 4)
+    want = np.where(S != 0.0, lay.codes, 0)
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("bits,r,mixed", [(4, 7, True), (3, 16, False), (2, 3, True)])
+def test_quantize_is_the_array_wise_argmin(bits, r, mixed):
+    """Independent statement with library routines: S by a matmul, the errors of all levels as one
+    array, numpy's argmin (which returns the first, i.e. lowest, index of the minimum)."""
+    lay = gen.make_layer(40, 64, r, 1, bits=bits, seed=11 + bits, mixed_sign=mixed)
+    Wb = gen.make_weight(40, 64, seed=5 + bits)
+    S = _f64(lay.B) @ _f64(lay.A)
+    E = (S[:, :, None] * lay.codebook.astype(np.float64)[None, None, :] - _f64(Wb)[:, :, None]) ** 2
+    codes, runner, gap, mag = oracle.quantize(Wb, lay.B, lay.A, lay.codebook, bits, details=True)
+    clear = gap > 1e-12 * mag                            # the two summation orders may differ in the last bits
+    assert clear.mean() > 0.999
+    assert np.array_equal(codes[clear], E.argmin(axis=2)[clear])
+    assert (gap >= 0).all() and (runner != codes).all()
+
+
+def test_quantize_ties_go_to_the_lower_code_and_signs_cancel():
+    import torch
+    levels = gen.int_codebook(3)                         # -4 .. 3
+    n = 32
+    B1 = gen.bf16_bits(torch.ones(1, 1))
+    A1 = gen.bf16_bits(torch.full((1, n), 2.0))          # S = 2 everywhere
+    mids = (levels[:-1] + levels[1:]) / 2.0              # exact midpoints between neighbouring levels
+    w = np.zeros((1, n), dtype=np.float32)
+    w[0, :mids.size] = 2.0 * mids                        # W / S on a midpoint: both neighbours are equally far
+    w[0, mids.size:mids.size + 2] = [100.0, -100.0]      # far outside the table: the end levels
+    Wb = gen.bf16_bits(torch.from_numpy(w))
+    got = oracle.quantize(Wb, B1, A1, levels, 3)
+    assert np.array_equal(got[0, :mids.size], np.arange(mids.size))            # the lower of the two codes
+    assert got[0, mids.size] == 7 and got[0, mids.size + 1] == 0
+    # S < 0: the products S * L[c] run downwards, ties still go to the lower code
+    Bn = gen.bf16_bits(-torch.ones(1, 1))
+    gotn = oracle.quantize(gen.bf16_bits(torch.from_numpy(-w)), Bn, A1, levels, 3)
+    assert np.array_equal(gotn, got)                     # (-S) * v - (-W) = -(S v - W): same errors
+
+
+def test_quantize_is_monotone_in_the_weight_for_positive_scales():
+    import torch
+    lay = gen.make_layer(8, 64, 4, 1, bits=4, seed=2)     # positive B, A
+    base = np.linspace(-0.2, 0.2, 8 * 64, dtype=np.float32).reshape(8, 64)
+    cols = np.sort(base, axis=0)                         # every column increases down the rows ...
+    Bsame = np.repeat(lay.B[:1], 8, axis=0)              # ... while S is the same in all rows
+    got = oracle.quantize(gen.bf16_bits(torch.from_numpy(cols)), Bsame, lay.A, lay.codebook, 4)
+    assert (np.diff(got.astype(np.int32), axis=0) >= 0).all()
+    assert got.min() == 0 and got.max() == 15            # the grid reaches both ends of the table
+
