@@ -162,6 +162,23 @@ int lords_linear_forward_host(const void *x_host, const uint8_t *Qpacked, const 
                               void *stream);
 
 /*
+ * Quantisation step of the alternating refinement (Alg. 1, step 2.1; Sec. 3.3): with the factors fixed,
+ *     Q_ij = argmin over the codes c of (S_ij * L[c] - W_ij)^2,   S = B A (Eq. 3),
+ * written as packed codes in the layout above (ready for the forward calls).  The paper does not say
+ * which level wins a tie: the lowest code does.  S is accumulated in fp32 and every level is tried in
+ * fp32, so a weight within rounding distance of the midpoint between two levels' products may get
+ * either neighbour.
+ *   W        : device, bf16 [m][n], the weight to quantise (out-features x in-features)
+ *   B, A     : device, bf16 [m][r] and [r][n]
+ *   codebook : HOST, 2^bits floats (ascending or not: codes index it as given)
+ *   Qpacked  : device, lords_packed_bytes(m, n, bits) bytes, fully overwritten
+ * Ranges as for the forward calls (n a multiple of the pack group); needs lords_init; enqueues on
+ * `stream` and returns without synchronising.
+ */
+int lords_quantize_codes(const void *W, const void *B, const void *A, const float *codebook, int bits, int m, int n,
+                         int r, uint8_t *Qpacked, void *stream);
+
+/*
  * Allocation-free forward (the paper has no counterpart: this is a deployment convenience).
  * For callers that must not allocate device memory -- for instance a plugin inside a server
  * whose memory pool already owns all of HBM, or a latency-critical loop that cannot take the
@@ -218,7 +235,8 @@ int lords_last_cuda_error(void);
  */
 int lords_set_option(const char *key, const char *value);
 
-/* Name of the path the most recent forward call dispatched to ("simt", "decode", "decode16", "umma"). */
+/* Name of the path the most recent call dispatched to ("simt", "decode", "decode16", "umma"; "quantize",
+ * "quantize_simt" for lords_quantize_codes). */
 const char *lords_last_path(void);
 
 /* Number of kernels the most recent forward call launched. */

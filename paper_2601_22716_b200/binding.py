@@ -48,6 +48,7 @@ def _load():
         "lords_linear_forward_f32": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_forward_host": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_forward_noalloc": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
+        "lords_quantize_codes": (ci, [p, p, p, p, ci, ci, ci, ci, p, p]),
         "lords_poll_status": (ci, [p]),
         "lords_read_status_detail": (ci, [p]),
         "lords_last_cuda_error": (ci, []),
@@ -72,7 +73,7 @@ def exported_symbols():
     return ["lords_version", "lords_strerror", "lords_equivalent_rank", "lords_packed_bytes",
             "lords_pack_codes", "lords_unpack_codes", "lords_init", "lords_shutdown",
             "lords_linear_forward", "lords_linear_forward_bits", "lords_linear_forward_f32",
-            "lords_linear_forward_host", "lords_linear_forward_noalloc", "lords_poll_status", "lords_read_status_detail", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
+            "lords_linear_forward_host", "lords_linear_forward_noalloc", "lords_quantize_codes", "lords_poll_status", "lords_read_status_detail", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
             "lords_last_launch_count"]
 
 
@@ -182,6 +183,13 @@ def lords_linear_forward_noalloc(x, Qpacked, B, A, codebook, bits, M, m, n, r, y
     _check(_load().lords_linear_forward_noalloc(x.data_ptr(), Qpacked.data_ptr(), B.data_ptr(), A.data_ptr(),
                                                 cb.ctypes.data, bits, M, m, n, r, y.data_ptr(),
                                                 _stream_ptr(stream)), "lords_linear_forward_noalloc")
+
+
+def lords_quantize_codes(W, B, A, codebook, bits, m, n, r, Qpacked, stream=None) -> None:
+    """Alg. 1 step 2.1 on the device: packed codes of the nearest levels of W / (B A)."""
+    cb = _cb_ptr(codebook, bits)
+    _check(_load().lords_quantize_codes(W.data_ptr(), B.data_ptr(), A.data_ptr(), cb.ctypes.data, bits, m, n, r,
+                                        Qpacked.data_ptr(), _stream_ptr(stream)), "lords_quantize_codes")
 
 
 def lords_poll_status(stream=None) -> int:

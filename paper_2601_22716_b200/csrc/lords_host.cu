@@ -284,6 +284,20 @@ int lords_linear_forward_host(const void *x_host, const uint8_t *Qpacked, const 
     return LORDS_OK;
 }
 
+int lords_quantize_codes(const void *W, const void *B, const void *A, const float *codebook, int bits, int m, int n,
+                         int r, uint8_t *Qpacked, void *stream)
+{
+    if (!W || !B || !A || !codebook || !Qpacked) return LORDS_ERR_NULL;
+    const int g = pack_group(bits);
+    if (g == 0) return LORDS_ERR_BITS;
+    if (m < 1 || n < 1 || r < 1 || r > LORDS_R_MAX || n % g != 0) return LORDS_ERR_SHAPE;
+    if (!aligned16(W) || !aligned16(B) || !aligned16(A) || !aligned16(Qpacked)) return LORDS_ERR_ALIGN;
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    st.last_launches = 0;
+    return launch_quantize(W, B, A, codebook, bits, m, n, r, Qpacked, st, static_cast<cudaStream_t>(stream));
+}
+
 int lords_poll_status(void *stream)
 {
     State &st = state();

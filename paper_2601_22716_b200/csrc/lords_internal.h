@@ -69,4 +69,8 @@ int launch_decode(const Problem &p, State &st, cudaStream_t stream);
 // LORDS_ERR_UNSUPPORTED for shapes outside its rules.
 int launch_decode16(const Problem &p, State &st, cudaStream_t stream);
 
+// Quantisation step (codes from W, B, A): tensor-core kernel where its rules hold, CUDA cores otherwise.
+int launch_quantize(const void *W, const void *B, const void *A, const float *levels, int bits, int m, int n, int r,
+                    uint8_t *Q, State &st, cudaStream_t stream);
+
 }  // namespace lords
