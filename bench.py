@@ -298,8 +298,13 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
         roof = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8TBs": gbs / 8000.0}
     else:
-        roof = {"bound": "tensor", "achieved": tfs, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": tfs / peaks["bf16_tflops"], "frac_of_sustained": tfs / peaks["bf16_tflops_sustained"],
+        # the kernel is timed inside a loop of about a second: the matching denominator is the library GEMM
+        # measured the same way (sustained under the power cap); a loop far shorter takes the burst figure
+        long_loop = ms_per_step * steps >= 300.0
+        peak = peaks["bf16_tflops_sustained"] if long_loop else peaks["bf16_tflops"]
+        roof = {"bound": "tensor", "achieved": tfs, "peak": peak, "unit": "TFLOP/s",
+                "peak_kind": "sustained" if long_loop else "burst", "frac": tfs / peak,
+                "frac_of_burst": tfs / peaks["bf16_tflops"], "frac_of_sustained": tfs / peaks["bf16_tflops_sustained"],
                 "frac_of_nominal_2.25PF": tfs / 2250.0}
     roof["peak_source"] = peaks["source"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(case)
@@ -394,6 +399,64 @@ def time_stack(M, mlp_bits, steps, device):
     return {"case": f"stack_m{M}_mlp{mlp_bits}bit", "ms_per_pass": ms, "ms_per_token": ms / M, "calls": len(calls),
             "algorithmic_bytes": byt, "gbs": gbs, "tflops": tfs, "frac_hbm": gbs / peaks["hbm_gbs"],
             "frac_tensor": tfs / peaks["bf16_tflops"], "steps": steps, "status_retries": status_retries}
+
+
+def time_quantize(name, m, n, r, bits, device, min_seconds=0.3):
+    """The step before the path (Alg. 1, step 2.1): weights -> packed codes on the device.  HBM-bound:
+    algorithmic bytes = W (bf16) + packed codes + B + A, each moved once."""
+    import numpy as np
+    import torch
+    from paper_2601_22716_b200 import binding as lords
+    from paper_2601_22716_b200 import inputs as gen
+
+    lay = gen.make_layer(m, n, r, 1, bits=bits, seed=0)
+    byt = 2 * m * n + m * n * bits // 8 + 2 * r * (m + n)
+    copies = max(2, -(-2 * L2_BYTES // byt) + 1)
+    W0 = torch.from_numpy(gen.make_weight(m, n, seed=1).view(np.int16)).to(device)
+    B0 = torch.from_numpy(lay.B.view(np.int16)).to(device)
+    A0 = torch.from_numpy(lay.A.view(np.int16)).to(device)
+    sets = [(torch.roll(W0, l, 0).contiguous(), torch.roll(B0, l, 0).contiguous(), A0.clone(),
+             torch.empty(m * n * bits // 8, dtype=torch.uint8, device=device)) for l in range(copies)]
+
+    def one_round():
+        for W, B, A, Q in sets:
+            lords.lords_quantize_codes(W, B, A, lay.codebook, bits, m, n, r, Q)
+
+    one_round()
+    torch.cuda.synchronize()
+    path = lords.lords_last_path()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        one_round()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        one_round()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    reps = int(max(3, min_seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)))
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / reps / copies
+    status = lords.lords_poll_status()
+    peaks = measured_peaks()
+    gbs = byt / (us * 1e-6) / 1e9
+    return {"case": name, "path": path, "us_per_call": us, "gbs": gbs, "tflops": None, "copies": copies, "rounds": reps,
+            "steps": 1, "status_retries": 0 if status == 0 else 1,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                         "algorithmic_bytes_per_launch": byt, "us_per_launch": us}}
 
 
 def run_sweep(device):
@@ -571,6 +634,10 @@ def main():
             cases.append({"case": name, "path": r2["path"], "us_per_call": r2["us_per_call"],
                           "gbs": r2["gbs"], "tflops": r2["tflops"], "roofline": r2["roofline"],
                           "copies": r2["copies"], "rounds": r2["rounds"], "steps": k, "status_retries": r2["status_retries"]})
+
+    if not args.case and not args.no_extras and world == 1:
+        cases.append(time_quantize("quantize_q_nf4", 4096, 4096, 32, 4, device))
+        cases.append(time_quantize("quantize_gate_nf3", 14336, 4096, 48, 3, device))
 
     stack = []
     if not args.no_stack and not args.no_extras and not args.case and world == 1:

@@ -199,14 +199,24 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
     // mbarriers, 8 bytes each, in one run so that a warp can initialise them lane-parallel
     constexpr int kBarQFull = 0;                            // SQ, 1 arrival + TMA bytes
     constexpr int kBarQEmpty = kBarQFull + SQ;              // SQ, the warps of one group
-    constexpr int kBarAFull = kBarQEmpty + SQ;              // S, 1 arrival + TMA bytes
-    constexpr int kBarAxReady = kBarAFull + S;              // S: the warps of one converter group (B operand written)
+    // A barrier is waited on by parity alone, so whoever waits for its phase n must know that phase
+    // n - 1 has completed.  A warp that waits for every phase of a barrier knows; so does a group that
+    // owns the barrier.  The converter groups take the k-steps alternately: with an odd ring depth a
+    // stage would change hands every time round, and a group that polls "stage s, second filling"
+    // while the first filling (the other group's) is still in flight would see the phase it waits
+    // for as already complete.  The "factor tile landed" barriers are therefore indexed by the k-step
+    // modulo a multiple of the group count, which gives every barrier one owner; so are the "MMAs of
+    // the k-step done" barriers, which the worker groups wait on alternately.
+    constexpr int kAF = S % kConvGroups == 0 ? S : S * kConvGroups;
+    constexpr int kBarAFull = kBarQEmpty + SQ;              // kAF, 1 arrival + TMA bytes
+    constexpr int kBarAxReady = kBarAFull + kAF;            // S: the warps of one converter group (B operand written)
     constexpr int kBarReady = kBarAxReady + S;              // H * S: the warps of one worker group (W slot written)
-    constexpr int kBarMmaDone = kBarReady + H * S;          // S, one commit per half
-    constexpr int kBarAccFull = kBarMmaDone + S;            // 2: one per issuer
+    constexpr int kBarMmaDone = kBarReady + H * S;          // kAF, one commit per half
+    constexpr int kBarAccFull = kBarMmaDone + kAF;          // 2: one per issuer
     constexpr int kBarReduce = kBarAccFull + 2;             // 1: counts the bytes of the cluster's partial sums (leader's copy is used)
     constexpr int kBarCount = kBarReduce + 1;
     static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
+    static_assert(SQ % kGroups == 0, "one worker group per code-ring barrier");
     const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
     const uint32_t bar_a_full = bars + 8 * kBarAFull, bar_ax_ready = bars + 8 * kBarAxReady, bar_ready = bars + 8 * kBarReady;
     const uint32_t bar_mma_done = bars + 8 * kBarMmaDone, bar_acc_full = bars + 8 * kBarAccFull;
@@ -260,7 +270,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             tma_prefetch_desc(&p.tm_q);
             for (int it = 0; it < total; ++it) {
                 const int sq = it % SQ;
-                if (it >= SQ && !mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1), status, 1)) { failed = true; break; }
+                if (it >= SQ) {
+                    // a stage is freed by work that stands behind the dependency point: pass it first, so that
+                    // the bounded wait does not run while the previous launch (however long) still works
+                    if (it == SQ) griddep_wait();
+                    if (!mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1), status, 1)) { failed = true; break; }
+                }
                 const uint32_t bar = bar_q_full + 8 * sq;
                 mbar_expect_tx(bar, (uint32_t)C::QSTAGE);
                 tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (ks_a + it) * C::QROW, tile * kTileRows, bar);
@@ -309,7 +324,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             // one barrier per stage counts the bytes of the factor tile and of the x slice
             auto load_a = [&](int it) {
                 const int s = it % S, j0 = (ks_a + it) * kStep;
-                const uint32_t bar = bar_a_full + 8 * s;
+                const uint32_t bar = bar_a_full + 8 * (it % kAF);
                 mbar_expect_tx(bar, tx_a + (uint32_t)(NTOK * kStep * 2));
 #pragma unroll
                 for (int at = 0; at < kAtoms; ++at)
@@ -317,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             };
             auto load_x = [&](int it) {
                 const int s = it % S;
-                tma_load_2d(xs0 + s * C::XSTAGE, &p.tm_x, (ks_a + it) * kStep, 0, bar_a_full + 8 * s);
+                tma_load_2d(xs0 + s * C::XSTAGE, &p.tm_x, (ks_a + it) * kStep, 0, bar_a_full + 8 * (it % kAF));
             };
             // the factors are weights: the first stages are filled before the dependency point
             const int pre = total < S ? total : S;
@@ -325,7 +340,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
             griddep_wait();   // x may be the previous launch's output
             for (int it = 0; it < pre; ++it) load_x(it);
             for (int it = S; it < total; ++it) {
-                if (!mbar_wait(bar_mma_done + 8 * (it % S), (uint32_t)((it / S - 1) & 1), status, 2)) { failed = true; break; }
+                if (!mbar_wait(bar_mma_done + 8 * ((it - S) % kAF), (uint32_t)(((it - S) / kAF) & 1), status, 2)) { failed = true; break; }
                 load_a(it);
                 load_x(it);
             }
@@ -358,7 +373,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
                 for (int k = 0; k < kStep / 16; ++k)
                     umma_f16_ts(acc, wslot + k * 8, umma_desc_pack(b_lo + (k >> 2) * (kAtomBytes >> 4) + (k & 3) * 2, desc_hi),
                                 idesc, (it == first && k == 0) ? 0u : 1u);
-                umma_commit(bar_mma_done + 8 * s);
+                umma_commit(bar_mma_done + 8 * (it % kAF));
                 if (it + kStride >= total) umma_commit(bar_acc_full + 8 * j);
             }
             __syncwarp();
@@ -373,7 +388,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         constexpr int kRowIters = kNMax / kRowStep;            // 4
         for (int it = cgp; it < total; it += kConvGroups) {
             const int s = it % S;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full + 8 * s, (uint32_t)((it / S) & 1), status, 5))) { failed = true; break; }
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_a_full + 8 * (it % kAF), (uint32_t)((it / kAF) & 1), status, 5))) { failed = true; break; }
 #pragma unroll
             for (int at = 0; at < kAtoms; ++at) {
                 const uint32_t atom = ax_stage(s) + at * kAtomBytes;
@@ -435,7 +450,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
         for (int it = g; it < total; it += kGroups) {
             const int sq = it % SQ, s = it % S;
             // the W slot is free once the MMAs of step it - S have completed
-            if (it >= S && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * s, (uint32_t)((it / S - 1) & 1), status, 6))) { failed = true; break; }
+            if (it >= S && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * ((it - S) % kAF), (uint32_t)(((it - S) / kAF) & 1), status, 6))) { failed = true; break; }
             tc_fence_after_sync();
 
             // codes -> levels -> TMEM

@@ -63,6 +63,13 @@ constexpr int SD = 2;
 constexpr uint32_t kWCol = kSCol + SD * kStep;         // 320
 constexpr int WS = 3;                                  // W ring = activation ring depth
 constexpr int SA = 4;                                  // factor-tile ring depth
+// A barrier is waited on by parity alone, so whoever waits for its phase n must know that phase n - 1
+// has completed: true for a warp that waits for every phase of the barrier, and for a group (or an
+// issuer) that owns it.  Worker groups and main issuers take the k-steps alternately, and the W ring
+// has an odd depth, so a barrier per W slot would change hands every time round.  The barriers of
+// that ring which an alternating role waits on are therefore indexed by the k-step modulo WB, a
+// multiple of two: each of them has one owner.
+constexpr int WB = 2 * WS;
 constexpr int kXAtom = kTok * 128;                     // 16 tokens x 64 columns, 2 bytes each
 constexpr int kXStage = 2 * kXAtom;
 constexpr int kBTileBytes = kRows * 128;               // B[128 x 64 ranks] bf16
@@ -94,12 +101,12 @@ template <int BITS, int RP> struct XCfg {
     static constexpr int kBarAFull = kBarQEmpty + SQ;      // SA: 1 arrival + TMA bytes
     static constexpr int kBarADone = kBarAFull + SA;       // SA: scale MMA done (commit): frees the factor tile
     static constexpr int kBarXFull = kBarADone + SA;       // WS: 1 arrival + TMA bytes
-    static constexpr int kBarXReady = kBarXFull + WS;      // WS: the converter warps
-    static constexpr int kBarSFull = kBarXReady + WS;      // SD: scale MMA done (commit)
+    static constexpr int kBarXReady = kBarXFull + WS;      // WB: the converter warps
+    static constexpr int kBarSFull = kBarXReady + WB;      // SD: scale MMA done (commit)
     static constexpr int kBarSEmpty = kBarSFull + SD;      // SD: the warps of one worker group have read S
-    static constexpr int kBarReady = kBarSEmpty + SD;      // WS: the warps of one worker group have written W^
-    static constexpr int kBarMmaDone = kBarReady + WS;     // WS: main MMAs of the k-step done (commit): frees W slot and x tile
-    static constexpr int kBarAccFull = kBarMmaDone + WS;   // 2: one per main issuer
+    static constexpr int kBarReady = kBarSEmpty + SD;      // WB: the warps of one worker group have written W^
+    static constexpr int kBarMmaDone = kBarReady + WB;     // WB: main MMAs of the k-step done (commit): frees W slot and x tile
+    static constexpr int kBarAccFull = kBarMmaDone + WB;   // 2: one per main issuer
     static constexpr int kBarReduce = kBarAccFull + 2;     // 1: counts the bytes of the cluster's partial sums
     static constexpr int kBarBFull = kBarReduce + 1;       // 1: 1 arrival + TMA bytes of the B tile
     static constexpr int kBarCount = kBarBFull + 1;
@@ -239,7 +246,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             tma_prefetch_desc(&p.tm_q);
             for (int it = 0; it < total; ++it) {
                 const int sq = it % SQ;
-                if (it >= SQ && !mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1))) { failed = true; break; }
+                if (it >= SQ) {
+                    // a stage is freed by work that stands behind the dependency point: pass it first, so that
+                    // the bounded wait does not run while the previous launch (however long) still works
+                    if (it == SQ) griddep_wait();
+                    if (!mbar_wait(bar_q_empty + 8 * sq, (uint32_t)((it / SQ - 1) & 1))) { failed = true; break; }
+                }
                 const uint32_t bar = bar_q_full + 8 * sq;
                 mbar_expect_tx(bar, (uint32_t)C::QSTAGE);
                 tma_load_2d(q0 + sq * C::QSTAGE, &p.tm_q, (ks_a + it) * C::QROW, row0, bar);
@@ -330,7 +342,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             griddep_wait();
             for (int it = 0; it < total; ++it) {
                 const int sx = it % WS;
-                if (it >= WS && !mbar_wait(bar_mma_done + 8 * sx, (uint32_t)((it / WS - 1) & 1))) { failed = true; break; }
+                if (it >= WS && !mbar_wait(bar_mma_done + 8 * ((it - WS) % WB), (uint32_t)(((it - WS) / WB) & 1))) { failed = true; break; }
                 const uint32_t bar = bar_x_full + 8 * sx;
                 mbar_expect_tx(bar, (uint32_t)kXStage);
 #pragma unroll
@@ -381,8 +393,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         const uint32_t acc = tmem_base + (uint32_t)(j * 32);
         for (int it = j; it < total; it += 2) {
             const int ws = it % WS;
-            if (!mbar_wait(bar_x_ready + 8 * ws, (uint32_t)((it / WS) & 1)) ||
-                !mbar_wait(bar_ready + 8 * ws, (uint32_t)((it / WS) & 1))) { failed = true; break; }
+            if (!mbar_wait(bar_x_ready + 8 * (it % WB), (uint32_t)((it / WB) & 1)) ||
+                !mbar_wait(bar_ready + 8 * (it % WB), (uint32_t)((it / WB) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
                 const uint32_t wslot = tmem_base + kWCol + (uint32_t)(ws * 64);
@@ -391,7 +403,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
                 for (int k = 0; k < kStep / 16; ++k)
                     umma_f16_ts(acc, wslot + k * 8, umma_desc_pack(x_lo + (k >> 2) * (kXAtom >> 4) + (k & 3) * 2, desc_hi),
                                 idesc_m, (it == j && k == 0) ? 0u : 1u);
-                umma_commit(bar_mma_done + 8 * ws);
+                umma_commit(bar_mma_done + 8 * (it % WB));
                 if (it + 2 >= total) umma_commit(bar_acc_full + 8 * j);
             }
             __syncwarp();
@@ -419,7 +431,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             }
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_x_ready + 8 * sx);
+            if (lane == 0) mbar_arrive(bar_x_ready + 8 * (it % WB));
         }
     } else {
         // ------------------------------------------------------------------ worker warps
@@ -455,14 +467,14 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1)))) { failed = true; break; }
             dequant_half_row<BITS>(q0 + sq * C::QSTAGE + row * C::QROW, row, ch, lut_lane, sp);
             // the W slot is free once the MMAs of step it - WS have completed
-            if (it >= WS && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * ws, (uint32_t)((it / WS - 1) & 1)))) { failed = true; break; }
+            if (it >= WS && !__all_sync(0xffffffffu, mbar_wait(bar_mma_done + 8 * ((it - WS) % WB), (uint32_t)(((it - WS) / WB) & 1)))) { failed = true; break; }
             tc_fence_after_sync();
             tmem_st_32x32(lane_addr + kWCol + (uint32_t)(ws * 64 + ch * 32), sp);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(bar_ready + 8 * ws);
+                mbar_arrive(bar_ready + 8 * (it % WB));
                 mbar_arrive(bar_q_empty + 8 * sq);
             }
         }
