@@ -46,6 +46,8 @@ CASES = {
     "mlp3_down_m16":  dict(m=4096, n=14336, bits=3, r=48, M=16, outliers=0.0, bound="hbm"),
     "prefill_m2048":  dict(m=4096, n=14336, bits=4, r=32, M=2048, outliers=0.01, bound="tensor"),
 }
+# the step before the path (Alg. 1, step 2.1) on the same shapes: name -> (m, n, r, bits)
+QUANTIZE_CASES = {"quantize_q_nf4": (4096, 4096, 32, 4), "quantize_gate_nf3": (14336, 4096, 48, 3)}
 HEADLINE = "decode_q_m1"
 METRIC = "LoRDS dequant-GEMM: HBM GB/s at M=1, TFLOP/s at M=2048, % of roofline"
 
@@ -583,6 +585,8 @@ def main():
     ap.add_argument("--path", default="auto", help="force a kernel path (auto|simt|decode|umma)")
     ap.add_argument("--stack", action="store_true", help="(default) time the full Llama-3-8B linear stack as well")
     ap.add_argument("--no-stack", action="store_true", help="skip the 224-module Llama-3-8B linear stack")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="floor on the headline case's timed region (0: exactly --steps rounds, for profiler captures)")
     ap.add_argument("--sweep", action="store_true",
                     help="time every kernel path at M in {1, 2, 3, 4, 8, 16} on the q_proj, gate and down shapes and print the table")
     args = ap.parse_args()
@@ -615,9 +619,17 @@ def main():
             dist.destroy_process_group()
         return 0
 
+    if args.case in QUANTIZE_CASES:
+        if rank == 0:
+            print(json.dumps(time_quantize(args.case, *QUANTIZE_CASES[args.case], device, min_seconds=min(args.min_seconds, 0.3))))
+        lords.lords_shutdown()
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
     head = args.case or HEADLINE
     sampler = ClockSampler(local) if rank == 0 else None
-    res = time_case(head, args.steps, args.warmup, device, rank, world, sampler)
+    res = time_case(head, args.steps, args.warmup, device, rank, world, sampler, min_seconds=args.min_seconds)
     lay, packed = res.pop("_lay")
     c = CASES[head]
     cases = []
@@ -636,8 +648,8 @@ def main():
                           "copies": r2["copies"], "rounds": r2["rounds"], "steps": k, "status_retries": r2["status_retries"]})
 
     if not args.case and not args.no_extras and world == 1:
-        cases.append(time_quantize("quantize_q_nf4", 4096, 4096, 32, 4, device))
-        cases.append(time_quantize("quantize_gate_nf3", 14336, 4096, 48, 3, device))
+        for name, shape in QUANTIZE_CASES.items():
+            cases.append(time_quantize(name, *shape, device))
 
     stack = []
     if not args.no_stack and not args.no_extras and not args.case and world == 1:

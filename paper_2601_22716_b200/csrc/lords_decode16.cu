@@ -309,9 +309,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     // let a dependent launch (the next layer) begin its own weight prefetch as SMs become free
     griddep_launch_dependents();
     // Everything except the stream of packed codes waits here for the previous launch to finish: a CTA
-    // that starts early sets up, prefetches its codes and then stands still.  (Letting the workers
-    // run ahead of this point as well was tried; with it about one run in twenty of a 224-kernel
-    // graph ended in device-side timeouts whose cause was not found.)
+    // that starts early sets up, prefetches its codes and then stands still, so that every bounded
+    // wait below begins behind the dependency point.
     if (warp != kTmaQWarp) griddep_wait();
 
     if (warp == kTmaQWarp) {

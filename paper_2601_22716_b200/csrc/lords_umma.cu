@@ -46,8 +46,6 @@ constexpr int kThreads = (kWorkWarps + 4) * 32;   // 640
 constexpr int SA = 4;                          // factor-tile ring depth
 constexpr int DR = 8;                          // "main MMA of k-step done" barriers, indexed by k-step mod DR
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kWCol = 384;                // W ring: 4 slots of 32 columns
-constexpr int WD = 4;                          // W ring depth
 constexpr int SQ = 4;                          // code-tile ring depth (128 columns per stage)
 constexpr int kBTileBytes = BM * 128;
 constexpr int kClusterMax = 8;                 // largest k-split (cluster size) of the BN = 16 kernel
@@ -62,8 +60,13 @@ template <int BITS, int BN, int RP> struct UCfg {
     static constexpr int ATILE = RP * 128;
     static constexpr int SX = BN >= 256 ? (RP <= 32 ? 4 : 3) : BN >= 128 ? 6 : 8;
     static constexpr int XTILE = BN * 128;
-    static constexpr uint32_t SCOL = BN > 128 ? 256 : 128;       // S ring starts behind the accumulator
-    static constexpr int SD = (int)(kWCol - SCOL) / 64;          // S ring depth (2 / 4)
+    // TMEM behind the accumulator is one ring of 64-column slots.  A slot first holds S of a k-step
+    // (128 x 64 fp32, written by the scale MMA), then -- in the columns whose S values the writing
+    // warp itself has taken into registers -- the fp16 operand W^ of the same k-step, and is free
+    // again when the main MMAs of that k-step have completed.  One ring instead of an S ring and a W
+    // ring lets the scale MMA run as many k-steps ahead as there are slots.
+    static constexpr uint32_t SCOL = BN > 128 ? 256 : 128;       // the ring starts behind the accumulator
+    static constexpr int SD = (int)(kTmemCols - SCOL) / 64;      // slots (4 / 6)
     static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;
     static constexpr int LUT_BYTES = LUT_ENTRIES * 128;
     static constexpr int RED_BYTES = BN == 16 ? kClusterMax * 16 * BM * 4 : 0;
@@ -132,7 +135,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 {
     using C = UCfg<BITS, BN, RP>;
     constexpr int SX = C::SX, SD = C::SD, kATileBytes = C::ATILE;
-    static_assert(DR >= SX && DR >= WD && DR % WD == 0 && DR % 2 == 0, "done-barrier ring");
+    static_assert(DR >= SX && DR >= SD && DR % 2 == 0 && SD % 2 == 0, "done-barrier ring; one worker group per slot");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -151,16 +154,15 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
     constexpr int kBarQFull = kBarDone + DR;            // SQ
     constexpr int kBarQEmpty = kBarQFull + SQ;          // SQ: all 16 worker warps (two steps)
     constexpr int kBarSFull = kBarQEmpty + SQ;          // SD: scale MMA done (commit)
-    constexpr int kBarSEmpty = kBarSFull + SD;          // SD: one group has read S
-    constexpr int kBarWFull = kBarSEmpty + SD;          // WD: one group has written W^ (and converted x)
-    constexpr int kBarAccFull = kBarWFull + WD;         // 1
+    constexpr int kBarWFull = kBarSFull + SD;           // SD: one group has written W^ (and converted x)
+    constexpr int kBarAccFull = kBarWFull + SD;         // 1
     constexpr int kBarReduce = kBarAccFull + 1;         // 1: the epilogue warps of every CTA of the cluster
     constexpr int kBarCount = kBarReduce + 1;
     static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
     const uint32_t bar_x_full = bars + 8 * kBarXFull, bar_done = bars + 8 * kBarDone;
     const uint32_t bar_a_full = bars + 8 * kBarAFull, bar_a_done = bars + 8 * kBarADone;
     const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
-    const uint32_t bar_s_full = bars + 8 * kBarSFull, bar_s_empty = bars + 8 * kBarSEmpty;
+    const uint32_t bar_s_full = bars + 8 * kBarSFull;
     const uint32_t bar_w_full = bars + 8 * kBarWFull;
     const uint32_t bar_acc_full = bars + 8 * kBarAccFull, bar_reduce = bars + 8 * kBarReduce;
     const uint32_t tmem_slot = bars + 8 * kBarCount;
@@ -199,7 +201,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         for (int b = lane; b < kBarCount; b += 32) {
             uint32_t count = 1;
             if (b >= kBarQEmpty && b < kBarSFull) count = kWorkWarps;
-            else if (b >= kBarSEmpty && b < kBarAccFull) count = kGroupWarps;   // s_empty and w_full
+            else if (b >= kBarWFull && b < kBarAccFull) count = kGroupWarps;
             else if (b == kBarReduce) count = BN == 16 ? 1u : (uint32_t)(4 * (BN / (BN >= 64 ? BN / 4 : 16)));
             mbar_init(bars + 8 * b, count);
         }
@@ -312,8 +314,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         }
     } else if (warp == kScaleWarp) {
         // ------------------------------------------------------------------ scale-MMA issuer
-        // S of k-step j goes into S buffer j % SD as soon as the factor tile has landed and the workers
-        // have read the buffer's previous content: it runs ahead of the main MMAs by itself.
+        // S of k-step j goes into ring slot j % SD as soon as the factor tile has landed and the main MMAs
+        // of k-step j - SD are done with the slot: it runs SD k-steps ahead of the main MMAs by itself.
         uint32_t tmem_base;
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
         constexpr uint32_t idesc_s = umma_idesc_f16(1, 0, 1, BM, 64);     // bf16, B operand MN-major, N = 64
@@ -325,7 +327,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         for (int j = 0; j < total; ++j) {
             const int sa = j % SA, sd = j % SD;
             if (!mbar_wait(bar_a_full + 8 * sa, (uint32_t)((j / SA) & 1))) { failed = true; break; }
-            if (j >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((j / SD - 1) & 1))) { failed = true; break; }
+            // the slot is free once the main MMAs of k-step j - SD have read their operand out of it
+            if (j >= SD && !mbar_wait(bar_done + 8 * ((j - SD) % DR), (uint32_t)(((j - SD) / DR) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
                 const uint32_t a_lo = a_lo0 + (uint32_t)(sa * (kATileBytes >> 4));
@@ -345,17 +348,18 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         const uint32_t desc_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
         const uint32_t x_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((x0 & 0x3FFFFu) >> 4);
         for (int it = 0; it < total; ++it) {
-            const int sx = it % SX, ws = it % WD;
+            const int sx = it % SX, ws = it % SD;
             // W^ of the k-step is in TMEM and its activation tile has landed
-            if (!mbar_wait(bar_w_full + 8 * ws, (uint32_t)((it / WD) & 1))) { failed = true; break; }
+            if (!mbar_wait(bar_w_full + 8 * ws, (uint32_t)((it / SD) & 1))) { failed = true; break; }
             if (!mbar_wait(bar_x_full + 8 * sx, (uint32_t)((it / SX) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
-                const uint32_t wslot = tmem_base + kWCol + (uint32_t)(ws * 32);
+                const uint32_t wslot = tmem_base + C::SCOL + (uint32_t)(ws * 64);
                 const uint32_t x_lo = x_lo0 + (uint32_t)((sx * C::XTILE) >> 4);
 #pragma unroll
                 for (int k = 0; k < BK / 16; ++k)
-                    umma_f16_ts(tmem_base, wslot + k * 8, umma_desc_pack(x_lo + k * 2, desc_hi), idesc_m,
+                    // columns 0-31 of the k-step sit in slot columns 0-15, columns 32-63 in 32-47
+                    umma_f16_ts(tmem_base, wslot + (k >> 1) * 32 + (k & 1) * 8, umma_desc_pack(x_lo + k * 2, desc_hi), idesc_m,
                                 (it > 0 || k > 0) ? 1u : 0u);
                 umma_commit(bar_done + 8 * (it % DR));
                 if (it == total - 1) umma_commit(bar_acc_full);
@@ -372,16 +376,13 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
         const uint32_t lut_lane = lut + 4u * (uint32_t)lane;
 
         for (int it = g; it < total; it += 2) {
-            const int sx = it % SX, sd = it % SD, ws = it % WD, pr = it >> 1, sq = pr % SQ;
+            const int sx = it % SX, sd = it % SD, pr = it >> 1, sq = pr % SQ;
             if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * sd, (uint32_t)((it / SD) & 1)))) { failed = true; break; }
             tc_fence_after_sync();
             uint32_t s[32];
             tmem_ld_32x32(lane_addr + C::SCOL + (uint32_t)(sd * 64 + ch * 32), s);
             bool ok = mbar_wait(bar_q_full + 8 * sq, (uint32_t)((pr / SQ) & 1));
             tmem_wait_ld();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_s_empty + 8 * sd);      // S is in registers: the buffer may be refilled
             if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
             uint32_t out[16];
             dequant_chunk<BITS>(q0 + sq * C::QSTAGE + row * C::QROW, row, (it & 1) * 2 + ch, lut_lane, s, out);
@@ -404,17 +405,13 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 }
                 fence_proxy_async_smem();
             }
-            if (it >= WD && !__all_sync(0xffffffffu, mbar_wait(bar_done + 8 * ((it - WD) % DR), (uint32_t)(((it - WD) / DR) & 1)))) {
-                failed = true;
-                break;
-            }
-            tc_fence_after_sync();
-            tmem_st_32x16(lane_addr + kWCol + (uint32_t)(ws * 32 + ch * 16), out);
+            // W^ goes where this warp's own S values were: nobody else reads those columns of these lanes
+            tmem_st_32x16(lane_addr + C::SCOL + (uint32_t)(sd * 64 + ch * 32), out);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(bar_w_full + 8 * ws);
+                mbar_arrive(bar_w_full + 8 * sd);
                 mbar_arrive(bar_q_empty + 8 * sq);
             }
         }
