@@ -136,6 +136,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
     using C = UCfg<BITS, BN, RP>;
     constexpr int SX = C::SX, SD = C::SD, kATileBytes = C::ATILE;
     static_assert(DR >= SX && DR >= SD && DR % 2 == 0 && SD % 2 == 0, "done-barrier ring; one worker group per slot");
+    static_assert(SD >= SA, "the factor-tile lane frees a tile on the slot barrier of the same k-step");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -149,18 +150,17 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
     const uint32_t bars = red0 + C::RED_BYTES;
     constexpr int kBarXFull = 0;                        // SX: TMA bytes of the activation tile
     constexpr int kBarAFull = kBarXFull + SX;           // SA: TMA bytes of the factor tile
-    constexpr int kBarADone = kBarAFull + SA;           // SA: scale MMA of the k-step done (commit): frees the factor tile
-    constexpr int kBarDone = kBarADone + SA;            // DR: main MMA of the k-step done (commit): frees its x tile and its W slot
+    constexpr int kBarDone = kBarAFull + SA;            // DR: main MMA of the k-step done (commit): frees its x tile and its ring slot
     constexpr int kBarQFull = kBarDone + DR;            // SQ
     constexpr int kBarQEmpty = kBarQFull + SQ;          // SQ: all 16 worker warps (two steps)
-    constexpr int kBarSFull = kBarQEmpty + SQ;          // SD: scale MMA done (commit)
+    constexpr int kBarSFull = kBarQEmpty + SQ;          // SD: scale MMA done (commit): S is in the slot, the factor tile is free
     constexpr int kBarWFull = kBarSFull + SD;           // SD: one group has written W^ (and converted x)
     constexpr int kBarAccFull = kBarWFull + SD;         // 1
     constexpr int kBarReduce = kBarAccFull + 1;         // 1: the epilogue warps of every CTA of the cluster
     constexpr int kBarCount = kBarReduce + 1;
     static_assert(8 * kBarCount + 8 <= C::BAR_BYTES, "barrier area");
     const uint32_t bar_x_full = bars + 8 * kBarXFull, bar_done = bars + 8 * kBarDone;
-    const uint32_t bar_a_full = bars + 8 * kBarAFull, bar_a_done = bars + 8 * kBarADone;
+    const uint32_t bar_a_full = bars + 8 * kBarAFull;
     const uint32_t bar_q_full = bars + 8 * kBarQFull, bar_q_empty = bars + 8 * kBarQEmpty;
     const uint32_t bar_s_full = bars + 8 * kBarSFull;
     const uint32_t bar_w_full = bars + 8 * kBarWFull;
@@ -306,7 +306,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
             const uint32_t tx = (uint32_t)(p.r_pad * 128);
             for (int j = 0; j < total; ++j) {
                 const int sa = j % SA;
-                if (j >= SA && !mbar_wait(bar_a_done + 8 * sa, (uint32_t)((j / SA - 1) & 1))) { failed = true; break; }
+                // the tile's slot is free once the scale MMA of k-step j - SA has completed: that is the
+                // commit the workers wait for as well (this lane looks at every phase of those barriers
+                // in turn, and no slot barrier can run a phase ahead of it: the scale MMA of k-step
+                // j - SA + SD needs a factor tile that this lane has not loaded yet)
+                if (j >= SA && !mbar_wait(bar_s_full + 8 * ((j - SA) % SD), (uint32_t)(((j - SA) / SD) & 1))) { failed = true; break; }
                 const uint32_t bar = bar_a_full + 8 * sa;
                 mbar_expect_tx(bar, tx);
                 tma_load_2d(a0 + sa * kATileBytes, &p.tm_a, (2 * pa + j) * BK, 0, bar);
@@ -336,7 +340,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                     umma_f16_ss(tmem_base + C::SCOL + sd * 64, umma_desc_pack(b_lo + k * 2, desc_hi),
                                 umma_desc_pack(a_lo + k * 128, desc_hi), idesc_s, k > 0);
                 umma_commit(bar_s_full + 8 * sd);
-                umma_commit(bar_a_done + 8 * sa);
             }
             __syncwarp();
         }
