@@ -73,8 +73,16 @@ def measured_peaks():
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised
 # under profiles/ (None until a capture of that case exists).
-NCU_TRAFFIC_BYTES = {"decode_q_m1": 8960256,    # profiles/decode_kernel_decode_q_m1.md
-                     "decode_q_m8": 9030656}    # profiles/decode16_kernel_decode_q_m8.md
+NCU_TRAFFIC_BYTES = {
+    "decode_q_m1": 8976640,         # profiles/decode_kernel_decode_q_m1.md
+    "decode_q_m8": 9029632,         # profiles/decode16_kernel_decode_q_m8_down_m16.md
+    "mlp3_gate_m1": 23850496,       # profiles/decode_kernel_mlp3_gate_m1_down_m1.md
+    "mlp3_down_m1": 23938560,       # same
+    "mlp3_down_m16": 24299520,      # profiles/decode16_kernel_decode_q_m8_down_m16.md
+    "prefill_m2048": 144602368,     # profiles/umma_kernel_prefill_m2048.md (the scale-MMA kernel; the pre-pass moves 73.7 MB more)
+    "quantize_q_nf4": 34142720,     # profiles/quantize_kernel_q_nf4_gate_nf3.md (8.4 MB of codes were still in L2 at the end)
+    "quantize_gate_nf3": 130091264,
+}
 
 
 class ClockSampler:
@@ -457,7 +465,7 @@ def time_quantize(name, m, n, r, bits, device, min_seconds=0.3):
     return {"case": name, "path": path, "us_per_call": us, "gbs": gbs, "tflops": None, "copies": copies, "rounds": reps,
             "steps": 1, "status_retries": 0 if status == 0 else 1,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                         "frac": gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": NCU_TRAFFIC_BYTES.get(name),
                          "algorithmic_bytes_per_launch": byt, "us_per_launch": us}}
 
 

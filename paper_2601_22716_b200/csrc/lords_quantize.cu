@@ -4,9 +4,10 @@
 //
 // written out as packed codes in the library's layout.  The paper does not say which level wins a tie:
 // the lowest code does.  S is rebuilt tile by tile on the tensor cores exactly as the forward kernels
-// rebuild it (bf16 operands from shared memory, fp32 in TMEM, never stored in full); every level is
-// then tried in turn in fp32 (one fused multiply-add and a square per level), so the decision is taken
-// in fp32 with S accumulated in fp32.
+// rebuild it (bf16 operands from shared memory, fp32 in TMEM, never stored in full).  The decision is
+// taken in fp32 with S accumulated in fp32: for a strictly ascending level table by bisection over the
+// midpoints between neighbouring levels (log2 of the level count products and comparisons per weight),
+// for any other table by trying every level in turn (one fused multiply-add and a square per level).
 //
 // One CTA owns 128 rows of W and a range of 64-column steps.  Warp roles (6 warps):
 //   0..3  search: thread t owns row t; per step it reads its 64 values of S from TMEM (two loads of
@@ -50,6 +51,7 @@ struct alignas(64) QuantParams {
     const uint16_t *B;    // bf16 [m][r]
     uint8_t *Q;           // packed codes, row pitch n * bits / 8
     float levels[16];
+    float mids[16];       // ascending table: mids[c] = (levels[c] + levels[c + 1]) / 2
     int bits, m, n, r, r_pad;
     int steps;            // 64-column steps per row (n / 64)
     int steps_per_cta;
@@ -70,6 +72,40 @@ __device__ __forceinline__ uint32_t nearest_code(float s, float w, const float (
         if (e < e_best) { e_best = e; best = (uint32_t)c; }
     }
     return best;
+}
+
+// The same for a strictly ascending table, by bisection over the midpoints between neighbouring levels:
+// (s v - w)^2 = s^2 (v - w/s)^2, so the nearest level to t = w / s wins whatever the sign of s, and
+// t > mid  <=>  b > a mid  with a = |s|, b = w sign(s).  The code is the number of midpoints below t; a
+// weight exactly on a midpoint keeps the lower code, and s = 0 (every level equally good) gives code 0.
+// The thresholds of the later steps are picked by selects on the earlier outcomes: log2(LEVELS)
+// products and comparisons instead of LEVELS.
+template <int LEVELS>
+__device__ __forceinline__ uint32_t nearest_code_sorted(float s, float w, const float (&md)[16])
+{
+    const float a = fabsf(s);
+    float b = s < 0.0f ? -w : w;
+    b = a == 0.0f ? -INFINITY : b;
+    if constexpr (LEVELS == 16) {
+        const bool p3 = b > a * md[7];
+        const bool p2 = b > a * (p3 ? md[11] : md[3]);
+        const float m1 = p3 ? (p2 ? md[13] : md[9]) : (p2 ? md[5] : md[1]);
+        const bool p1 = b > a * m1;
+        const float m0hi = p2 ? (p1 ? md[14] : md[12]) : (p1 ? md[10] : md[8]);
+        const float m0lo = p2 ? (p1 ? md[6] : md[4]) : (p1 ? md[2] : md[0]);
+        const bool p0 = b > a * (p3 ? m0hi : m0lo);
+        return ((uint32_t)p3 << 3) | ((uint32_t)p2 << 2) | ((uint32_t)p1 << 1) | (uint32_t)p0;
+    } else if constexpr (LEVELS == 8) {
+        const bool p2 = b > a * md[3];
+        const bool p1 = b > a * (p2 ? md[5] : md[1]);
+        const float m0 = p2 ? (p1 ? md[6] : md[4]) : (p1 ? md[2] : md[0]);
+        const bool p0 = b > a * m0;
+        return ((uint32_t)p2 << 2) | ((uint32_t)p1 << 1) | (uint32_t)p0;
+    } else {
+        const bool p1 = b > a * md[1];
+        const bool p0 = b > a * (p1 ? md[2] : md[0]);
+        return ((uint32_t)p1 << 1) | (uint32_t)p0;
+    }
 }
 
 // 32 codes of one row -> packed bytes at `dst` (the row's byte offset of these 32 columns).
@@ -113,8 +149,8 @@ __device__ __forceinline__ void store_codes(uint8_t *dst, const uint32_t (&c)[32
     }
 }
 
-template <int BITS>
-__global__ void __launch_bounds__(kThreadsQ, 1) lords_quantize_kernel(const __grid_constant__ QuantParams p)
+template <int BITS, bool SORTED>
+__global__ void __launch_bounds__(kThreadsQ, 3) lords_quantize_kernel(const __grid_constant__ QuantParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -210,7 +246,7 @@ __global__ void __launch_bounds__(kThreadsQ, 1) lords_quantize_kernel(const __gr
         const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
         float lv[16];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) lv[c] = p.levels[c];
+        for (int c = 0; c < 16; ++c) lv[c] = SORTED ? p.mids[c] : p.levels[c];
         const size_t qpitch = (size_t)p.n * BITS / 8;
         for (int it = 0; it < total; ++it) {
             const int sd = it % kSDQ;
@@ -243,8 +279,14 @@ __global__ void __launch_bounds__(kThreadsQ, 1) lords_quantize_kernel(const __gr
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int c = v * 8 + e * 2;
-                            codes[c] = nearest_code<(1 << BITS)>(__uint_as_float(s[c]), __uint_as_float(ww[e] << 16), lv);
-                            codes[c + 1] = nearest_code<(1 << BITS)>(__uint_as_float(s[c + 1]), __uint_as_float(ww[e] & 0xFFFF0000u), lv);
+                            const float w0 = __uint_as_float(ww[e] << 16), w1 = __uint_as_float(ww[e] & 0xFFFF0000u);
+                            if constexpr (SORTED) {
+                                codes[c] = nearest_code_sorted<(1 << BITS)>(__uint_as_float(s[c]), w0, lv);
+                                codes[c + 1] = nearest_code_sorted<(1 << BITS)>(__uint_as_float(s[c + 1]), w1, lv);
+                            } else {
+                                codes[c] = nearest_code<(1 << BITS)>(__uint_as_float(s[c]), w0, lv);
+                                codes[c + 1] = nearest_code<(1 << BITS)>(__uint_as_float(s[c + 1]), w1, lv);
+                            }
                         }
                     }
                     store_codes<BITS>(p.Q + (size_t)i * qpitch + (size_t)(col0 + h * 32) * BITS / 8, codes);
@@ -299,23 +341,23 @@ __global__ void lords_quantize_simt_kernel(const uint16_t *__restrict__ W, const
     for (int b = 0; b < BYTES; ++b) dst[b] = b < 8 ? (uint8_t)(lo >> (8 * b)) : (uint8_t)(hi >> (8 * (b - 8)));
 }
 
-template <int BITS> int launch_quantize_tc(QuantParams &k, const State &st, cudaStream_t stream)
+template <int BITS, bool SORTED> int launch_quantize_tc(QuantParams &k, const State &st, cudaStream_t stream)
 {
     static bool done[kMaxDevices] = {};
     const int dev = device_slot(st);
     if (!done[dev]) {
-        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_quantize_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemQ));
+        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_quantize_kernel<BITS, SORTED>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemQ));
         done[dev] = true;
     }
     const int row_tiles = (k.m + kRowsQ - 1) / kRowsQ;
     // column ranges: about two CTAs per SM in all, at least four steps each
-    int splits = (2 * st.sm_count + row_tiles - 1) / row_tiles;
+    int splits = (6 * st.sm_count + row_tiles - 1) / row_tiles;
     if (splits > k.steps / 4) splits = k.steps / 4;
     if (splits < 1) splits = 1;
     if (splits > 65535) splits = 65535;
     k.steps_per_cta = (k.steps + splits - 1) / splits;
     splits = (k.steps + k.steps_per_cta - 1) / k.steps_per_cta;
-    lords_quantize_kernel<BITS><<<dim3((unsigned)row_tiles, (unsigned)splits), kThreadsQ, kSmemQ, stream>>>(k);
+    lords_quantize_kernel<BITS, SORTED><<<dim3((unsigned)row_tiles, (unsigned)splits), kThreadsQ, kSmemQ, stream>>>(k);
     LORDS_CUDA_TRY(cudaGetLastError());
     return LORDS_OK;
 }
@@ -330,13 +372,21 @@ int launch_quantize(const void *W, const void *B, const void *A, const float *le
         QuantParams k;
         k.W = static_cast<const uint16_t *>(W); k.B = static_cast<const uint16_t *>(B); k.Q = Q;
         for (int c = 0; c < 16; ++c) k.levels[c] = c < (1 << bits) ? levels[c] : 0.0f;
+        // a strictly ascending table (every NormalFloat table is) is searched by bisection over its
+        // midpoints, any other table level by level
+        bool sorted = true;
+        for (int c = 0; c + 1 < (1 << bits); ++c) sorted = sorted && levels[c] < levels[c + 1];
+        for (int c = 0; c < 16; ++c) k.mids[c] = (sorted && c + 1 < (1 << bits)) ? 0.5f * (levels[c] + levels[c + 1]) : 0.0f;
         k.bits = bits; k.m = m; k.n = n; k.r = r; k.r_pad = (r + 15) / 16 * 16;
         k.steps = n / kColsQ;
         k.status = st.status_word;
         if (!make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, A, (uint64_t)n, (uint64_t)r, 64, (uint32_t)k.r_pad,
                          CU_TENSOR_MAP_SWIZZLE_128B))
             return LORDS_ERR_CUDA;
-        const int rc = bits == 4 ? launch_quantize_tc<4>(k, st, stream) : bits == 3 ? launch_quantize_tc<3>(k, st, stream) : launch_quantize_tc<2>(k, st, stream);
+        const int rc = sorted ? (bits == 4 ? launch_quantize_tc<4, true>(k, st, stream)
+                                           : bits == 3 ? launch_quantize_tc<3, true>(k, st, stream) : launch_quantize_tc<2, true>(k, st, stream))
+                              : (bits == 4 ? launch_quantize_tc<4, false>(k, st, stream)
+                                           : bits == 3 ? launch_quantize_tc<3, false>(k, st, stream) : launch_quantize_tc<2, false>(k, st, stream));
         if (rc != LORDS_OK) return rc;
         st.last_launches = 1;
         st.last_path = "quantize";

@@ -67,7 +67,7 @@ template <int BITS, int BN, int RP> struct UCfg {
     // ring lets the scale MMA run as many k-steps ahead as there are slots.
     static constexpr uint32_t SCOL = BN > 128 ? 256 : 128;       // the ring starts behind the accumulator
     static constexpr int SD = (int)(kTmemCols - SCOL) / 64;      // slots (4 / 6)
-    static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;
+    static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : BITS == 3 ? 64 : 16;   // one entry per code pair
     static constexpr int LUT_BYTES = LUT_ENTRIES * 128;
     static constexpr int RED_BYTES = BN == 16 ? kClusterMax * 16 * BM * 4 : 0;
     static constexpr int BAR_BYTES = 512;
@@ -110,6 +110,15 @@ __device__ __forceinline__ void dequant_chunk(uint32_t qrow, int row, int c, uin
                 const uint32_t sh = b == 0 ? (w[wi] << 7) : (w[wi] >> (8 * b - 7));
                 lv[wi * 4 + b] = lds_u32(lut_lane + (sh & 0x7F80u));
             }
+    } else if constexpr (BITS == 2) {
+        // 32-byte rows: chunk c is the 64-bit group at byte 8c; pair p sits at bit 4p of it
+        const uint32_t w[2] = {lds_u32(qrow + 8 * c), lds_u32(qrow + 8 * c + 4)};
+#pragma unroll
+        for (int pp = 0; pp < 16; ++pp) {
+            const int off = 4 * (pp & 7);
+            const uint32_t sh = off >= 7 ? (w[pp >> 3] >> (off - 7)) : (w[pp >> 3] << (7 - off));
+            lv[pp] = lds_u32(lut_lane + (sh & 0x780u));
+        }
     } else {
         // 48-byte rows: chunk c is the 96-bit group at byte 12c; pair p sits at bit 6p of it
         const uint32_t w[3] = {lds_u32(qrow + 12 * c), lds_u32(qrow + 12 * c + 4), lds_u32(qrow + 12 * c + 8)};
@@ -263,8 +272,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 #pragma unroll
             for (int i = 0; i < C::LUT_ENTRIES / kWorkWarps; ++i) {
                 const int entry = warp + kWorkWarps * i;
-                const int lo = BITS == 4 ? (entry & 15) : (entry & 7);
-                const int hi = BITS == 4 ? (entry >> 4) : (entry >> 3);
+                const int lo = entry & ((1 << BITS) - 1);
+                const int hi = entry >> BITS;
                 const __half2 v = __floats2half2_rn(p.levels[lo], p.levels[hi]);
                 sts_u32(lut + 4u * (uint32_t)(entry * 32 + lane), *reinterpret_cast<const uint32_t *>(&v));
             }
@@ -684,12 +693,12 @@ template <int BITS> int launch_bits(UmmaParams &k, const Problem &p, State &st, 
 
 }  // namespace
 
-// Rules of this path: 3- or 4-bit codes; r <= 64; n a multiple of 64 (4-bit) or 128 (3-bit), which
-// makes every TMA row pitch a multiple of 16 bytes.  Anything else: LORDS_ERR_UNSUPPORTED.
+// Rules of this path: r <= 64; n a multiple of 64 (2- and 4-bit codes) or 128 (3-bit), which makes
+// every TMA row pitch a multiple of 16 bytes.  Anything else: LORDS_ERR_UNSUPPORTED.
 int launch_umma(const Problem &p, State &st, cudaStream_t stream)
 {
-    if (p.bits != 3 && p.bits != 4) return LORDS_ERR_UNSUPPORTED;
-    if (p.r > kRMaxUmma || p.n % (p.bits == 4 ? 64 : 128) != 0) return LORDS_ERR_UNSUPPORTED;
+    if (p.bits < 2 || p.bits > 4) return LORDS_ERR_UNSUPPORTED;
+    if (p.r > kRMaxUmma || p.n % (p.bits == 3 ? 128 : 64) != 0) return LORDS_ERR_UNSUPPORTED;
 
     UmmaParams k;
     k.B = p.B;
@@ -699,7 +708,7 @@ int launch_umma(const Problem &p, State &st, cudaStream_t stream)
     k.npairs = (p.n + 127) / 128;
     k.y = p.y; k.y_f32 = p.y_f32;
     k.status = st.status_word;
-    const int rc = p.bits == 4 ? launch_bits<4>(k, p, st, stream) : launch_bits<3>(k, p, st, stream);
+    const int rc = p.bits == 4 ? launch_bits<4>(k, p, st, stream) : p.bits == 3 ? launch_bits<3>(k, p, st, stream) : launch_bits<2>(k, p, st, stream);
     if (rc != LORDS_OK) return rc;
     st.last_path = "umma";
     return LORDS_OK;

@@ -249,6 +249,13 @@ UMMA_SHAPES = [
     (4, 256, 1024, 8, 257, 256, True),   # a second token tile with one token in it
     (4, 1024, 512, 16, 600, 32, False),  # more tiles than resident CTAs: the last wave is filled with split tiles
     (3, 1100, 512, 32, 620, 32, True),
+    # 2-bit codes (the paper's ultra-low-bit setting) and ranks of its Table 7
+    (2, 384, 1024, 12, 5, 0, True),
+    (2, 130, 192, 6, 1, 0, False),       # n = 1.5 code stages
+    (2, 256, 2048, 15, 40, 32, True),
+    (2, 200, 1024, 32, 70, 64, False),
+    (2, 300, 1536, 24, 100, 128, True),
+    (2, 384, 1280, 48, 300, 256, False),
 ]
 
 
@@ -265,7 +272,8 @@ def test_umma_kernel_shapes(lords, bits, m, n, r, M, bn, mixed):
 
 
 @pytest.mark.parametrize("bits,m,n,r,M,bn", [(4, 256, 512, 32, 16, 0), (3, 131, 384, 7, 9, 0), (4, 140, 256, 16, 33, 32),
-                                             (3, 256, 512, 48, 200, 256), (4, 1280, 256, 8, 500, 32)])
+                                             (3, 256, 512, 48, 200, 256), (4, 1280, 256, 8, 500, 32),
+                                             (2, 256, 512, 16, 4, 0), (2, 140, 320, 5, 130, 128)])
 def test_umma_kernel_integer_case_is_bit_exact(lords, bits, m, n, r, M, bn):
     lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m + M)
     lords.lords_set_option("bn", str(bn))

@@ -6,6 +6,8 @@ two.  The test asserts that the codes are equal wherever the oracle's choice was
 that rounding distance, that every other difference is the oracle's runner-up code, and that such near
 ties are rare; then that the packed codes, fed to the forward path, reproduce the oracle's forward of
 the oracle's codes up to the forward tolerances."""
+import dataclasses
+
 import numpy as np
 import pytest
 
@@ -122,3 +124,46 @@ def test_quantize_then_forward_matches_the_oracle(lords):
     What = oracle.dequant_rows(Q.cpu().numpy().reshape(m, -1), lay.B, lay.A, lay.codebook, 4)
     Wf = gen.bf16_to_f32(Wb).astype(np.float64)
     assert np.mean((What - Wf) ** 2) < 0.1 * np.mean(Wf ** 2)
+
+
+@pytest.mark.parametrize("bits", [4, 3, 2])
+def test_quantize_with_a_table_that_is_not_ascending(lords, bits):
+    """An ascending table is searched by bisection over its midpoints, any other one level by level:
+    a permuted table takes the second route and must give the oracle's codes just the same."""
+    lay = gen.make_layer(256, 256, 16, 1, bits=bits, seed=70 + bits, mixed_sign=True)
+    rng = np.random.default_rng(bits)
+    lay = dataclasses.replace(lay, codebook=np.ascontiguousarray(lay.codebook[rng.permutation(1 << bits)]))
+    Wb = gen.make_weight(256, 256, seed=80 + bits, sigma=0.025)
+    Q, used = _quantize_on_gpu(lords, Wb, lay)
+    assert used == "quantize"
+    _check_codes(lords, Q, Wb, lay)
+
+
+def test_quantize_exact_ties_and_zero_scale_take_the_lowest_code(lords):
+    """Integers, so that nothing rounds: weights exactly half-way between two levels keep the lower
+    code for either sign of S, and rows whose S is zero (every level equally good) get code 0."""
+    import torch
+    m, n, r = 128, 64, 2
+    levels = np.array([-6, -4, -2, 0, 2, 4, 6, 8], dtype=np.float32)      # 3 bits, ascending
+    rng = np.random.default_rng(5)
+    Bf = np.zeros((m, r), dtype=np.float32)
+    Bf[:, 0] = rng.choice([-2.0, -1.0, 1.0, 2.0], size=m)
+    Bf[::7, 0] = 0.0                                     # rows with S = 0
+    Af = np.zeros((r, n), dtype=np.float32)
+    Af[0, :] = 1.0
+    S = Bf @ Af
+    lo = rng.integers(0, 7, size=(m, n))
+    W = S * (levels[lo] + 1.0)                           # exactly between level lo and lo + 1 (in units of S)
+    W[::7, :] = rng.integers(-5, 6, size=(len(range(0, m, 7)), n))
+    lay = dataclasses.replace(gen.make_integer_layer(m, n, r, 1, bits=3, seed=1), B=gen.bf16_bits(torch.from_numpy(Bf)),
+                              A=gen.bf16_bits(torch.from_numpy(Af)), codebook=levels)
+    Wb = gen.bf16_bits(torch.from_numpy(W.astype(np.float32)))
+    assert np.array_equal(gen.bf16_to_f32(Wb), W.astype(np.float32))
+    want = oracle.quantize(Wb, lay.B, lay.A, lay.codebook, 3)
+    expect = lo.copy()
+    expect[::7, :] = 0
+    assert np.array_equal(want, expect)                  # the oracle follows the tie rule ...
+    Q, used = _quantize_on_gpu(lords, Wb, lay)
+    assert used == "quantize"
+    got = oracle.unpack_codes(Q.cpu().numpy().reshape(m, -1), m, n, 3)
+    assert np.array_equal(got, expect)                   # ... and so does the kernel, bit for bit
