@@ -79,11 +79,11 @@ template <int BITS, int H> struct DCfg {
     static constexpr int S = S_TMEM < 4 ? S_TMEM : 4;          // W / factor ring depth (4 / 3)
     static constexpr int AXSTAGE = kAtoms * kAtomBytes;
     static constexpr int XSTAGE = 2 * kStep * 2;               // the k-step's slice of x, two tokens (bf16)
-    static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;   // one entry per code pair
+    static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : BITS == 3 ? 64 : 16;   // one entry per code pair
     // 32 lane-private copies of every entry (word = lane, so the lookups of a warp never conflict).
     // 4-bit: an entry every 256 bytes and the table on a 64 KB boundary, which lets one byte
     // permute build a lookup address: byte 0 = 4 * lane, byte 1 = the code pair's byte, bytes 2..3 =
-    // the table's base.  3-bit: an entry every 128 bytes, offsets OR-ed into the table-size-aligned base.
+    // the table's base.  3- and 2-bit: an entry every 128 bytes, offsets OR-ed into the table-size-aligned base.
     static constexpr int LUT_STRIDE = BITS == 4 ? 256 : 128;
     static constexpr int LUT_BYTES = LUT_ENTRIES * LUT_STRIDE;
     static constexpr int RED_BYTES = kClusterMax * 2 * TILE_ROWS * 4;   // the cluster's partials, [rank][token][row]
@@ -139,6 +139,22 @@ __device__ __forceinline__ void dequant_row_to_tmem(uint32_t qrow, int row, int 
                     // the table's lane address with that byte as byte 1
                     out[wi * 4 + b] = lds_u32(__byte_perm(w[wi], lut_lane, 0x7604u | (uint32_t)(b << 4)));
                 }
+            tmem_st_32x32(taddr + half * 32, out);
+        }
+    } else if constexpr (BITS == 2) {
+        // 32-byte rows: half h is the 16 bytes at 16 h, code pair P at bit 4P of them
+#pragma unroll
+        for (int hh = 0; hh < kHalves; ++hh) {
+            const int half = kHalves == 2 ? hh : ch;
+            const uint4 c0 = lds_v4(qrow + 16 * half);
+            const uint32_t w[4] = {c0.x, c0.y, c0.z, c0.w};
+            uint32_t out[32];
+#pragma unroll
+            for (int pp = 0; pp < 32; ++pp) {
+                const int off = 4 * (pp & 7);
+                const uint32_t sh = off >= 7 ? (w[pp >> 3] >> (off - 7)) : (w[pp >> 3] << (7 - off));
+                out[pp] = lds_u32((sh & 0x780u) | lut_lane);
+            }
             tmem_st_32x32(taddr + half * 32, out);
         }
     } else {
@@ -297,8 +313,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode_kernel(const __grid_
 #pragma unroll
             for (int i = 0; i < C::LUT_ENTRIES / kWorkWarps; ++i) {
                 const int entry = warp + kWorkWarps * i;
-                const int lo = BITS == 4 ? (entry & 15) : (entry & 7);
-                const int hi = BITS == 4 ? (entry >> 4) : (entry >> 3);
+                const int lo = entry & ((1 << BITS) - 1);
+                const int hi = entry >> BITS;
                 const __half2 v = __floats2half2_rn(p.levels[lo], p.levels[hi]);
                 sts_u32(lut + (uint32_t)(entry * C::LUT_STRIDE + 4 * lane), *reinterpret_cast<const uint32_t *>(&v));
             }
@@ -701,16 +717,15 @@ template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem
 
 }  // namespace
 
-// Rules of this path: 3- or 4-bit codes; M <= 2 with M * ceil16(r) <= 64; n a multiple of 32 (4-bit)
-// or 128 (3-bit), which makes every TMA row pitch a multiple of 16 bytes.  Anything else:
-// LORDS_ERR_UNSUPPORTED.
+// Rules of this path: M <= 2 with M * ceil16(r) <= 64; n a multiple of 32 (4-bit), 64 (2-bit) or 128
+// (3-bit), which makes every TMA row pitch a multiple of 16 bytes.  Anything else: LORDS_ERR_UNSUPPORTED.
 int launch_decode(const Problem &p, State &st, cudaStream_t stream)
 {
-    if (p.bits != 3 && p.bits != 4) return LORDS_ERR_UNSUPPORTED;
+    if (p.bits < 2 || p.bits > 4) return LORDS_ERR_UNSUPPORTED;
     if (p.M > 2) return LORDS_ERR_UNSUPPORTED;
     const int r_pad = (p.r + 15) / 16 * 16;
     if (p.M * r_pad > kNMax) return LORDS_ERR_UNSUPPORTED;
-    if (p.n % (p.bits == 4 ? 32 : 128) != 0) return LORDS_ERR_UNSUPPORTED;
+    if (p.n % (p.bits == 4 ? 32 : p.bits == 2 ? 64 : 128) != 0) return LORDS_ERR_UNSUPPORTED;
 
     DecodeParams k;
     k.x = p.x; k.B = p.B;
@@ -720,7 +735,8 @@ int launch_decode(const Problem &p, State &st, cudaStream_t stream)
     k.status = st.status_word;
     int rc;
     if (p.bits == 4) rc = p.M == 1 ? launch_bits_tok<4, 1>(k, p, st, stream) : launch_bits_tok<4, 2>(k, p, st, stream);
-    else rc = p.M == 1 ? launch_bits_tok<3, 1>(k, p, st, stream) : launch_bits_tok<3, 2>(k, p, st, stream);
+    else if (p.bits == 3) rc = p.M == 1 ? launch_bits_tok<3, 1>(k, p, st, stream) : launch_bits_tok<3, 2>(k, p, st, stream);
+    else rc = p.M == 1 ? launch_bits_tok<2, 1>(k, p, st, stream) : launch_bits_tok<2, 2>(k, p, st, stream);
     if (rc != LORDS_OK) return rc;
     st.last_launches = 1;
     st.last_path = "decode";

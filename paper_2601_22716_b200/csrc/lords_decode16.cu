@@ -81,10 +81,10 @@ template <int BITS, int RP> struct XCfg {
     static constexpr int SQ = BITS == 4 ? 4 : 6;               // code-tile ring depth (even: one group per barrier)
     static constexpr int AATOM = RP * 128;                     // RP ranks x 64 columns bf16
     static constexpr int ASTAGE = 2 * AATOM;
-    static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : 64;   // one entry per code pair
+    static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : BITS == 3 ? 64 : 16;   // one entry per code pair
     // 32 lane-private copies of every entry (word = lane).  4-bit: entries 256 bytes apart, table on
-    // a 64 KB boundary, lookup address by one byte permute; 3-bit: entries 128 bytes apart, offsets
-    // OR-ed into the table-size-aligned base.
+    // a 64 KB boundary, lookup address by one byte permute; 3- and 2-bit: entries 128 bytes apart,
+    // offsets OR-ed into the table-size-aligned base.
     static constexpr int LUT_STRIDE = BITS == 4 ? 256 : 128;
     static constexpr int LUT_BYTES = LUT_ENTRIES * LUT_STRIDE;
     static constexpr int RED_BYTES = kClusterMax * kTok * kRows * 4;   // the cluster's partials, [rank][token][row]
@@ -146,6 +146,18 @@ __device__ __forceinline__ void dequant_half_row(uint32_t qrow, int row, int ch,
                 const __half2 wv = __hmul2(*reinterpret_cast<const __half2 *>(&lv), *reinterpret_cast<const __half2 *>(&sp[wi * 4 + b]));
                 sp[wi * 4 + b] = *reinterpret_cast<const uint32_t *>(&wv);
             }
+    } else if constexpr (BITS == 2) {
+        // 32-byte rows: half ch is the 16 bytes at 16 ch, pair P at bit 4P of them
+        const uint4 c0 = lds_v4(qrow + 16 * ch);
+        const uint32_t w[4] = {c0.x, c0.y, c0.z, c0.w};
+#pragma unroll
+        for (int pp = 0; pp < 32; ++pp) {
+            const int off = 4 * (pp & 7);
+            const uint32_t sh = off >= 7 ? (w[pp >> 3] >> (off - 7)) : (w[pp >> 3] << (7 - off));
+            const uint32_t lv = lds_u32((sh & 0x780u) | lut_lane);
+            const __half2 wv = __hmul2(*reinterpret_cast<const __half2 *>(&lv), *reinterpret_cast<const __half2 *>(&sp[pp]));
+            sp[pp] = *reinterpret_cast<const uint32_t *>(&wv);
+        }
     } else {
         // half ch = pairs 32 ch .. 32 ch + 31 = bits 192 ch .. of the 384-bit row = words 6 ch .. 6 ch + 5
         const uint32_t base = qrow + 24 * ch;
@@ -274,8 +286,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
 #pragma unroll
             for (int i = 0; i < C::LUT_ENTRIES / kWorkWarps; ++i) {
                 const int entry = warp + kWorkWarps * i;
-                const int lo = BITS == 4 ? (entry & 15) : (entry & 7);
-                const int hi = BITS == 4 ? (entry >> 4) : (entry >> 3);
+                const int lo = entry & ((1 << BITS) - 1);
+                const int hi = entry >> BITS;
                 const __half2 v = __floats2half2_rn(p.levels[lo], p.levels[hi]);
                 sts_u32(lut + (uint32_t)(entry * C::LUT_STRIDE + 4 * lane), *reinterpret_cast<const uint32_t *>(&v));
             }
@@ -651,16 +663,16 @@ template <int BITS, int RP> int launch_variant(Dec16Params &k, const Problem &p,
 
 }  // namespace
 
-// Rules of this path: 3- or 4-bit codes; M <= 16 (with automatic dispatch one or two tokens go to the
+// Rules of this path: M <= 16 (with automatic dispatch one or two tokens go to the
 // reassociated decode kernel first, and come here when that one declines the rank); r <= 32 (4-bit) or <= 64 (3-bit), which is what the shared-memory layout holds;
-// n a multiple of 64 (4-bit) or 128 (3-bit), which makes every TMA row pitch a multiple of 16 bytes.
+// n a multiple of 64 (2- and 4-bit) or 128 (3-bit), which makes every TMA row pitch a multiple of 16 bytes.
 // Anything else: LORDS_ERR_UNSUPPORTED.
 int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
 {
-    if (p.bits != 3 && p.bits != 4) return LORDS_ERR_UNSUPPORTED;
+    if (p.bits < 2 || p.bits > 4) return LORDS_ERR_UNSUPPORTED;
     if (p.M > kTok) return LORDS_ERR_UNSUPPORTED;
     if (p.r > (p.bits == 4 ? 32 : 64)) return LORDS_ERR_UNSUPPORTED;
-    if (p.n % (p.bits == 4 ? 64 : 128) != 0) return LORDS_ERR_UNSUPPORTED;
+    if (p.n % (p.bits == 3 ? 128 : 64) != 0) return LORDS_ERR_UNSUPPORTED;
 
     Dec16Params k;
     k.B = p.B;
@@ -672,7 +684,8 @@ int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
     k.status = st.status_word;
     int rc;
     if (p.bits == 4) rc = launch_variant<4, 32>(k, p, st, stream);
-    else rc = k.r_pad <= 32 ? launch_variant<3, 32>(k, p, st, stream) : launch_variant<3, 64>(k, p, st, stream);
+    else if (p.bits == 3) rc = k.r_pad <= 32 ? launch_variant<3, 32>(k, p, st, stream) : launch_variant<3, 64>(k, p, st, stream);
+    else rc = k.r_pad <= 32 ? launch_variant<2, 32>(k, p, st, stream) : launch_variant<2, 64>(k, p, st, stream);
     if (rc != LORDS_OK) return rc;
     st.last_launches = 1;
     st.last_path = "decode16";

@@ -109,6 +109,14 @@ DECODE_SHAPES = [
     (3, 520, 1152, 48, 1, True),
     (3, 256, 128, 16, 2, False),
     (3, 2048, 4096, 32, 2, False),
+    # 2-bit codes and ranks of the paper's Table 7 (6, 12, 15: rows of B that are not 16-byte multiples)
+    (2, 512, 4096, 32, 2, False),
+    (2, 300, 1088, 6, 1, True),      # ragged rows; n = 8.5 k-steps; r padded to 16
+    (2, 1000, 2048, 15, 2, True),
+    (2, 64, 8192, 64, 1, False),
+    (2, 256, 64, 12, 1, True),       # half a k-step
+    (4, 512, 1024, 12, 2, True),
+    (3, 384, 1024, 15, 1, True),
 ]
 
 
@@ -122,7 +130,7 @@ def test_decode_kernel_shapes(lords, bits, m, n, r, M, mixed):
 
 
 @pytest.mark.parametrize("bits,m,n,r,M", [(4, 700, 2048, 32, 1), (4, 256, 1024, 16, 2), (3, 384, 1024, 48, 1),
-                                          (3, 131, 256, 8, 2)])
+                                          (3, 131, 256, 8, 2), (2, 300, 1024, 6, 1), (2, 512, 320, 24, 2)])
 def test_decode_kernel_integer_case_is_bit_exact(lords, bits, m, n, r, M):
     lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m)
     dl, y32, ybf = _run(lords, lay, "decode")
@@ -182,6 +190,12 @@ DECODE16_SHAPES = [
     (3, 2048, 4096, 32, 8, False),
     (3, 640, 2048, 48, 2, True),      # two tokens with a rank the reassociated kernel declines
     (4, 256, 512, 32, 1, False),
+    # 2-bit codes and ranks of the paper's Table 7
+    (2, 384, 1024, 32, 5, True),
+    (2, 300, 1088, 6, 3, True),
+    (2, 1000, 2048, 48, 16, True),
+    (2, 256, 64, 12, 9, True),
+    (4, 512, 1024, 15, 8, True),
 ]
 
 
@@ -195,7 +209,7 @@ def test_decode16_kernel_shapes(lords, bits, m, n, r, M, mixed):
 
 
 @pytest.mark.parametrize("bits,m,n,r,M", [(4, 700, 2048, 32, 8), (4, 256, 512, 16, 16), (3, 384, 1024, 48, 3),
-                                          (3, 131, 384, 7, 9)])
+                                          (3, 131, 384, 7, 9), (2, 300, 1024, 5, 4), (2, 256, 192, 40, 16)])
 def test_decode16_kernel_integer_case_is_bit_exact(lords, bits, m, n, r, M):
     lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m + M)
     dl, y32, ybf = _run(lords, lay, "decode16")
