@@ -14,6 +14,38 @@ State &state()
     return s;
 }
 
+// Small host buffers are moved by a kernel that reads or writes the pinned host memory directly
+// (mapped into the device's address space): two DMA copies of a few KB cost about 10 us each in
+// latency, a kernel's loads and stores across the bus about 2 us.
+__global__ void lords_copy16_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, size_t n16)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) dst[i] = src[i];
+}
+
+constexpr size_t kDirectHostBytes = 1u << 20;   // above this the copy engines win
+
+// The device's address of a pinned, mapped host buffer; false for pageable or foreign memory.
+static bool mapped_device_pointer(const void *host, void **dev)
+{
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, host) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    if (a.type != cudaMemoryTypeHost || a.devicePointer == nullptr) return false;
+    *dev = a.devicePointer;
+    return true;
+}
+
+static int copy16(const void *src, void *dst, size_t bytes, cudaStream_t s)
+{
+    const size_t n16 = bytes / 16;
+    const unsigned blocks = (unsigned)((n16 + 255) / 256 < 64 ? (n16 + 255) / 256 : 64);
+    lords_copy16_kernel<<<blocks, 256, 0, s>>>(static_cast<const uint4 *>(src), static_cast<uint4 *>(dst), n16);
+    LORDS_CUDA_TRY(cudaGetLastError());
+    return LORDS_OK;
+}
+
 int cuda_fail(cudaError_t e)
 {
     state().last_cuda_error = (int)e;
@@ -277,10 +309,27 @@ int lords_linear_forward_host(const void *x_host, const uint8_t *Qpacked, const 
         st.stage_y_bytes = yb;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    LORDS_CUDA_TRY(cudaMemcpyAsync(st.stage_x, x_host, xb, cudaMemcpyHostToDevice, s));
-    int rc = forward_common(st.stage_x, Qpacked, B, A, codebook, bits, M, m, n, r, st.stage_y, 0, stream);
+    void *x_map = nullptr, *y_map = nullptr;
+    const bool aligned = xb % 16 == 0 && yb % 16 == 0 && (reinterpret_cast<uintptr_t>(x_host) | reinterpret_cast<uintptr_t>(y_host)) % 16 == 0;
+    const bool direct = aligned && xb <= kDirectHostBytes && yb <= kDirectHostBytes && mapped_device_pointer(x_host, &x_map) &&
+                        mapped_device_pointer(y_host, &y_map);
+    int rc;
+    if (direct) {
+        rc = copy16(x_map, st.stage_x, xb, s);
+        if (rc != LORDS_OK) return rc;
+    } else {
+        LORDS_CUDA_TRY(cudaMemcpyAsync(st.stage_x, x_host, xb, cudaMemcpyHostToDevice, s));
+    }
+    rc = forward_common(st.stage_x, Qpacked, B, A, codebook, bits, M, m, n, r, st.stage_y, 0, stream);
     if (rc != LORDS_OK) return rc;
-    LORDS_CUDA_TRY(cudaMemcpyAsync(y_host, st.stage_y, yb, cudaMemcpyDeviceToHost, s));
+    const int kernels = st.last_launches;
+    if (direct) {
+        rc = copy16(st.stage_y, y_map, yb, s);
+        if (rc != LORDS_OK) return rc;
+        st.last_launches = kernels + 2;
+    } else {
+        LORDS_CUDA_TRY(cudaMemcpyAsync(y_host, st.stage_y, yb, cudaMemcpyDeviceToHost, s));
+    }
     return LORDS_OK;
 }
 
