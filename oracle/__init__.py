@@ -50,6 +50,8 @@ def _load():
         lib.lords_oracle_round_bf16.argtypes = [p, i64, p]
         lib.lords_oracle_quantize.restype = ci
         lib.lords_oracle_quantize.argtypes = [p, p, p, p, ci, i64, i64, i64, p, p, p, p]
+        lib.lords_oracle_backward.restype = ci
+        lib.lords_oracle_backward.argtypes = [p, p, p, p, p, p, ci, i64, i64, i64, i64, p, p, p]
         lib.lords_oracle_equivalent_rank.restype = i64
         lib.lords_oracle_equivalent_rank.argtypes = [i64, i64, i64]
         _lib = lib
@@ -165,3 +167,21 @@ def quantize(W, B, A, codebook, bits: int, details: bool = False):
         raise ValueError(f"oracle quantize failed: {rc}")
     return (codes, runner, gap, mag) if details else codes
 
+
+def backward(g, x, qpacked, B, A, codebook, bits: int):
+    """Gradients of sum(g * y) for y = x W^T with the codes fixed (Sec. 3.4): (dx [M, n], dB [m, r], dA [r, n]), fp64.
+
+    g and x are bf16 bit patterns [M, m] and [M, n]."""
+    g = _c(g, np.uint16); x = _c(x, np.uint16); B = _c(B, np.uint16); A = _c(A, np.uint16)
+    qpacked = _c(qpacked, np.uint8); codebook = _c(codebook, np.float32)
+    M, n = x.shape
+    m, r = B.shape
+    assert g.shape == (M, m) and A.shape == (r, n) and codebook.size == 2**bits and qpacked.size == packed_bytes(m, n, bits)
+    dx = np.empty((M, n), dtype=np.float64)
+    dB = np.empty((m, r), dtype=np.float64)
+    dA = np.empty((r, n), dtype=np.float64)
+    rc = _load().lords_oracle_backward(_ptr(g), _ptr(x), _ptr(qpacked), _ptr(B), _ptr(A), _ptr(codebook), bits,
+                                       M, m, n, r, _ptr(dx), _ptr(dB), _ptr(dA))
+    if rc != 0:
+        raise ValueError(f"oracle backward failed: {rc}")
+    return dx, dB, dA

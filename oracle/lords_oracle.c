@@ -32,6 +32,15 @@
  * Not pinned: a forward output on real model weights -- the paper prints no
  * worked numeric example of the forward path ("parity unpinned" for that only).
  *
+ * The backward of the layer with the codes frozen (multiplicative fine-tuning of B and A, Sec. 3.4;
+ * the chain rule through W^ = L[Q] (.) (BA) as in Eq. 5's gradient with respect to S) is stated in
+ * lords_oracle_backward: with g = dL/dy,
+ *     dx = g W^,    dW^ = g^T x,    dS = dW^ (.) L[Q],    dB = dS A^T,    dA = B^T dS.
+ * Pins: y is linear in every single entry of x, B and A, so replacing one entry by another bf16 value
+ * changes the scalar sum(g (.) y) of two forward passes by exactly (difference) x (gradient entry);
+ * the tests take such differences on sampled entries, and check <g, y> identities that follow from
+ * linearity (sum(dx (.) x) = sum(dB (.) B) = sum(dA (.) A) = sum(g (.) y)).
+ *
  * The step before the path, the quantisation step of Alg. 1 (step 2.1), is stated here too
  * (lords_oracle_quantize): Q_ij = argmin over the levels v of (S_ij v - W_ij)^2 with S = BA, every
  * level tried in turn in fp64.  The paper does not say which level wins a tie: the lowest code does.
@@ -293,5 +302,60 @@ int lords_oracle_quantize(const uint16_t *W, const uint16_t *B, const uint16_t *
         free(S_row);
     }
     return rc;
+}
+
+/*
+ * Backward of y = x W^T, W^ = L[Q] (.) (B A), with the codes fixed (Sec. 3.4: only B and A are trained;
+ * Eq. 5 gives the same chain rule through S = BA).  g = dL/dy is M x m (bf16 bit patterns, like x).
+ *   dx = g W^                       M x n
+ *   dW^ = g^T x                     m x n   (held row by row only)
+ *   dS  = dW^ (.) L[Q]
+ *   dB  = dS A^T                    m x r
+ *   dA  = B^T dS                    r x n
+ * Any of dx, dB, dA may be NULL.  fp64, sums in index order (dA: rows of W in order).
+ */
+int lords_oracle_backward(const uint16_t *g, const uint16_t *x, const uint8_t *qpacked, const uint16_t *B,
+                          const uint16_t *A, const float *codebook, int bits, int64_t M, int64_t m, int64_t n,
+                          int64_t r, double *dx, double *dB, double *dA)
+{
+    if (!g || !x || !qpacked || !B || !A || !codebook || M < 1 || m < 1 || n < 1 || r < 1 || !group_ok(n, bits))
+        return ORACLE_ERR_ARG;
+    int64_t row_bytes = n * bits / 8;
+    double *S_row = (double *)malloc(sizeof(double) * (size_t)n);
+    double *dS_row = (double *)malloc(sizeof(double) * (size_t)n);
+    if (!S_row || !dS_row) {
+        free(S_row); free(dS_row);
+        return ORACLE_ERR_NOMEM;
+    }
+    if (dx) for (int64_t e = 0; e < M * n; ++e) dx[e] = 0.0;
+    if (dA) for (int64_t e = 0; e < r * n; ++e) dA[e] = 0.0;
+    for (int64_t i = 0; i < m; ++i) {
+        const uint8_t *qrow = qpacked + i * row_bytes;
+        scale_row(B, A, n, r, i, S_row);                                        /* S_i = (BA)_i */
+        for (int64_t j = 0; j < n; ++j) {
+            double level = (double)codebook[read_code(qrow, j, bits)];
+            double dW = 0.0;                                                    /* dW^_ij = sum_t g_ti x_tj */
+            for (int64_t t = 0; t < M; ++t) dW += bf16_to_f64(g[t * m + i]) * bf16_to_f64(x[t * n + j]);
+            dS_row[j] = dW * level;                                             /* dS_ij = dW^_ij L[Q_ij] */
+            if (dx) {
+                double w = level * S_row[j];                                    /* W^_ij */
+                for (int64_t t = 0; t < M; ++t) dx[t * n + j] += bf16_to_f64(g[t * m + i]) * w;
+            }
+        }
+        if (dB)
+            for (int64_t k = 0; k < r; ++k) {                                   /* dB_ik = sum_j dS_ij A_kj */
+                double acc = 0.0;
+                for (int64_t j = 0; j < n; ++j) acc += dS_row[j] * bf16_to_f64(A[k * n + j]);
+                dB[i * r + k] = acc;
+            }
+        if (dA)
+            for (int64_t k = 0; k < r; ++k) {                                   /* dA_kj += B_ik dS_ij */
+                double b = bf16_to_f64(B[i * r + k]);
+                for (int64_t j = 0; j < n; ++j) dA[k * n + j] += b * dS_row[j];
+            }
+    }
+    free(S_row);
+    free(dS_row);
+    return ORACLE_OK;
 }
 

@@ -304,3 +304,73 @@ def test_quantize_is_monotone_in_the_weight_for_positive_scales():
     assert (np.diff(got.astype(np.int32), axis=0) >= 0).all()
     assert got.min() == 0 and got.max() == 15            # the grid reaches both ends of the table
 
+
+
+# ---- backward with the codes fixed (Sec. 3.4; chain rule of Eq. 5 through S = BA) ------------------------
+
+def _loss(g, y64):
+    """The scalar whose gradients the backward returns: sum(g * y), g widened exactly."""
+    return float(np.sum(gen.bf16_to_f32(g).astype(np.float64) * y64))
+
+
+def _replace_entry(bits16, idx, factor=1.5):
+    """A copy of a bf16 array with one entry multiplied by 1.5 (exact in bf16 for these inputs' few
+    significand bits or not -- the returned difference is the exact one either way)."""
+    import torch
+    out = bits16.copy()
+    old = float(gen.bf16_to_f32(bits16[idx:idx + 1] if bits16.ndim == 1 else np.array([bits16[idx]], dtype=np.uint16))[0])
+    new_bits = gen.bf16_bits(torch.tensor([old * factor + 0.25]))
+    out[idx] = new_bits[0]
+    new = float(gen.bf16_to_f32(new_bits)[0])
+    return out, new - old
+
+
+@pytest.mark.parametrize("bits,m,n,r,M,mixed", [(4, 24, 64, 5, 3, True), (3, 16, 96, 3, 2, True), (2, 20, 40, 4, 4, False)])
+def test_backward_matches_exact_differences_of_the_forward(bits, m, n, r, M, mixed):
+    """y is linear in every single entry of x, of B and of A.  Replacing one entry by another bf16
+    value therefore changes sum(g * y) by exactly (new - old) * (that entry of the gradient), up to
+    fp64 rounding: a finite difference with no truncation error, through the forward oracle only."""
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=11 * m + n, mixed_sign=mixed)
+    packed = oracle.pack_codes(lay.codes, bits)
+    g = gen.make_layer(m, m, 1, M, bits=4, seed=5).x[:, :m].copy()          # any bf16 numbers, M x m
+    dx, dB, dA = oracle.backward(g, lay.x, packed, lay.B, lay.A, lay.codebook, bits)
+    base = _loss(g, oracle.forward(lay.x, packed, lay.B, lay.A, lay.codebook, bits))
+    rng = np.random.default_rng(m + n)
+    scale = max(1.0, abs(base))
+    for _ in range(12):
+        t, j = int(rng.integers(M)), int(rng.integers(n))
+        x2, d = _replace_entry(lay.x.reshape(-1), t * n + j)
+        l2 = _loss(g, oracle.forward(x2.reshape(M, n), packed, lay.B, lay.A, lay.codebook, bits))
+        assert abs((l2 - base) - d * dx[t, j]) <= 1e-11 * scale * max(1.0, abs(d))
+        i, k = int(rng.integers(m)), int(rng.integers(r))
+        B2, d = _replace_entry(lay.B.reshape(-1), i * r + k)
+        l2 = _loss(g, oracle.forward(lay.x, packed, B2.reshape(m, r), lay.A, lay.codebook, bits))
+        assert abs((l2 - base) - d * dB[i, k]) <= 1e-11 * scale * max(1.0, abs(d))
+        k, j = int(rng.integers(r)), int(rng.integers(n))
+        A2, d = _replace_entry(lay.A.reshape(-1), k * n + j)
+        l2 = _loss(g, oracle.forward(lay.x, packed, lay.B, A2.reshape(r, n), lay.codebook, bits))
+        assert abs((l2 - base) - d * dA[k, j]) <= 1e-11 * scale * max(1.0, abs(d))
+
+
+def test_backward_euler_identities():
+    """y is homogeneous of degree one in x, in B and in A separately, so each gradient paired with its
+    own argument gives back the loss: <dx, x> = <dB, B> = <dA, A> = sum(g * y)."""
+    lay = gen.make_layer(40, 128, 6, 5, bits=4, seed=3, mixed_sign=True)
+    packed = oracle.pack_codes(lay.codes, 4)
+    g = gen.make_layer(40, 64, 1, 5, bits=4, seed=8).x[:, :40].copy()
+    dx, dB, dA = oracle.backward(g, lay.x, packed, lay.B, lay.A, lay.codebook, 4)
+    loss = _loss(g, oracle.forward(lay.x, packed, lay.B, lay.A, lay.codebook, 4))
+    f64 = lambda b: gen.bf16_to_f32(b).astype(np.float64)
+    for got in (np.sum(dx * f64(lay.x)), np.sum(dB * f64(lay.B)), np.sum(dA * f64(lay.A))):
+        assert abs(got - loss) <= 1e-10 * max(1.0, abs(loss))
+
+
+def test_backward_input_gradient_is_g_times_the_dequantised_weight():
+    """dx = g W^: a library matmul with the oracle's own dequantised rows (pinned by P1/P2)."""
+    lay = gen.make_layer(48, 96, 7, 3, bits=3, seed=21, mixed_sign=True)
+    packed = oracle.pack_codes(lay.codes, 3)
+    g = gen.make_layer(48, 64, 1, 3, bits=4, seed=9).x[:, :48].copy()
+    dx, _, _ = oracle.backward(g, lay.x, packed, lay.B, lay.A, lay.codebook, 3)
+    What = oracle.dequant_rows(packed, lay.B, lay.A, lay.codebook, 3)
+    want = gen.bf16_to_f32(g).astype(np.float64) @ What
+    assert np.allclose(dx, want, rtol=1e-12, atol=1e-12 * np.abs(want).max())
