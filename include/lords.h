@@ -182,6 +182,34 @@ int lords_quantize_codes(const void *W, const void *B, const void *A, const floa
                          int r, uint8_t *Qpacked, void *stream);
 
 /*
+ * Backward of the layer with the codes fixed: what multiplicative fine-tuning of B and A needs
+ * (Sec. 3.4; the chain rule through S = BA is that of Eq. 5).  With g = dL/dy, bf16 [M][m]:
+ *     dx = g W^  [M][n],     dS = (g^T x) (.) L[Q]  (never stored),     dB = dS A^T  [m][r],     dA = B^T dS  [r][n].
+ *
+ * lords_transpose_codes: Qt_packed (device, lords_packed_bytes(n, m, bits) bytes) receives the packed
+ *   codes of Q^T, n rows of m codes; m must be a multiple of the pack group like n.  The codes are
+ *   frozen during fine-tuning, so this is done once per layer.
+ * lords_linear_backward_input[_f32]: dx = g W^ as the forward of the transposed layer,
+ *   W^T = L[Q^T] (.) (A^T B^T): the same kernels, dispatch, operand ranges and error behaviour as the
+ *   forward calls, with (m, n) exchanged.  B and A are the layer's own factors ([m][r], [r][n]); their
+ *   transposes are made per call in library-owned scratch that grows (cudaMalloc) when a larger layer
+ *   is seen, so the first call of a given size must not be made during stream capture.
+ *   dx: device, bf16 [M][n] (or float [M][n] for _f32).
+ * lords_linear_backward_factors: dB (device, float [m][r]) and dA (device, float [r][n]); either may
+ *   be NULL.  fp32 on the CUDA cores, every element summed by one thread in a fixed order (runs are
+ *   bit-identical).  x: device, bf16 [M][n].  Any bits in {2,3,4}, r <= LORDS_R_MAX.
+ * All enqueue on `stream` and return without synchronising; all need lords_init.
+ */
+int lords_transpose_codes(const uint8_t *Qpacked, int bits, int m, int n, uint8_t *Qt_packed, void *stream);
+int lords_linear_backward_input(const void *dy, const uint8_t *Qt_packed, const void *B, const void *A, const float *codebook,
+                                int bits, int M, int m, int n, int r, void *dx, void *stream);
+int lords_linear_backward_input_f32(const void *dy, const uint8_t *Qt_packed, const void *B, const void *A,
+                                    const float *codebook, int bits, int M, int m, int n, int r, float *dx32, void *stream);
+int lords_linear_backward_factors(const void *dy, const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                                  const float *codebook, int bits, int M, int m, int n, int r, float *dB, float *dA,
+                                  void *stream);
+
+/*
  * Allocation-free forward (the paper has no counterpart: this is a deployment convenience).
  * For callers that must not allocate device memory -- for instance a plugin inside a server
  * whose memory pool already owns all of HBM, or a latency-critical loop that cannot take the

@@ -49,6 +49,10 @@ def _load():
         "lords_linear_forward_host": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_forward_noalloc": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_quantize_codes": (ci, [p, p, p, p, ci, ci, ci, ci, p, p]),
+        "lords_transpose_codes": (ci, [p, ci, ci, ci, p, p]),
+        "lords_linear_backward_input": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
+        "lords_linear_backward_input_f32": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
+        "lords_linear_backward_factors": (ci, [p, p, p, p, p, p, ci, ci, ci, ci, ci, p, p, p]),
         "lords_poll_status": (ci, [p]),
         "lords_read_status_detail": (ci, [p]),
         "lords_last_cuda_error": (ci, []),
@@ -73,7 +77,8 @@ def exported_symbols():
     return ["lords_version", "lords_strerror", "lords_equivalent_rank", "lords_packed_bytes",
             "lords_pack_codes", "lords_unpack_codes", "lords_init", "lords_shutdown",
             "lords_linear_forward", "lords_linear_forward_bits", "lords_linear_forward_f32",
-            "lords_linear_forward_host", "lords_linear_forward_noalloc", "lords_quantize_codes", "lords_poll_status", "lords_read_status_detail", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
+            "lords_linear_forward_host", "lords_linear_forward_noalloc", "lords_quantize_codes", "lords_transpose_codes",
+            "lords_linear_backward_input", "lords_linear_backward_input_f32", "lords_linear_backward_factors", "lords_poll_status", "lords_read_status_detail", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
             "lords_last_launch_count"]
 
 
@@ -190,6 +195,37 @@ def lords_quantize_codes(W, B, A, codebook, bits, m, n, r, Qpacked, stream=None)
     cb = _cb_ptr(codebook, bits)
     _check(_load().lords_quantize_codes(W.data_ptr(), B.data_ptr(), A.data_ptr(), cb.ctypes.data, bits, m, n, r,
                                         Qpacked.data_ptr(), _stream_ptr(stream)), "lords_quantize_codes")
+
+
+def lords_transpose_codes(Qpacked, bits, m, n, Qt_packed, stream=None) -> None:
+    """Packed codes of Q^T (n rows of m codes) from the packed codes of Q, on the device."""
+    _check(_load().lords_transpose_codes(Qpacked.data_ptr(), bits, m, n, Qt_packed.data_ptr(), _stream_ptr(stream)),
+           "lords_transpose_codes")
+
+
+def lords_linear_backward_input(dy, Qt_packed, B, A, codebook, bits, M, m, n, r, dx, stream=None) -> None:
+    """dx = dy W^ (bf16 [M, n]) for a layer whose transposed codes Qt_packed were made by lords_transpose_codes."""
+    cb = _cb_ptr(codebook, bits)
+    _check(_load().lords_linear_backward_input(dy.data_ptr(), Qt_packed.data_ptr(), B.data_ptr(), A.data_ptr(), cb.ctypes.data,
+                                               bits, M, m, n, r, dx.data_ptr(), _stream_ptr(stream)),
+           "lords_linear_backward_input")
+
+
+def lords_linear_backward_input_f32(dy, Qt_packed, B, A, codebook, bits, M, m, n, r, dx32, stream=None) -> None:
+    """The same with the fp32 accumulator stored (float [M, n])."""
+    cb = _cb_ptr(codebook, bits)
+    _check(_load().lords_linear_backward_input_f32(dy.data_ptr(), Qt_packed.data_ptr(), B.data_ptr(), A.data_ptr(),
+                                                   cb.ctypes.data, bits, M, m, n, r, dx32.data_ptr(), _stream_ptr(stream)),
+           "lords_linear_backward_input_f32")
+
+
+def lords_linear_backward_factors(dy, x, Qpacked, B, A, codebook, bits, M, m, n, r, dB, dA, stream=None) -> None:
+    """dB (float [m, r]) and dA (float [r, n]) of the layer with the codes fixed; either may be None."""
+    cb = _cb_ptr(codebook, bits)
+    _check(_load().lords_linear_backward_factors(dy.data_ptr(), x.data_ptr(), Qpacked.data_ptr(), B.data_ptr(), A.data_ptr(),
+                                                 cb.ctypes.data, bits, M, m, n, r,
+                                                 None if dB is None else dB.data_ptr(), None if dA is None else dA.data_ptr(),
+                                                 _stream_ptr(stream)), "lords_linear_backward_factors")
 
 
 def lords_poll_status(stream=None) -> int:

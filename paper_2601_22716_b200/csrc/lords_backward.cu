@@ -1,0 +1,256 @@
+// Backward of the layer y = x W^T, W^ = L[Q] (.) (B A), with the codes fixed: the gradients that
+// multiplicative fine-tuning of B and A needs (Sec. 3.4; the chain rule through S = BA is the one of
+// Eq. 5).  With g = dL/dy (M x m):
+//
+//     dx = g W^                                   (M x n)
+//     dS = (g^T x) (.) L[Q]                       (m x n, never stored: built tile by tile)
+//     dB = dS A^T   (m x r),     dA = B^T dS      (r x n)
+//
+// dx is the forward operator of the transposed layer: W^T = L[Q^T] (.) (A^T B^T), so with a transposed
+// copy of the packed codes (made once: the codes are frozen) and the transposed factors it runs on the
+// forward kernels as they are.  This file holds what that needs -- the transposition of packed codes
+// and of a bf16 matrix -- and the kernels for dB and dA.
+//
+// dB and dA run on the CUDA cores in fp32 (bf16 inputs are widened exactly).  One kernel, two roles:
+//   role 0 (dB): a CTA owns 64 rows of W and walks over the columns in steps of 64;
+//   role 1 (dA): a CTA owns 64 columns and walks over the rows in steps of 64.
+// Per step it forms the 64 x 64 tile of g^T x by a shared-memory-tiled product over the tokens,
+// multiplies by the levels of the tile's codes, and folds the tile into its accumulators with the
+// matching 64-column (or 64-row) slice of A (or B).  Every output element is summed by one thread in
+// a fixed order: no atomics, runs are bit-identical.  Bound: fp32 ALU, 2 m n M fused multiply-adds
+// for the two roles together (the tile of g^T x is formed once per role).
+#include <cuda_runtime.h>
+
+#include "lords_internal.h"
+
+namespace lords {
+
+namespace {
+
+__device__ __forceinline__ float bf16f(uint16_t h) { return __uint_as_float((uint32_t)h << 16); }
+
+// Code (i, j) of a packed row-major code matrix with `row_bytes` bytes per row.
+__device__ __forceinline__ uint32_t read_code(const uint8_t *__restrict__ q, size_t row_bytes, int i, int j, int bits)
+{
+    const uint8_t *row = q + (size_t)i * row_bytes;
+    const int bit = j * bits, byte = bit >> 3, sh = bit & 7;
+    uint32_t v = row[byte];
+    if (sh + bits > 8) v |= (uint32_t)row[byte + 1] << 8;
+    return (v >> sh) & ((1u << bits) - 1u);
+}
+
+// ---- transposition of packed codes -----------------------------------------------------------------
+// Thread (j, group): the codes Q[i0 .. i0 + 31][j] become 32 consecutive codes of row j of Q^T.
+// Neighbouring threads take neighbouring j, so the reads of one row of Q are contiguous.
+__global__ void lords_transpose_codes_kernel(const uint8_t *__restrict__ Q, uint8_t *__restrict__ Qt, int m, int n, int bits)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i0 = blockIdx.y * 32;
+    if (j >= n) return;
+    const size_t row_bytes = (size_t)n * bits / 8, trow_bytes = (size_t)m * bits / 8;
+    const int count = m - i0 < 32 ? m - i0 : 32;        // a multiple of the pack group, like m
+    unsigned long long lo = 0;                          // up to 128 bits of packed codes
+    unsigned long long hi = 0;
+    for (int ii = 0; ii < count; ++ii) {
+        const unsigned long long c = read_code(Q, row_bytes, i0 + ii, j, bits);
+        const int bit = ii * bits;
+        if (bit < 64) {
+            lo |= c << bit;
+            if (bit + bits > 64) hi |= c >> (64 - bit);
+        } else {
+            hi |= c << (bit - 64);
+        }
+    }
+    uint8_t *dst = Qt + (size_t)j * trow_bytes + (size_t)i0 * bits / 8;
+    const int bytes = count * bits / 8;
+    for (int b = 0; b < bytes; ++b) dst[b] = (uint8_t)(b < 8 ? lo >> (8 * b) : hi >> (8 * (b - 8)));
+}
+
+// ---- transposition of a bf16 matrix [rows][cols] -> [cols][rows] --------------------------------------
+__global__ void lords_transpose_bf16_kernel(const uint16_t *__restrict__ src, uint16_t *__restrict__ dst, int rows, int cols)
+{
+    __shared__ uint16_t tile[32][33];
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int k = threadIdx.y; k < 32; k += blockDim.y) {
+        const int rr = r0 + k, cc = c0 + threadIdx.x;
+        tile[k][threadIdx.x] = (rr < rows && cc < cols) ? src[(size_t)rr * cols + cc] : (uint16_t)0;
+    }
+    __syncthreads();
+    for (int k = threadIdx.y; k < 32; k += blockDim.y) {
+        const int cc = c0 + k, rr = r0 + threadIdx.x;
+        if (cc < cols && rr < rows) dst[(size_t)cc * rows + rr] = tile[threadIdx.x][k];
+    }
+}
+
+// ---- dB and dA -------------------------------------------------------------------------------------------
+constexpr int kT = 64;          // tile edge (rows of W and columns of W per step)
+constexpr int kTok = 16;        // tokens per shared-memory slice of the g^T x product
+constexpr int kBwThreads = 256;
+constexpr int kRMaxBw = 128;    // = LORDS_R_MAX
+
+struct BwParams {
+    const uint16_t *g;    // bf16 [M][m]
+    const uint16_t *x;    // bf16 [M][n]
+    const uint8_t *q;     // packed codes [m][n * bits / 8]
+    const uint16_t *B;    // bf16 [m][r]
+    const uint16_t *A;    // bf16 [r][n]
+    float levels[16];
+    int bits, M, m, n, r;
+    float *dB;            // [m][r]
+    float *dA;            // [r][n]
+};
+
+// ROLE 0: dB for rows blockIdx.x * 64 ..; ROLE 1: dA for columns blockIdx.x * 64 ...
+template <int ROLE>
+__global__ void __launch_bounds__(kBwThreads) lords_backward_factors_kernel(const BwParams p)
+{
+    __shared__ __align__(16) float gs[kTok][kT];   // g[t][i0 + ..]
+    __shared__ __align__(16) float xs[kTok][kT];   // x[t][j0 + ..]
+    __shared__ float ds[kT][kT + 1];               // dS tile
+    __shared__ uint16_t fs[kRMaxBw][kT + 2];       // ROLE 0: A[k][j0 + ..]; ROLE 1: B[i0 + ..][k] stored [k][i]
+                                                   // (rows 33 words apart: neighbouring k fall into different banks)
+
+    const int tid = threadIdx.x;
+    const int ty = tid >> 4, tx = tid & 15;   // 16 x 16 threads, a 4 x 4 micro-tile each
+    const int own0 = blockIdx.x * kT;         // first owned row (ROLE 0) or column (ROLE 1)
+    const int walk_len = ROLE == 0 ? p.n : p.m;
+    const size_t row_bytes = (size_t)p.n * p.bits / 8;
+
+    // accumulators: output element e = tid + 256 * a of the owned [64][r] (ROLE 0: [i][k]) or [r][64]
+    // (ROLE 1: [k][j]) block
+    // (r rounded up to a multiple of 4, so that the block is a whole number of elements per thread)
+    constexpr int kAccMax = kRMaxBw * kT / kBwThreads;     // 32
+    float acc[kAccMax];
+    const int r4 = (p.r + 3) & ~3;
+    const int nacc4 = r4 * kT / kBwThreads;
+#pragma unroll
+    for (int a = 0; a < kAccMax; ++a) acc[a] = 0.0f;
+
+    for (int w0 = 0; w0 < walk_len; w0 += kT) {
+        const int i0 = ROLE == 0 ? own0 : w0, j0 = ROLE == 0 ? w0 : own0;
+        // ---- tile of g^T x over all tokens
+        float c[4][4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) c[a][b] = 0.0f;
+        for (int t0 = 0; t0 < p.M; t0 += kTok) {
+            for (int e = tid; e < kTok * kT; e += kBwThreads) {
+                const int t = t0 + e / kT, cidx = e % kT;
+                gs[e / kT][cidx] = (t < p.M && i0 + cidx < p.m) ? bf16f(p.g[(size_t)t * p.m + i0 + cidx]) : 0.0f;
+                xs[e / kT][cidx] = (t < p.M && j0 + cidx < p.n) ? bf16f(p.x[(size_t)t * p.n + j0 + cidx]) : 0.0f;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int t = 0; t < kTok; ++t) {
+                const float4 g4 = *reinterpret_cast<const float4 *>(&gs[t][ty * 4]);
+                const float4 x4 = *reinterpret_cast<const float4 *>(&xs[t][tx * 4]);
+                const float gv[4] = {g4.x, g4.y, g4.z, g4.w}, xv[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) c[a][b] = fmaf(gv[a], xv[b], c[a][b]);
+            }
+            __syncthreads();
+        }
+        // ---- dS = (g^T x) (.) L[Q]
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int i = i0 + ty * 4 + a, j = j0 + tx * 4 + b;
+                float lv = 0.0f;
+                if (i < p.m && j < p.n) lv = p.levels[read_code(p.q, row_bytes, i, j, p.bits)];
+                ds[ty * 4 + a][tx * 4 + b] = c[a][b] * lv;
+            }
+        // ---- the factor slice that folds the tile: A[:, j0 ..] (ROLE 0) or B[i0 .., :] (ROLE 1), zero padded
+        for (int e = tid; e < r4 * kT; e += kBwThreads) {
+            const int k = e / kT, cidx = e % kT;
+            uint16_t v = 0;
+            if (k < p.r) {
+                if (ROLE == 0) { if (j0 + cidx < p.n) v = p.A[(size_t)k * p.n + j0 + cidx]; }
+                else { if (i0 + cidx < p.m) v = p.B[(size_t)(i0 + cidx) * p.r + k]; }
+            }
+            fs[k][cidx] = v;
+        }
+        __syncthreads();
+        // ---- fold: ROLE 0: dB[i][k] += sum_j dS[i][j] A[k][j];  ROLE 1: dA[k][j] += sum_i B[i][k] dS[i][j]
+#pragma unroll
+        for (int a = 0; a < kAccMax; ++a) {
+            if (a >= nacc4) break;
+            const int e = tid + kBwThreads * a;
+            float s = acc[a];
+            if (ROLE == 0) {
+                const int i = e / r4, k = e % r4;
+#pragma unroll 8
+                for (int j = 0; j < kT; ++j) s = fmaf(ds[i][j], bf16f(fs[k][j]), s);
+            } else {
+                const int k = e / kT, j = e % kT;
+#pragma unroll 8
+                for (int i = 0; i < kT; ++i) s = fmaf(bf16f(fs[k][i]), ds[i][j], s);
+            }
+            acc[a] = s;
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int a = 0; a < kAccMax; ++a) {
+        if (a >= nacc4) break;
+        const int e = tid + kBwThreads * a;
+        if (ROLE == 0) {
+            const int i = own0 + e / r4, k = e % r4;
+            if (i < p.m && k < p.r) p.dB[(size_t)i * p.r + k] = acc[a];
+        } else {
+            const int k = e / kT, j = own0 + e % kT;
+            if (k < p.r && j < p.n) p.dA[(size_t)k * p.n + j] = acc[a];
+        }
+    }
+}
+
+}  // namespace
+
+int launch_transpose_codes(const uint8_t *Q, int m, int n, int bits, uint8_t *Qt, cudaStream_t stream)
+{
+    const dim3 grid((unsigned)((n + 127) / 128), (unsigned)((m + 31) / 32));
+    if (grid.y > 65535u) return LORDS_ERR_SHAPE;
+    lords_transpose_codes_kernel<<<grid, 128, 0, stream>>>(Q, Qt, m, n, bits);
+    LORDS_CUDA_TRY(cudaGetLastError());
+    return LORDS_OK;
+}
+
+int launch_transpose_bf16(const uint16_t *src, int rows, int cols, uint16_t *dst, cudaStream_t stream)
+{
+    const dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((rows + 31) / 32));
+    if (grid.y > 65535u) return LORDS_ERR_SHAPE;
+    lords_transpose_bf16_kernel<<<grid, dim3(32, 8), 0, stream>>>(src, dst, rows, cols);
+    LORDS_CUDA_TRY(cudaGetLastError());
+    return LORDS_OK;
+}
+
+int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t *q, const uint16_t *B, const uint16_t *A,
+                            const float *levels, int bits, int M, int m, int n, int r, float *dB, float *dA,
+                            State &st, cudaStream_t stream)
+{
+    if (r > kRMaxBw) return LORDS_ERR_SHAPE;
+    BwParams p;
+    p.g = g; p.x = x; p.q = q; p.B = B; p.A = A;
+    for (int c = 0; c < 16; ++c) p.levels[c] = c < (1 << bits) ? levels[c] : 0.0f;
+    p.bits = bits; p.M = M; p.m = m; p.n = n; p.r = r;
+    p.dB = dB; p.dA = dA;
+    int launches = 0;
+    if (dB) {
+        lords_backward_factors_kernel<0><<<(unsigned)((m + kT - 1) / kT), kBwThreads, 0, stream>>>(p);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        ++launches;
+    }
+    if (dA) {
+        lords_backward_factors_kernel<1><<<(unsigned)((n + kT - 1) / kT), kBwThreads, 0, stream>>>(p);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        ++launches;
+    }
+    st.last_launches = launches;
+    st.last_path = "backward_factors";
+    return LORDS_OK;
+}
+
+}  // namespace lords

@@ -258,6 +258,7 @@ int lords_shutdown(void)
         cudaFree(st.status_word);
         if (st.stage_x) cudaFree(st.stage_x);
         if (st.stage_y) cudaFree(st.stage_y);
+        if (st.bw_scratch) cudaFree(st.bw_scratch);
     }
     int fp = st.forced_path, fs = st.forced_splitk, fb = st.forced_bn;
     st = State();
@@ -345,6 +346,78 @@ int lords_quantize_codes(const void *W, const void *B, const void *A, const floa
     if (!st.initialised) return LORDS_ERR_NOT_INIT;
     st.last_launches = 0;
     return launch_quantize(W, B, A, codebook, bits, m, n, r, Qpacked, st, static_cast<cudaStream_t>(stream));
+}
+
+int lords_transpose_codes(const uint8_t *Qpacked, int bits, int m, int n, uint8_t *Qt_packed, void *stream)
+{
+    if (!Qpacked || !Qt_packed) return LORDS_ERR_NULL;
+    const int g = pack_group(bits);
+    if (g == 0) return LORDS_ERR_BITS;
+    if (m < 1 || n < 1 || n % g != 0 || m % g != 0) return LORDS_ERR_SHAPE;
+    if (!aligned16(Qpacked) || !aligned16(Qt_packed)) return LORDS_ERR_ALIGN;
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    const int rc = launch_transpose_codes(Qpacked, m, n, bits, Qt_packed, static_cast<cudaStream_t>(stream));
+    if (rc != LORDS_OK) return rc;
+    st.last_launches = 1;
+    st.last_path = "transpose_codes";
+    return LORDS_OK;
+}
+
+// dx = g W^ is the forward of the transposed layer: W^T = L[Q^T] (.) (A^T B^T).
+static int backward_input_common(const void *dy, const uint8_t *Qt, const void *B, const void *A, const float *cb, int bits,
+                                 int M, int m, int n, int r, void *dx, int dx_f32, void *stream)
+{
+    if (!dy || !Qt || !B || !A || !cb || !dx) return LORDS_ERR_NULL;
+    if (m < 1 || n < 1 || r < 1 || r > LORDS_R_MAX) return LORDS_ERR_SHAPE;
+    if (!aligned16(B) || !aligned16(A)) return LORDS_ERR_ALIGN;
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    const size_t at_bytes = ((size_t)n * r * 2 + 255) & ~(size_t)255, bt_bytes = (size_t)r * m * 2;
+    if (at_bytes + bt_bytes > st.bw_scratch_bytes) {
+        if (st.bw_scratch) cudaFree(st.bw_scratch);
+        st.bw_scratch = nullptr; st.bw_scratch_bytes = 0;
+        LORDS_CUDA_TRY(cudaMalloc(&st.bw_scratch, at_bytes + bt_bytes));
+        st.bw_scratch_bytes = at_bytes + bt_bytes;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint16_t *At = reinterpret_cast<uint16_t *>(st.bw_scratch), *Bt = reinterpret_cast<uint16_t *>(st.bw_scratch + at_bytes);
+    int rc = launch_transpose_bf16(static_cast<const uint16_t *>(A), r, n, At, s);       // A [r][n] -> [n][r]
+    if (rc == LORDS_OK) rc = launch_transpose_bf16(static_cast<const uint16_t *>(B), m, r, Bt, s);   // B [m][r] -> [r][m]
+    if (rc != LORDS_OK) return rc;
+    // the transposed layer has n out-features and m in-features; its "B" is A^T and its "A" is B^T
+    rc = forward_common(dy, Qt, At, Bt, cb, bits, M, n, m, r, dx, dx_f32, stream);
+    if (rc != LORDS_OK) return rc;
+    st.last_launches += 2;
+    return LORDS_OK;
+}
+
+int lords_linear_backward_input(const void *dy, const uint8_t *Qt_packed, const void *B, const void *A, const float *codebook,
+                                int bits, int M, int m, int n, int r, void *dx, void *stream)
+{
+    return backward_input_common(dy, Qt_packed, B, A, codebook, bits, M, m, n, r, dx, 0, stream);
+}
+
+int lords_linear_backward_input_f32(const void *dy, const uint8_t *Qt_packed, const void *B, const void *A,
+                                    const float *codebook, int bits, int M, int m, int n, int r, float *dx32, void *stream)
+{
+    return backward_input_common(dy, Qt_packed, B, A, codebook, bits, M, m, n, r, dx32, 1, stream);
+}
+
+int lords_linear_backward_factors(const void *dy, const void *x, const uint8_t *Qpacked, const void *B, const void *A,
+                                  const float *codebook, int bits, int M, int m, int n, int r, float *dB, float *dA,
+                                  void *stream)
+{
+    if (!dy || !x || !Qpacked || !B || !A || !codebook || (!dB && !dA)) return LORDS_ERR_NULL;
+    const int g = pack_group(bits);
+    if (g == 0) return LORDS_ERR_BITS;
+    if (M < 1 || M > LORDS_M_MAX || m < 1 || n < 1 || n % g != 0) return LORDS_ERR_SHAPE;
+    if (r < 1 || r > LORDS_R_MAX) return LORDS_ERR_SHAPE;
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    return launch_backward_factors(static_cast<const uint16_t *>(dy), static_cast<const uint16_t *>(x), Qpacked,
+                                   static_cast<const uint16_t *>(B), static_cast<const uint16_t *>(A), codebook, bits, M, m,
+                                   n, r, dB, dA, st, static_cast<cudaStream_t>(stream));
 }
 
 int lords_poll_status(void *stream)

@@ -35,6 +35,8 @@ struct State {
     uint8_t *stage_x = nullptr;     // device staging for the host-buffer entry point
     uint8_t *stage_y = nullptr;
     size_t stage_x_bytes = 0, stage_y_bytes = 0;
+    uint8_t *bw_scratch = nullptr;  // transposed factors for the input gradient
+    size_t bw_scratch_bytes = 0;
     int forced_path = 0;            // 0 auto, 1 simt, 2 decode (reassociated form), 3 umma (scale-MMA form), 4 decode16
     int forced_splitk = 0;          // 0 auto
     int forced_bn = 0;              // 0 auto; else the token tile of the scale-MMA kernel (32, 64, 128, 256)
@@ -72,5 +74,13 @@ int launch_decode16(const Problem &p, State &st, cudaStream_t stream);
 // Quantisation step (codes from W, B, A): tensor-core kernel where its rules hold, CUDA cores otherwise.
 int launch_quantize(const void *W, const void *B, const void *A, const float *levels, int bits, int m, int n, int r,
                     uint8_t *Q, State &st, cudaStream_t stream);
+
+// Backward with the codes fixed (Sec. 3.4): transposition of packed codes and of a bf16 matrix (what the
+// input gradient needs to run on the forward kernels), and the gradients of B and A on the CUDA cores.
+int launch_transpose_codes(const uint8_t *Q, int m, int n, int bits, uint8_t *Qt, cudaStream_t stream);
+int launch_transpose_bf16(const uint16_t *src, int rows, int cols, uint16_t *dst, cudaStream_t stream);
+int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t *q, const uint16_t *B, const uint16_t *A,
+                            const float *levels, int bits, int M, int m, int n, int r, float *dB, float *dA,
+                            State &st, cudaStream_t stream);
 
 }  // namespace lords

@@ -1,0 +1,153 @@
+"""GPU backward with the codes fixed (Sec. 3.4) against the fp64 oracle, through the C ABI.
+
+dx runs on the forward kernels (the transposed layer), so it is held to the forward's criteria: the
+fp32 accumulator within the normwise and per-element tolerances, the bf16 output the RNE rounding of
+that accumulator and within one bf16 ulp of the rounded oracle value.  dB and dA are fp32 sums on the
+CUDA cores over exactly widened bf16 inputs: a sum of K products carries a relative rounding error of
+the order of sqrt(K) * 2^-24 (K up to a few million here: about 1e-4 of the norm at worst), so they are
+held to 1e-4 normwise and 1e-3 per element (relative to max(|value|, rms)); integer inputs are exact.
+The transposition of the packed codes is integer work: bit-exact."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2601_22716_b200 import inputs as gen
+from _util import check_against_oracle, error_metrics
+
+pytestmark = pytest.mark.gpu
+
+FACTOR_NORMWISE_TOL = 1e-4
+FACTOR_ELEMENT_TOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def lords():
+    import torch
+    from paper_2601_22716_b200 import binding
+    assert torch.cuda.is_available()
+    binding.lords_init(0, 0)
+    yield binding
+    binding.lords_set_option("path", "auto")
+    binding.lords_shutdown()
+
+
+def _dev(a16):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a16).view(np.int16)).to("cuda:0")
+
+
+def _grad_out(M, m, seed, integer=False):
+    """g = dL/dy as bf16 bit patterns: N(0, 1), or small integers for the exact cases."""
+    import torch
+    g = torch.Generator().manual_seed(1000 + seed)
+    if integer:
+        v = torch.randint(-2, 3, (M, m), generator=g).float()
+    else:
+        v = torch.randn(M, m, generator=g)
+    return gen.bf16_bits(v)
+
+
+@pytest.mark.parametrize("bits,m,n", [(4, 64, 96), (4, 38, 70), (3, 96, 64), (3, 160, 352), (2, 44, 132), (2, 256, 64),
+                                      (4, 1000, 2048)])
+def test_transposed_codes_are_bit_exact(lords, bits, m, n):
+    import torch
+    rng = np.random.default_rng(m * n + bits)
+    codes = rng.integers(0, 1 << bits, size=(m, n), dtype=np.uint8)
+    q = torch.from_numpy(oracle.pack_codes(codes, bits)).to("cuda:0")
+    qt = torch.full((lords.lords_packed_bytes(n, m, bits),), 0xA5, dtype=torch.uint8, device="cuda:0")
+    lords.lords_transpose_codes(q, bits, m, n, qt)
+    torch.cuda.synchronize()
+    want = oracle.pack_codes(np.ascontiguousarray(codes.T), bits)
+    assert np.array_equal(qt.cpu().numpy().reshape(want.shape), want)
+
+
+BACKWARD_SHAPES = [
+    # bits, m, n, r, M, mixed, path the input gradient is expected to take
+    (4, 512, 384, 32, 1, True, "decode"),        # the transposed layer has 512 in-features
+    (4, 1024, 300, 12, 2, True, "decode"),       # ragged out-features of the transposed layer
+    (3, 256, 544, 48, 8, True, "decode16"),
+    (2, 320, 256, 6, 5, False, "decode16"),
+    (4, 384, 256, 32, 200, True, "umma"),
+    (3, 512, 160, 16, 40, False, "umma"),
+    (4, 38, 66, 5, 3, True, "simt"),             # nothing a multiple of a tile
+    (3, 96, 64, 100, 4, False, "simt"),          # a rank the tensor-core paths decline
+]
+
+
+@pytest.mark.parametrize("bits,m,n,r,M,mixed,path", BACKWARD_SHAPES)
+def test_backward_against_the_oracle(lords, bits, m, n, r, M, mixed, path):
+    import torch
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=7 * m + n + r + M, mixed_sign=mixed)
+    g = _grad_out(M, m, m + n)
+    packed = oracle.pack_codes(lay.codes, bits)
+    dx64, dB64, dA64 = oracle.backward(g, lay.x, packed, lay.B, lay.A, lay.codebook, bits)
+
+    q = torch.from_numpy(packed).to("cuda:0")
+    qt = torch.empty(lords.lords_packed_bytes(n, m, bits), dtype=torch.uint8, device="cuda:0")
+    lords.lords_transpose_codes(q, bits, m, n, qt)
+    gd, xd, Bd, Ad = _dev(g), _dev(lay.x), _dev(lay.B), _dev(lay.A)
+    dx32 = torch.zeros((M, n), dtype=torch.float32, device="cuda:0")
+    dxbf = torch.zeros((M, n), dtype=torch.int16, device="cuda:0")
+    lords.lords_linear_backward_input_f32(gd, qt, Bd, Ad, lay.codebook, bits, M, m, n, r, dx32)
+    lords.lords_linear_backward_input(gd, qt, Bd, Ad, lay.codebook, bits, M, m, n, r, dxbf)
+    assert lords.lords_last_path() == path
+    dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
+    dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
+    lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, bits, M, m, n, r, dB, dA)
+    assert lords.lords_last_path() == "backward_factors" and lords.lords_last_launch_count() == 2
+    torch.cuda.synchronize()
+    assert lords.lords_poll_status() == 0
+
+    check_against_oracle(dx32.cpu().numpy(), dxbf.cpu().numpy().view(np.uint16), dx64)
+    for name, got, want in (("dB", dB.cpu().numpy(), dB64), ("dA", dA.cpu().numpy(), dA64)):
+        assert np.isfinite(got).all(), name
+        nw, el = error_metrics(got, want)
+        assert nw <= FACTOR_NORMWISE_TOL and el <= FACTOR_ELEMENT_TOL, (name, nw, el)
+
+
+@pytest.mark.parametrize("bits,m,n,r,M", [(4, 256, 384, 8, 3), (3, 160, 128, 5, 20), (2, 128, 320, 40, 2)])
+def test_backward_integer_case_is_bit_exact(lords, bits, m, n, r, M):
+    """Small integers everywhere: every product and partial sum is an exact integer below 2^24."""
+    import torch
+    lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m)
+    g = _grad_out(M, m, m, integer=True)
+    packed = oracle.pack_codes(lay.codes, bits)
+    dx64, dB64, dA64 = oracle.backward(g, lay.x, packed, lay.B, lay.A, lay.codebook, bits)
+    q = torch.from_numpy(packed).to("cuda:0")
+    qt = torch.empty(lords.lords_packed_bytes(n, m, bits), dtype=torch.uint8, device="cuda:0")
+    lords.lords_transpose_codes(q, bits, m, n, qt)
+    gd, xd, Bd, Ad = _dev(g), _dev(lay.x), _dev(lay.B), _dev(lay.A)
+    dx32 = torch.zeros((M, n), dtype=torch.float32, device="cuda:0")
+    dB = torch.zeros((m, r), dtype=torch.float32, device="cuda:0")
+    dA = torch.zeros((r, n), dtype=torch.float32, device="cuda:0")
+    lords.lords_linear_backward_input_f32(gd, qt, Bd, Ad, lay.codebook, bits, M, m, n, r, dx32)
+    lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, bits, M, m, n, r, dB, dA)
+    torch.cuda.synchronize()
+    assert lords.lords_poll_status() == 0
+    assert np.array_equal(dx32.cpu().numpy().astype(np.float64), dx64)
+    assert np.array_equal(dB.cpu().numpy().astype(np.float64), dB64)
+    assert np.array_equal(dA.cpu().numpy().astype(np.float64), dA64)
+
+
+def test_backward_factors_one_at_a_time_and_bad_arguments(lords):
+    import torch
+    lay = gen.make_layer(128, 128, 8, 2, bits=4, seed=1)
+    g = _grad_out(2, 128, 3)
+    packed = oracle.pack_codes(lay.codes, 4)
+    _, dB64, dA64 = oracle.backward(g, lay.x, packed, lay.B, lay.A, lay.codebook, 4)
+    q = torch.from_numpy(packed).to("cuda:0")
+    gd, xd, Bd, Ad = _dev(g), _dev(lay.x), _dev(lay.B), _dev(lay.A)
+    dB = torch.zeros((128, 8), dtype=torch.float32, device="cuda:0")
+    dA = torch.zeros((8, 128), dtype=torch.float32, device="cuda:0")
+    lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, 4, 2, 128, 128, 8, dB, None)
+    assert lords.lords_last_launch_count() == 1
+    lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, 4, 2, 128, 128, 8, None, dA)
+    torch.cuda.synchronize()
+    assert error_metrics(dB.cpu().numpy(), dB64)[0] <= FACTOR_NORMWISE_TOL
+    assert error_metrics(dA.cpu().numpy(), dA64)[0] <= FACTOR_NORMWISE_TOL
+    with pytest.raises(lords.LordsError) as ei:
+        lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, 4, 2, 128, 128, 8, None, None)
+    assert ei.value.status == -1
+    with pytest.raises(lords.LordsError) as ei:        # m = 127 is not a multiple of the 4-bit pack group
+        lords.lords_transpose_codes(q, 4, 127, 128, torch.empty(128 * 64, dtype=torch.uint8, device="cuda:0"))
+    assert ei.value.status == -2
