@@ -48,6 +48,8 @@ CASES = {
 }
 # the step before the path (Alg. 1, step 2.1) on the same shapes: name -> (m, n, r, bits)
 QUANTIZE_CASES = {"quantize_q_nf4": (4096, 4096, 32, 4), "quantize_gate_nf3": (14336, 4096, 48, 3)}
+# the backward with the codes fixed (Sec. 3.4): name -> (m, n, r, bits, M)
+BACKWARD_CASES = {"backward_q_m512": (4096, 4096, 32, 4, 512)}
 HEADLINE = "decode_q_m1"
 METRIC = "LoRDS dequant-GEMM: HBM GB/s at M=1, TFLOP/s at M=2048, % of roofline"
 
@@ -502,6 +504,69 @@ def time_quantize(name, m, n, r, bits, device, min_seconds=0.3):
                          "algorithmic_bytes_per_launch": byt, "us_per_launch": us}}
 
 
+# fp32 FMA throughput of the CUDA cores: 148 SMs x 128 lanes x 2 flops at the 1965 MHz boost clock
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def time_backward(name, m, n, r, bits, M, device, min_seconds=0.3):
+    """The backward with the codes fixed (Sec. 3.4) on one layer shape: dx = g W^ on the forward
+    kernels (transposed codes, made once outside the timed region; the per-call transposition of the
+    factors inside it), then dB and dA on the CUDA cores.  Reported separately."""
+    import numpy as np
+    import torch
+    from paper_2601_22716_b200 import binding as lords
+    from paper_2601_22716_b200 import inputs as gen
+
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=0)
+    q = torch.from_numpy(lords.lords_pack_codes(lay.codes, bits)).to(device)
+    qt = torch.empty(lords.lords_packed_bytes(n, m, bits), dtype=torch.uint8, device=device)
+    lords.lords_transpose_codes(q, bits, m, n, qt)
+    B = torch.from_numpy(lay.B.view(np.int16)).to(device)
+    A = torch.from_numpy(lay.A.view(np.int16)).to(device)
+    x = torch.from_numpy(lay.x.view(np.int16)).to(device)
+    g = torch.from_numpy(gen.make_layer(m, m, 1, M, bits=4, seed=1).x[:, :m].copy().view(np.int16)).to(device)
+    dx = torch.zeros((M, n), dtype=torch.int16, device=device)
+    dB = torch.zeros((m, r), dtype=torch.float32, device=device)
+    dA = torch.zeros((r, n), dtype=torch.float32, device=device)
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        path = lords.lords_last_path()
+        total, reps = 0.0, 0
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        while total < min_seconds * 1e3 / 2 and reps < 200:
+            flush.zero_()                      # L2 flush between timed calls (a write larger than L2)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            total += e0.elapsed_time(e1)
+            reps += 1
+        return total / reps * 1e3, path, reps
+
+    us_dx, path_dx, reps_dx = timed(lambda: lords.lords_linear_backward_input(g, qt, B, A, lay.codebook, bits, M, m, n, r, dx))
+    us_f, path_f, reps_f = timed(lambda: lords.lords_linear_backward_factors(g, x, q, B, A, lay.codebook, bits, M, m, n, r, dB, dA))
+    status = lords.lords_poll_status()
+    peaks = measured_peaks()
+    flops = 2.0 * M * m * n
+    tf_dx = flops / (us_dx * 1e-6) / 1e12
+    tf_f = (flops + 4.0 * m * n * r) / (us_f * 1e-6) / 1e12      # g^T x formed once (one CTA per tile of W), plus the two folds
+    return {"case": name, "path": f"{path_dx}+{path_f}", "us_per_call": us_dx + us_f, "gbs": None, "tflops": None,
+            "copies": 1, "rounds": reps_dx, "steps": 1, "status_retries": 0 if status == 0 else 1,
+            "input_gradient": {"us": us_dx, "path": path_dx, "tflops": tf_dx,
+                               "roofline": {"bound": "tensor", "achieved": tf_dx, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                            "frac": tf_dx / peaks["bf16_tflops"], "peak_kind": "burst", "traffic": None}},
+            "factor_gradients": {"us": us_f, "path": path_f, "tflops": tf_f},
+            "roofline": {"bound": "alu", "achieved": tf_f, "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s",
+                         "frac": tf_f / FP32_ALU_TFLOPS, "peak_source": "148 SMs x 128 fp32 lanes x 2 flops x 1.965 GHz",
+                         "traffic": None, "us_per_launch": us_f}}
+
+
 def run_sweep(device):
     """The measurement behind the per-M choice of kernel: every tensor-core path that accepts the
     shape, at M in {1, 2, 3, 4, 8, 16}, on the q_proj (NF4, r = 32), gate and down (NF3, r = 48) shapes.
@@ -660,6 +725,13 @@ def main():
             dist.destroy_process_group()
         return 0
 
+    if args.case in BACKWARD_CASES:
+        if rank == 0:
+            print(json.dumps(time_backward(args.case, *BACKWARD_CASES[args.case], device, min_seconds=min(args.min_seconds, 0.3))))
+        lords.lords_shutdown()
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
     if args.case in QUANTIZE_CASES:
         if rank == 0:
             print(json.dumps(time_quantize(args.case, *QUANTIZE_CASES[args.case], device, min_seconds=min(args.min_seconds, 0.3))))
@@ -691,6 +763,8 @@ def main():
     if not args.case and not args.no_extras and world == 1:
         for name, shape in QUANTIZE_CASES.items():
             cases.append(time_quantize(name, *shape, device))
+        for name, shape in BACKWARD_CASES.items():
+            cases.append(time_backward(name, *shape, device))
 
     stack = []
     if not args.no_stack and not args.no_extras and not args.case and world == 1:

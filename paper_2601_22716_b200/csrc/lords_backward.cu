@@ -11,14 +11,18 @@
 // forward kernels as they are.  This file holds what that needs -- the transposition of packed codes
 // and of a bf16 matrix -- and the kernels for dB and dA.
 //
-// dB and dA run on the CUDA cores in fp32 (bf16 inputs are widened exactly).  One kernel, two roles:
-//   role 0 (dB): a CTA owns 64 rows of W and walks over the columns in steps of 64;
-//   role 1 (dA): a CTA owns 64 columns and walks over the rows in steps of 64.
-// Per step it forms the 64 x 64 tile of g^T x by a shared-memory-tiled product over the tokens,
-// multiplies by the levels of the tile's codes, and folds the tile into its accumulators with the
-// matching 64-column (or 64-row) slice of A (or B).  Every output element is summed by one thread in
-// a fixed order: no atomics, runs are bit-identical.  Bound: fp32 ALU, 2 m n M fused multiply-adds
-// for the two roles together (the tile of g^T x is formed once per role).
+// dB and dA run on the CUDA cores in fp32 (bf16 inputs are widened exactly).  A 64 x 64 tile of dS is
+// formed by a shared-memory-tiled product g^T x over the tokens, multiplied by the levels of the
+// tile's codes, and folded with the matching 64-column slice of A (for dB) and 64-row slice of B (for
+// dA).  Two schedules:
+//   tiles: one CTA per tile of W; it writes the tile's contributions to dB and dA into the library's
+//          workspace, and a second kernel adds the contributions of a row (or column) of tiles in tile
+//          order.  g^T x is formed once, and the grid fills the machine.  Taken when the workspace
+//          holds the contributions (4 r (m n / 64 + n m / 64) bytes).
+//   walk:  one CTA per 64 rows (dB) or 64 columns (dA) walks over the other dimension and keeps its
+//          sums in registers.  No scratch memory, g^T x formed once per gradient.
+// Either way every output element is summed in a fixed order without atomics: runs are bit-identical.
+// Bound: fp32 ALU, m n M fused multiply-adds for the tile product (twice with the second schedule).
 #include <cuda_runtime.h>
 
 #include "lords_internal.h"
@@ -207,6 +211,103 @@ __global__ void __launch_bounds__(kBwThreads) lords_backward_factors_kernel(cons
     }
 }
 
+// Schedule "tiles": CTA (jt, it) handles rows it * 64 .. and columns jt * 64 .. of W.
+//   part_dB[jt][i][k4]  (k4 < r4: r rounded up to a multiple of 4) and part_dA[it][k4][j]
+__global__ void __launch_bounds__(kBwThreads) lords_backward_tile_kernel(const BwParams p, float *__restrict__ part_dB,
+                                                                         float *__restrict__ part_dA)
+{
+    __shared__ __align__(16) float gs[kTok][kT];
+    __shared__ __align__(16) float xs[kTok][kT];
+    __shared__ float ds[kT][kT + 1];
+    __shared__ uint16_t fs[kRMaxBw][kT + 2];
+
+    const int tid = threadIdx.x;
+    const int ty = tid >> 4, tx = tid & 15;
+    const int jt = blockIdx.x, it = blockIdx.y;
+    const int i0 = it * kT, j0 = jt * kT;
+    const size_t row_bytes = (size_t)p.n * p.bits / 8;
+    const int r4 = (p.r + 3) & ~3;
+    const int nacc4 = r4 * kT / kBwThreads;
+
+    float c[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) c[a][b] = 0.0f;
+    for (int t0 = 0; t0 < p.M; t0 += kTok) {
+        for (int e = tid; e < kTok * kT; e += kBwThreads) {
+            const int t = t0 + e / kT, cidx = e % kT;
+            gs[e / kT][cidx] = (t < p.M && i0 + cidx < p.m) ? bf16f(p.g[(size_t)t * p.m + i0 + cidx]) : 0.0f;
+            xs[e / kT][cidx] = (t < p.M && j0 + cidx < p.n) ? bf16f(p.x[(size_t)t * p.n + j0 + cidx]) : 0.0f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int t = 0; t < kTok; ++t) {
+            const float4 g4 = *reinterpret_cast<const float4 *>(&gs[t][ty * 4]);
+            const float4 x4 = *reinterpret_cast<const float4 *>(&xs[t][tx * 4]);
+            const float gv[4] = {g4.x, g4.y, g4.z, g4.w}, xv[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) c[a][b] = fmaf(gv[a], xv[b], c[a][b]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int i = i0 + ty * 4 + a, j = j0 + tx * 4 + b;
+            float lv = 0.0f;
+            if (i < p.m && j < p.n) lv = p.levels[read_code(p.q, row_bytes, i, j, p.bits)];
+            ds[ty * 4 + a][tx * 4 + b] = c[a][b] * lv;
+        }
+    if (part_dB) {
+        for (int e = tid; e < r4 * kT; e += kBwThreads) {           // A[k][j0 ..], zero padded
+            const int k = e / kT, cidx = e % kT;
+            fs[k][cidx] = (k < p.r && j0 + cidx < p.n) ? p.A[(size_t)k * p.n + j0 + cidx] : (uint16_t)0;
+        }
+        __syncthreads();
+        float *out = part_dB + ((size_t)jt * p.m + i0) * r4;
+        for (int a = 0; a < nacc4; ++a) {
+            const int e = tid + kBwThreads * a, i = e / r4, k = e % r4;
+            float s = 0.0f;
+#pragma unroll 8
+            for (int j = 0; j < kT; ++j) s = fmaf(ds[i][j], bf16f(fs[k][j]), s);
+            if (i0 + i < p.m) out[(size_t)i * r4 + k] = s;
+        }
+    }
+    __syncthreads();
+    if (part_dA) {
+        for (int e = tid; e < r4 * kT; e += kBwThreads) {           // B[i0 ..][k] stored [k][i], zero padded
+            const int k = e / kT, cidx = e % kT;
+            fs[k][cidx] = (k < p.r && i0 + cidx < p.m) ? p.B[(size_t)(i0 + cidx) * p.r + k] : (uint16_t)0;
+        }
+        __syncthreads();
+        float *out = part_dA + (size_t)it * r4 * p.n + j0;
+        for (int a = 0; a < nacc4; ++a) {
+            const int e = tid + kBwThreads * a, k = e / kT, j = e % kT;
+            float s = 0.0f;
+#pragma unroll 8
+            for (int i = 0; i < kT; ++i) s = fmaf(bf16f(fs[k][i]), ds[i][j], s);
+            if (j0 + j < p.n) out[(size_t)k * p.n + j] = s;
+        }
+    }
+}
+
+// out[e] = sum over tiles t (in order) of part[t * stride + pos(e)]: dB (rows = m, inner = r, inner4 = r4)
+// or dA (rows = r, inner = inner4 = n).
+__global__ void lords_backward_reduce_kernel(const float *__restrict__ part, float *__restrict__ out, int tiles, size_t stride,
+                                             int rows, int inner, int inner4)
+{
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= (size_t)rows * inner) return;
+    const size_t row = e / inner, col = e % inner;
+    float s = 0.0f;
+    for (int t = 0; t < tiles; ++t) s += part[(size_t)t * stride + row * inner4 + col];
+    out[e] = s;
+}
+
 }  // namespace
 
 int launch_transpose_codes(const uint8_t *Q, int m, int n, int bits, uint8_t *Qt, cudaStream_t stream)
@@ -238,6 +339,31 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
     p.bits = bits; p.M = M; p.m = m; p.n = n; p.r = r;
     p.dB = dB; p.dA = dA;
     int launches = 0;
+    // schedule "tiles" when the workspace holds the tiles' contributions
+    const int r4 = (r + 3) & ~3, it_n = (m + kT - 1) / kT, jt_n = (n + kT - 1) / kT;
+    const size_t need_b = dB ? (size_t)jt_n * m * r4 * sizeof(float) : 0, need_a = dA ? (size_t)it_n * r4 * n * sizeof(float) : 0;
+    if (it_n <= 65535 && need_b + need_a + 256 <= st.workspace_bytes && st.forced_path != 1) {
+        float *part_b = dB ? reinterpret_cast<float *>(st.workspace) : nullptr;
+        float *part_a = dA ? reinterpret_cast<float *>(st.workspace + ((need_b + 255) & ~(size_t)255)) : nullptr;
+        lords_backward_tile_kernel<<<dim3((unsigned)jt_n, (unsigned)it_n), kBwThreads, 0, stream>>>(p, part_b, part_a);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        ++launches;
+        if (dB) {
+            const size_t total = (size_t)m * r;
+            lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(part_b, dB, jt_n, (size_t)m * r4, m, r, r4);
+            LORDS_CUDA_TRY(cudaGetLastError());
+            ++launches;
+        }
+        if (dA) {
+            const size_t total = (size_t)r * n;
+            lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(part_a, dA, it_n, (size_t)r4 * n, r, n, n);
+            LORDS_CUDA_TRY(cudaGetLastError());
+            ++launches;
+        }
+        st.last_launches = launches;
+        st.last_path = "backward_tiles";
+        return LORDS_OK;
+    }
     if (dB) {
         lords_backward_factors_kernel<0><<<(unsigned)((m + kT - 1) / kT), kBwThreads, 0, stream>>>(p);
         LORDS_CUDA_TRY(cudaGetLastError());
@@ -249,7 +375,7 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
         ++launches;
     }
     st.last_launches = launches;
-    st.last_path = "backward_factors";
+    st.last_path = "backward_walk";
     return LORDS_OK;
 }
 

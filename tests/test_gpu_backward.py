@@ -91,18 +91,24 @@ def test_backward_against_the_oracle(lords, bits, m, n, r, M, mixed, path):
     lords.lords_linear_backward_input_f32(gd, qt, Bd, Ad, lay.codebook, bits, M, m, n, r, dx32)
     lords.lords_linear_backward_input(gd, qt, Bd, Ad, lay.codebook, bits, M, m, n, r, dxbf)
     assert lords.lords_last_path() == path
-    dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
-    dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
-    lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, bits, M, m, n, r, dB, dA)
-    assert lords.lords_last_path() == "backward_factors" and lords.lords_last_launch_count() == 2
-    torch.cuda.synchronize()
-    assert lords.lords_poll_status() == 0
-
     check_against_oracle(dx32.cpu().numpy(), dxbf.cpu().numpy().view(np.uint16), dx64)
-    for name, got, want in (("dB", dB.cpu().numpy(), dB64), ("dA", dA.cpu().numpy(), dA64)):
-        assert np.isfinite(got).all(), name
-        nw, el = error_metrics(got, want)
-        assert nw <= FACTOR_NORMWISE_TOL and el <= FACTOR_ELEMENT_TOL, (name, nw, el)
+    # both schedules of the factor gradients: one CTA per tile of W with the contributions summed by a
+    # second kernel (taken when the workspace holds them), and the walk that needs no scratch memory
+    for option, schedule, launches in (("auto", "backward_tiles", 3), ("simt", "backward_walk", 2)):
+        dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
+        dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
+        lords.lords_set_option("path", option)
+        try:
+            lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, bits, M, m, n, r, dB, dA)
+        finally:
+            lords.lords_set_option("path", "auto")
+        assert lords.lords_last_path() == schedule and lords.lords_last_launch_count() == launches
+        torch.cuda.synchronize()
+        assert lords.lords_poll_status() == 0
+        for name, got, want in (("dB", dB.cpu().numpy(), dB64), ("dA", dA.cpu().numpy(), dA64)):
+            assert np.isfinite(got).all(), (schedule, name)
+            nw, el = error_metrics(got, want)
+            assert nw <= FACTOR_NORMWISE_TOL and el <= FACTOR_ELEMENT_TOL, (schedule, name, nw, el)
 
 
 @pytest.mark.parametrize("bits,m,n,r,M", [(4, 256, 384, 8, 3), (3, 160, 128, 5, 20), (2, 128, 320, 40, 2)])
@@ -121,12 +127,19 @@ def test_backward_integer_case_is_bit_exact(lords, bits, m, n, r, M):
     dB = torch.zeros((m, r), dtype=torch.float32, device="cuda:0")
     dA = torch.zeros((r, n), dtype=torch.float32, device="cuda:0")
     lords.lords_linear_backward_input_f32(gd, qt, Bd, Ad, lay.codebook, bits, M, m, n, r, dx32)
-    lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, bits, M, m, n, r, dB, dA)
     torch.cuda.synchronize()
-    assert lords.lords_poll_status() == 0
     assert np.array_equal(dx32.cpu().numpy().astype(np.float64), dx64)
-    assert np.array_equal(dB.cpu().numpy().astype(np.float64), dB64)
-    assert np.array_equal(dA.cpu().numpy().astype(np.float64), dA64)
+    for option in ("auto", "simt"):
+        dB.fill_(float("nan")); dA.fill_(float("nan"))
+        lords.lords_set_option("path", option)
+        try:
+            lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, bits, M, m, n, r, dB, dA)
+        finally:
+            lords.lords_set_option("path", "auto")
+        torch.cuda.synchronize()
+        assert lords.lords_poll_status() == 0
+        assert np.array_equal(dB.cpu().numpy().astype(np.float64), dB64), option
+        assert np.array_equal(dA.cpu().numpy().astype(np.float64), dA64), option
 
 
 def test_backward_factors_one_at_a_time_and_bad_arguments(lords):
@@ -140,7 +153,7 @@ def test_backward_factors_one_at_a_time_and_bad_arguments(lords):
     dB = torch.zeros((128, 8), dtype=torch.float32, device="cuda:0")
     dA = torch.zeros((8, 128), dtype=torch.float32, device="cuda:0")
     lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, 4, 2, 128, 128, 8, dB, None)
-    assert lords.lords_last_launch_count() == 1
+    assert lords.lords_last_launch_count() == 2        # the tile kernel and one sum
     lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, 4, 2, 128, 128, 8, None, dA)
     torch.cuda.synchronize()
     assert error_metrics(dB.cpu().numpy(), dB64)[0] <= FACTOR_NORMWISE_TOL
