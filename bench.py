@@ -82,8 +82,9 @@ NCU_TRAFFIC_BYTES = {
     "mlp3_down_m1": 23938560,       # same
     "mlp3_down_m16": 24299520,      # profiles/decode16_kernel_decode_q_m8_down_m16.md
     "prefill_m2048": 144602368,     # profiles/umma_kernel_prefill_m2048.md (the scale-MMA kernel; the pre-pass moves 73.7 MB more)
-    "quantize_q_nf4": 34142720,     # profiles/quantize_kernel_q_nf4_gate_nf3.md (8.4 MB of codes were still in L2 at the end)
-    "quantize_gate_nf3": 130091264,
+    "quantize_q_nf4": 34117888,     # profiles/quantize_kernel_q_nf4_gate_nf3.md (8.4 MB of codes were still in L2 at the end)
+    "quantize_gate_nf3": 131614720,
+    "backward_q_m512": 29558272,    # profiles/backward_tile_kernel_backward_q_m512.md (the factor-gradient kernel)
 }
 
 
@@ -539,7 +540,7 @@ def time_backward(name, m, n, r, bits, M, device, min_seconds=0.3):
         for _ in range(3):
             fn()
         torch.cuda.synchronize()
-        while total < min_seconds * 1e3 / 2 and reps < 200:
+        while reps < 1 or (total < min_seconds * 1e3 / 2 and reps < 200):
             flush.zero_()                      # L2 flush between timed calls (a write larger than L2)
             e0.record()
             fn()
@@ -564,7 +565,7 @@ def time_backward(name, m, n, r, bits, M, device, min_seconds=0.3):
             "factor_gradients": {"us": us_f, "path": path_f, "tflops": tf_f},
             "roofline": {"bound": "alu", "achieved": tf_f, "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s",
                          "frac": tf_f / FP32_ALU_TFLOPS, "peak_source": "148 SMs x 128 fp32 lanes x 2 flops x 1.965 GHz",
-                         "traffic": None, "us_per_launch": us_f}}
+                         "traffic": NCU_TRAFFIC_BYTES.get(name), "us_per_launch": us_f}}
 
 
 def run_sweep(device):
