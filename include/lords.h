@@ -210,6 +210,28 @@ int lords_linear_backward_factors(const void *dy, const void *x, const uint8_t *
                                   void *stream);
 
 /*
+ * Comparators for the paper's efficiency claims (Sec. 4.4, Table 6), on the same GPU and the same packed
+ * codes: a block-scaled layer (Eq. 2), and that layer with an additive low-rank adapter that cannot be
+ * merged into the quantised weights (Sec. 3.4).
+ *     lords_blockscale_forward:  y = x (L[Q] (.) (s (x) 1))^T,  scales: device, bf16 [m][ceil(n / blk)],
+ *         one scale per row and block of `blk` consecutive in-feature columns (blk a multiple of 64).
+ *     lords_adapter_forward:     y = x W_block^T + (x A_l^T) B_l^T,  A_l: device, bf16 [r][n];
+ *         B_l: device, bf16 [m][r]; three launches (the block-scaled product into the library's
+ *         workspace in fp32, u = x A_l^T, y = product + u B_l^T).
+ * M <= 16 (they are decode comparators); n a multiple of 64 (2- and 4-bit codes) or 128 (3-bit); other
+ * shapes return LORDS_ERR_UNSUPPORTED.  y: device, bf16 [M][m] (float for the _f32 variants).  Operand
+ * ranges, status word and error behaviour as for the forward calls.
+ */
+int lords_blockscale_forward(const void *x, const uint8_t *Qpacked, const void *scales, const float *codebook, int bits,
+                             int blk, int M, int m, int n, void *y, void *stream);
+int lords_blockscale_forward_f32(const void *x, const uint8_t *Qpacked, const void *scales, const float *codebook, int bits,
+                                 int blk, int M, int m, int n, float *y32, void *stream);
+int lords_adapter_forward(const void *x, const uint8_t *Qpacked, const void *scales, const void *A_l, const void *B_l,
+                          const float *codebook, int bits, int blk, int M, int m, int n, int r, void *y, void *stream);
+int lords_adapter_forward_f32(const void *x, const uint8_t *Qpacked, const void *scales, const void *A_l, const void *B_l,
+                              const float *codebook, int bits, int blk, int M, int m, int n, int r, float *y32, void *stream);
+
+/*
  * Allocation-free forward (the paper has no counterpart: this is a deployment convenience).
  * For callers that must not allocate device memory -- for instance a plugin inside a server
  * whose memory pool already owns all of HBM, or a latency-critical loop that cannot take the

@@ -185,3 +185,26 @@ def backward(g, x, qpacked, B, A, codebook, bits: int):
     if rc != 0:
         raise ValueError(f"oracle backward failed: {rc}")
     return dx, dB, dA
+
+
+def adapter_forward(x, qpacked, s, blk: int, A_l, B_l, codebook, bits: int) -> np.ndarray:
+    """The comparator of Sec. 4.4 / Table 6 in fp64: a block-scaled layer (Eq. 2, one scale s[i, j // blk]
+    per row and block) plus an additive low-rank adapter that stays separate (Sec. 3.4),
+
+        y = x W_block^T + (x A_l^T) B_l^T,      W_block = L[Q] (.) (s (x) 1).
+
+    The block-scaled term is the forward above with B = s and A = the 0/1 block indicator (the
+    special case that the block-wise pin checks against an independent Eq. 2 dequantiser); the adapter
+    term is two library matmuls.  All inputs are bf16 bit patterns except the codes and the level table."""
+    s = _c(s, np.uint16); x = _c(x, np.uint16); A_l = _c(A_l, np.uint16); B_l = _c(B_l, np.uint16)
+    m, nblk = s.shape
+    M, n = x.shape
+    assert nblk * blk >= n and (nblk - 1) * blk < n and A_l.shape[1] == n and B_l.shape == (m, A_l.shape[0])
+    ind = np.zeros((nblk, n), dtype=np.uint16)
+    for b in range(nblk):
+        ind[b, b * blk:(b + 1) * blk] = 0x3F80                      # bf16 1.0
+    y = forward(x, qpacked, s, ind, codebook, bits)
+
+    def f64(bits16):
+        return (bits16.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return y + (f64(x) @ f64(A_l).T) @ f64(B_l).T

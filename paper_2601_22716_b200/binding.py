@@ -53,6 +53,10 @@ def _load():
         "lords_linear_backward_input": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_backward_input_f32": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_backward_factors": (ci, [p, p, p, p, p, p, ci, ci, ci, ci, ci, p, p, p]),
+        "lords_blockscale_forward": (ci, [p, p, p, p, ci, ci, ci, ci, ci, p, p]),
+        "lords_blockscale_forward_f32": (ci, [p, p, p, p, ci, ci, ci, ci, ci, p, p]),
+        "lords_adapter_forward": (ci, [p, p, p, p, p, p, ci, ci, ci, ci, ci, ci, p, p]),
+        "lords_adapter_forward_f32": (ci, [p, p, p, p, p, p, ci, ci, ci, ci, ci, ci, p, p]),
         "lords_poll_status": (ci, [p]),
         "lords_read_status_detail": (ci, [p]),
         "lords_last_cuda_error": (ci, []),
@@ -78,7 +82,8 @@ def exported_symbols():
             "lords_pack_codes", "lords_unpack_codes", "lords_init", "lords_shutdown",
             "lords_linear_forward", "lords_linear_forward_bits", "lords_linear_forward_f32",
             "lords_linear_forward_host", "lords_linear_forward_noalloc", "lords_quantize_codes", "lords_transpose_codes",
-            "lords_linear_backward_input", "lords_linear_backward_input_f32", "lords_linear_backward_factors", "lords_poll_status", "lords_read_status_detail", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
+            "lords_linear_backward_input", "lords_linear_backward_input_f32", "lords_linear_backward_factors",
+            "lords_blockscale_forward", "lords_blockscale_forward_f32", "lords_adapter_forward", "lords_adapter_forward_f32", "lords_poll_status", "lords_read_status_detail", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
             "lords_last_launch_count"]
 
 
@@ -226,6 +231,22 @@ def lords_linear_backward_factors(dy, x, Qpacked, B, A, codebook, bits, M, m, n,
                                                  cb.ctypes.data, bits, M, m, n, r,
                                                  None if dB is None else dB.data_ptr(), None if dA is None else dA.data_ptr(),
                                                  _stream_ptr(stream)), "lords_linear_backward_factors")
+
+
+def lords_blockscale_forward(x, Qpacked, scales, codebook, bits, blk, M, m, n, y, stream=None, f32=False) -> None:
+    """Comparator (Eq. 2): y = x (L[Q] (.) (s (x) 1))^T; y is bf16 [M, m], or float with f32=True."""
+    cb = _cb_ptr(codebook, bits)
+    fn = _load().lords_blockscale_forward_f32 if f32 else _load().lords_blockscale_forward
+    _check(fn(x.data_ptr(), Qpacked.data_ptr(), scales.data_ptr(), cb.ctypes.data, bits, blk, M, m, n, y.data_ptr(),
+              _stream_ptr(stream)), "lords_blockscale_forward")
+
+
+def lords_adapter_forward(x, Qpacked, scales, A_l, B_l, codebook, bits, blk, M, m, n, r, y, stream=None, f32=False) -> None:
+    """Comparator (Sec. 3.4 / 4.4): the block-scaled layer plus an additive rank-r adapter, three launches."""
+    cb = _cb_ptr(codebook, bits)
+    fn = _load().lords_adapter_forward_f32 if f32 else _load().lords_adapter_forward
+    _check(fn(x.data_ptr(), Qpacked.data_ptr(), scales.data_ptr(), A_l.data_ptr(), B_l.data_ptr(), cb.ctypes.data, bits, blk,
+              M, m, n, r, y.data_ptr(), _stream_ptr(stream)), "lords_adapter_forward")
 
 
 def lords_poll_status(stream=None) -> int:

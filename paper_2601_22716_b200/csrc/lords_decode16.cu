@@ -126,6 +126,9 @@ struct alignas(64) Dec16Params {
     void *y;
     int y_f32;
     int *status;
+    // block-scale instantiation (Eq. 2, the comparator): one scale per row and block of `blk` columns
+    const uint16_t *scales;   // bf16 [m][nblk]
+    int blk, nblk;
 };
 
 // 64 columns of one row: code pairs -> level pairs, times the matching pairs of S (sp, in and out).
@@ -175,7 +178,10 @@ __device__ __forceinline__ void dequant_half_row(uint32_t qrow, int row, int ch,
     }
 }
 
-template <int BITS, int RP>
+// BLOCK: the scale of an element is its row's block scale (Eq. 2: S = s (x) 1) instead of (BA)_ij: no
+// scale MMA, no factor tiles; a worker thread's 64 columns lie in one block (blk is a multiple of 64),
+// so its S values are one number read from global memory.  Everything else is the same kernel.
+template <int BITS, int RP, bool BLOCK>
 __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __grid_constant__ Dec16Params p)
 {
     using C = XCfg<BITS, RP>;
@@ -211,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
     const uint32_t bar_ready = bars + 8 * C::kBarReady, bar_mma_done = bars + 8 * C::kBarMmaDone;
     const uint32_t bar_acc_full = bars + 8 * C::kBarAccFull, bar_reduce = bars + 8 * C::kBarReduce;
     const uint32_t bar_b_full = bars + 8 * C::kBarBFull;
-    const bool b_by_tma = (p.r & 7) == 0;      // rows of B are 16-byte multiples: the tile comes by TMA
+    const bool b_by_tma = !BLOCK && (p.r & 7) == 0;      // rows of B are 16-byte multiples: the tile comes by TMA
     const uint32_t tmem_slot = bars + 8 * C::kBarCount;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -293,7 +299,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             }
             // B tile: 128 rows x 64 ranks (zero padded) bf16, K-major, 128-byte swizzle: by TMA (below)
             // or, when a row of B is not a multiple of 16 bytes, element by element here
-            if (!b_by_tma && tid < 256) {
+            if (!BLOCK && !b_by_tma && tid < 256) {
                 const int rr = tid >> 1, half = tid & 1;
                 const int i = row0 + rr;
 #pragma unroll
@@ -329,7 +335,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         // all done above
     } else if (warp == kTmaAWarp) {
         // ------------------------------------------------------------------ factor tiles A[:, k-step] (weights)
-        if (lane == 0) {
+        if (!BLOCK && lane == 0) {
             if (b_by_tma) {
                 mbar_expect_tx(bar_b_full, (uint32_t)kBTileBytes);
                 tma_load_2d(b_tile, &p.tm_b, 0, row0, bar_b_full);
@@ -376,7 +382,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         const int sj = warp - kScaleWarp0;
         static_assert(SD == 2 && SA % 2 == 0, "one scale issuer per S buffer; each factor-ring barrier belongs to one of them");
         if (b_by_tma && sj < total && !mbar_wait(bar_b_full, 0)) failed = true;
-        for (int it = sj; it < total && !failed; it += 2) {
+        for (int it = sj; !BLOCK && it < total && !failed; it += 2) {
             const int sa = it % SA, sd = it % SD;
             if (!mbar_wait(bar_a_full + 8 * sa, (uint32_t)((it / SA) & 1))) { failed = true; break; }
             if (it >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((it / SD - 1) & 1))) { failed = true; break; }
@@ -457,10 +463,17 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         const bool stamper = wg == 0 && lane == 0;
         for (int it = g; it < total; it += 2) {
             const int sq = it % SQ, sd = it % SD, ws = it % WS;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * sd, (uint32_t)((it / SD) & 1)))) { failed = true; break; }
-            tc_fence_after_sync();
             // this thread's 64 columns of S, as 32 fp16 pairs
             uint32_t sp[32];
+            if constexpr (BLOCK) {
+                const int i = row0 + row, blkidx = ((ks_a + it) * kStep + ch * 64) / p.blk;
+                const float sc = (i < p.m && blkidx < p.nblk) ? __uint_as_float((uint32_t)p.scales[(size_t)i * p.nblk + blkidx] << 16) : 0.0f;
+                const __half2 s2 = __floats2half2_rn(sc, sc);
+#pragma unroll
+                for (int pp = 0; pp < 32; ++pp) sp[pp] = *reinterpret_cast<const uint32_t *>(&s2);
+            } else {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_s_full + 8 * sd, (uint32_t)((it / SD) & 1)))) { failed = true; break; }
+            tc_fence_after_sync();
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 uint32_t s[32];
@@ -475,6 +488,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_s_empty + 8 * sd);      // S is in registers: the buffer may be refilled
+            }
             if (!__all_sync(0xffffffffu, mbar_wait(bar_q_full + 8 * sq, (uint32_t)((it / SQ) & 1)))) { failed = true; break; }
             dequant_half_row<BITS>(q0 + sq * C::QSTAGE + row * C::QROW, row, ch, lut_lane, sp);
             // the W slot is free once the MMAs of step it - WS have completed
@@ -575,12 +589,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
 }
 
 // One (code width, rank slot) instantiation: launch attributes, resident clusters per size, launch.
-template <int BITS, int RP> struct Dec16Variant {
+template <int BITS, int RP, bool BLOCK> struct Dec16Variant {
     static int prepare(int dev)
     {
         static bool done[kMaxDevices] = {};
         if (!done[dev]) {
-            LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_decode16_kernel<BITS, RP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_decode16_kernel<BITS, RP, BLOCK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                 XCfg<BITS, RP>::SMEM));
             done[dev] = true;
         }
@@ -612,7 +626,7 @@ template <int BITS, int RP> struct Dec16Variant {
             cudaLaunchAttribute attr[2];
             fill(cfg, attr, cs, 1, nullptr);
             int n = 0;
-            const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_decode16_kernel<BITS, RP>, &cfg);
+            const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, lords_decode16_kernel<BITS, RP, BLOCK>, &cfg);
             if (e != cudaSuccess) (void)cudaGetLastError();
             cache[dev][cs] = (e == cudaSuccess && n >= 1) ? n : -1;
         }
@@ -620,9 +634,9 @@ template <int BITS, int RP> struct Dec16Variant {
     }
 };
 
-template <int BITS, int RP> int launch_variant(Dec16Params &k, const Problem &p, const State &st, cudaStream_t stream)
+template <int BITS, int RP, bool BLOCK = false> int launch_variant(Dec16Params &k, const Problem &p, const State &st, cudaStream_t stream)
 {
-    using V = Dec16Variant<BITS, RP>;
+    using V = Dec16Variant<BITS, RP, BLOCK>;
     using C = XCfg<BITS, RP>;
     const int dev = device_slot(st), forced_cs = st.forced_splitk;
     int rc = V::prepare(dev);
@@ -642,12 +656,15 @@ template <int BITS, int RP> int launch_variant(Dec16Params &k, const Problem &p,
     const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
     if (!make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)C::QROW, (uint32_t)kRows,
                      BITS == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.A, (uint64_t)p.n, (uint64_t)p.r, 64, (uint32_t)k.r_pad,
-                     CU_TENSOR_MAP_SWIZZLE_128B) ||
+        (!BLOCK && !make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.A, (uint64_t)p.n, (uint64_t)p.r, 64, (uint32_t)k.r_pad,
+                                CU_TENSOR_MAP_SWIZZLE_128B)) ||
         !make_map_2d(&k.tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.x, (uint64_t)p.n, (uint64_t)p.M, 64, (uint32_t)kTok,
                      CU_TENSOR_MAP_SWIZZLE_128B))
         return LORDS_ERR_CUDA;
-    if ((p.r & 7) == 0) {
+    if (BLOCK) {
+        k.tm_a = k.tm_x;      // not used
+        k.tm_b = k.tm_x;
+    } else if ((p.r & 7) == 0) {
         if (!make_map_2d(&k.tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.B, (uint64_t)p.r, (uint64_t)p.m, 64, (uint32_t)kRows,
                          CU_TENSOR_MAP_SWIZZLE_128B))
             return LORDS_ERR_CUDA;
@@ -657,7 +674,7 @@ template <int BITS, int RP> int launch_variant(Dec16Params &k, const Problem &p,
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
     V::fill(cfg, attr, cs, tiles, stream);
-    LORDS_CUDA_TRY(cudaLaunchKernelEx(&cfg, lords_decode16_kernel<BITS, RP>, k));
+    LORDS_CUDA_TRY(cudaLaunchKernelEx(&cfg, lords_decode16_kernel<BITS, RP, BLOCK>, k));
     return LORDS_OK;
 }
 
@@ -682,6 +699,7 @@ int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
     k.ksteps = (p.n + kStep - 1) / kStep;
     k.y = p.y; k.y_f32 = p.y_f32;
     k.status = st.status_word;
+    k.scales = nullptr; k.blk = 0; k.nblk = 0;
     int rc;
     if (p.bits == 4) rc = launch_variant<4, 32>(k, p, st, stream);
     else if (p.bits == 3) rc = k.r_pad <= 32 ? launch_variant<3, 32>(k, p, st, stream) : launch_variant<3, 64>(k, p, st, stream);
@@ -689,6 +707,30 @@ int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
     if (rc != LORDS_OK) return rc;
     st.last_launches = 1;
     st.last_path = "decode16";
+    return LORDS_OK;
+}
+
+// Block-scale comparator (Eq. 2): y = x (L[Q] (.) (s (x) 1))^T with one bf16 scale per row and block of `blk`
+// columns.  Rules: M <= 16; blk a multiple of 64; n a multiple of 64 (2- and 4-bit) or 128 (3-bit).
+int launch_blockscale16(const Problem &p, const uint16_t *scales, int blk, State &st, cudaStream_t stream)
+{
+    if (p.bits < 2 || p.bits > 4) return LORDS_ERR_UNSUPPORTED;
+    if (p.M > kTok || blk < 64 || blk % 64 != 0) return LORDS_ERR_UNSUPPORTED;
+    if (p.n % (p.bits == 3 ? 128 : 64) != 0) return LORDS_ERR_UNSUPPORTED;
+    Dec16Params k;
+    k.B = nullptr;
+    for (int c = 0; c < 16; ++c) k.levels[c] = p.levels[c];
+    k.M = p.M; k.m = p.m; k.n = p.n; k.r = 16;
+    k.r_pad = 16;
+    k.ksteps = (p.n + kStep - 1) / kStep;
+    k.y = p.y; k.y_f32 = p.y_f32;
+    k.status = st.status_word;
+    k.scales = scales; k.blk = blk; k.nblk = (p.n + blk - 1) / blk;
+    const int rc = p.bits == 4 ? launch_variant<4, 32, true>(k, p, st, stream)
+                 : p.bits == 3 ? launch_variant<3, 32, true>(k, p, st, stream) : launch_variant<2, 32, true>(k, p, st, stream);
+    if (rc != LORDS_OK) return rc;
+    st.last_launches = 1;
+    st.last_path = "blockscale16";
     return LORDS_OK;
 }
 

@@ -420,6 +420,72 @@ int lords_linear_backward_factors(const void *dy, const void *x, const uint8_t *
                                    n, r, dB, dA, st, static_cast<cudaStream_t>(stream));
 }
 
+static int blockscale_common(const void *x, const uint8_t *q, const void *scales, const float *cb, int bits, int blk, int M,
+                             int m, int n, void *y, int y_f32, void *stream)
+{
+    if (!x || !q || !scales || !cb || !y) return LORDS_ERR_NULL;
+    const int g = pack_group(bits);
+    if (g == 0) return LORDS_ERR_BITS;
+    if (M < 1 || m < 1 || n < 1 || n % g != 0 || blk < 1) return LORDS_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(q) || !aligned16(y)) return LORDS_ERR_ALIGN;
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    Problem p;
+    p.x = static_cast<const uint16_t *>(x);
+    p.q = q;
+    p.B = nullptr; p.A = nullptr;
+    for (int c = 0; c < 16; ++c) p.levels[c] = c < (1 << bits) ? cb[c] : 0.0f;
+    p.bits = bits; p.M = M; p.m = m; p.n = n; p.r = 16;
+    p.y = y; p.y_f32 = y_f32;
+    st.last_launches = 0;
+    return launch_blockscale16(p, static_cast<const uint16_t *>(scales), blk, st, static_cast<cudaStream_t>(stream));
+}
+
+int lords_blockscale_forward(const void *x, const uint8_t *Qpacked, const void *scales, const float *codebook, int bits,
+                             int blk, int M, int m, int n, void *y, void *stream)
+{
+    return blockscale_common(x, Qpacked, scales, codebook, bits, blk, M, m, n, y, 0, stream);
+}
+
+int lords_blockscale_forward_f32(const void *x, const uint8_t *Qpacked, const void *scales, const float *codebook, int bits,
+                                 int blk, int M, int m, int n, float *y32, void *stream)
+{
+    return blockscale_common(x, Qpacked, scales, codebook, bits, blk, M, m, n, y32, 1, stream);
+}
+
+static int adapter_common(const void *x, const uint8_t *q, const void *scales, const void *Al, const void *Bl, const float *cb,
+                          int bits, int blk, int M, int m, int n, int r, void *y, int y_f32, void *stream)
+{
+    if (!Al || !Bl || !y) return LORDS_ERR_NULL;
+    if (r < 1 || r > LORDS_R_MAX) return LORDS_ERR_SHAPE;
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    // scratch: the block-scaled product's fp32 accumulators [M][m], then u [M][r]
+    const size_t y32_bytes = ((size_t)M * m * sizeof(float) + 255) & ~(size_t)255;
+    if (M < 1 || m < 1 || y32_bytes + (size_t)M * r * sizeof(float) > st.workspace_bytes) return LORDS_ERR_WORKSPACE;
+    float *y32 = reinterpret_cast<float *>(st.workspace), *u = reinterpret_cast<float *>(st.workspace + y32_bytes);
+    int rc = blockscale_common(x, q, scales, cb, bits, blk, M, m, n, y32, 1, stream);
+    if (rc != LORDS_OK) return rc;
+    rc = launch_adapter(static_cast<const uint16_t *>(x), static_cast<const uint16_t *>(Al), static_cast<const uint16_t *>(Bl), y32, u,
+                        y, y_f32, M, m, n, r, static_cast<cudaStream_t>(stream));
+    if (rc != LORDS_OK) return rc;
+    st.last_launches = 3;
+    st.last_path = "blockscale16+adapter";
+    return LORDS_OK;
+}
+
+int lords_adapter_forward(const void *x, const uint8_t *Qpacked, const void *scales, const void *A_l, const void *B_l,
+                          const float *codebook, int bits, int blk, int M, int m, int n, int r, void *y, void *stream)
+{
+    return adapter_common(x, Qpacked, scales, A_l, B_l, codebook, bits, blk, M, m, n, r, y, 0, stream);
+}
+
+int lords_adapter_forward_f32(const void *x, const uint8_t *Qpacked, const void *scales, const void *A_l, const void *B_l,
+                              const float *codebook, int bits, int blk, int M, int m, int n, int r, float *y32, void *stream)
+{
+    return adapter_common(x, Qpacked, scales, A_l, B_l, codebook, bits, blk, M, m, n, r, y32, 1, stream);
+}
+
 int lords_poll_status(void *stream)
 {
     State &st = state();

@@ -83,4 +83,10 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
                             const float *levels, int bits, int M, int m, int n, int r, float *dB, float *dA,
                             State &st, cudaStream_t stream);
 
+// Comparators (Sec. 4.4, Table 6): the block-scale instantiation of the 16-token decode kernel (Eq. 2) and
+// the two extra launches of an additive low-rank adapter on top of it.
+int launch_blockscale16(const Problem &p, const uint16_t *scales, int blk, State &st, cudaStream_t stream);
+int launch_adapter(const uint16_t *x, const uint16_t *Al, const uint16_t *Bl, const float *y32, float *u, void *y, int y_f32,
+                   int M, int m, int n, int r, cudaStream_t stream);
+
 }  // namespace lords

@@ -374,3 +374,33 @@ def test_backward_input_gradient_is_g_times_the_dequantised_weight():
     What = oracle.dequant_rows(packed, lay.B, lay.A, lay.codebook, 3)
     want = gen.bf16_to_f32(g).astype(np.float64) @ What
     assert np.allclose(dx, want, rtol=1e-12, atol=1e-12 * np.abs(want).max())
+
+
+# ---- the additive-adapter comparator (Sec. 3.4, Sec. 4.4 / Table 6) --------------------------------------
+
+def test_adapter_comparator_against_brute_force():
+    """Four nested loops on a tiny problem: block scale times level times x, plus the adapter's two sums."""
+    import torch
+    m, n, blk, M, r, bits = 6, 64, 32, 2, 3, 4
+    lay, s = gen.make_blockwise_layer(m, n, blk, M, bits=bits, seed=4)
+    g = torch.Generator().manual_seed(9)
+    Al = gen.bf16_bits(torch.randn(r, n, generator=g) * 0.1)
+    Bl = gen.bf16_bits(torch.randn(m, r, generator=g) * 0.1)
+    qp = oracle.pack_codes(lay.codes, bits)
+    got = oracle.adapter_forward(lay.x, qp, s, blk, Al, Bl, lay.codebook, bits)
+    xf, sf, af, bf = _f64(lay.x), _f64(s), _f64(Al), _f64(Bl)
+    for t in range(M):
+        for i in range(m):
+            acc = 0.0
+            for j in range(n):
+                acc += xf[t, j] * float(lay.codebook[lay.codes[i, j]]) * sf[i, j // blk]
+            for k in range(r):
+                u = 0.0
+                for j in range(n):
+                    u += xf[t, j] * af[k, j]
+                acc += u * bf[i, k]
+            assert abs(got[t, i] - acc) <= 1e-12 * max(1.0, abs(acc))
+    # without an adapter it is the block-wise forward itself
+    zero = np.zeros_like(Al)
+    assert np.array_equal(oracle.adapter_forward(lay.x, qp, s, blk, zero, Bl, lay.codebook, bits),
+                          oracle.forward(lay.x, qp, lay.B, lay.A, lay.codebook, bits))
