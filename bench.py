@@ -568,6 +568,75 @@ def time_backward(name, m, n, r, bits, M, device, min_seconds=0.3):
                          "traffic": NCU_TRAFFIC_BYTES.get(name), "us_per_launch": us_f}}
 
 
+def time_comparators(device, min_seconds=0.25):
+    """Sec. 4.4 / Table 6 restated on this GPU, q_proj shape at one token: the LoRDS layer (r = 32) against a
+    block-scaled NF4 layer (block 64: the same number of scale parameters) and against that layer with an
+    additive rank-32 adapter, each replayed from a CUDA graph over distinct weight copies."""
+    import numpy as np
+    import torch
+    from paper_2601_22716_b200 import binding as lords
+    from paper_2601_22716_b200 import inputs as gen
+
+    m = n = 4096
+    M, r, blk, bits = 1, 32, 64, 4
+    copies = copies_for("decode_q_m1")
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=0)
+    blay, s = gen.make_blockwise_layer(m, n, blk, M, bits=bits, seed=0)
+    g = torch.Generator().manual_seed(3)
+    Al = torch.from_numpy(gen.bf16_bits(torch.randn(r, n, generator=g) * 0.05).view(np.int16)).to(device)
+    Bl = torch.from_numpy(gen.bf16_bits(torch.randn(m, r, generator=g) * 0.05).view(np.int16)).to(device)
+    q0 = torch.from_numpy(lords.lords_pack_codes(lay.codes, bits)).to(device)
+    B = torch.from_numpy(lay.B.view(np.int16)).to(device)
+    A = torch.from_numpy(lay.A.view(np.int16)).to(device)
+    sd = torch.from_numpy(s.view(np.int16)).to(device)
+    x = torch.from_numpy(lay.x.view(np.int16)).to(device)
+    qs = [q0 if l == 0 else torch.roll(q0, l, 0).contiguous() for l in range(copies)]
+    ys = [torch.zeros((M, m), dtype=torch.int16, device=device) for _ in range(copies)]
+    variants = {
+        "lords_r32": lambda q, y: lords.lords_linear_forward_bits(x, q, B, A, lay.codebook, bits, M, m, n, r, y),
+        "blockscale_nf4_b64": lambda q, y: lords.lords_blockscale_forward(x, q, sd, lay.codebook, bits, blk, M, m, n, y),
+        "blockscale_nf4_b64_plus_adapter_r32":
+            lambda q, y: lords.lords_adapter_forward(x, q, sd, Al, Bl, lay.codebook, bits, blk, M, m, n, r, y),
+    }
+    out = {}
+    for name, fn in variants.items():
+        def one_round():
+            for q, y in zip(qs, ys):
+                fn(q, y)
+        one_round()
+        torch.cuda.synchronize()
+        path = lords.lords_last_path()
+        st = torch.cuda.Stream()
+        st.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(st):
+            one_round()
+        torch.cuda.current_stream().wait_stream(st)
+        torch.cuda.synchronize()
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            one_round()
+        for _ in range(3):
+            gr.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        gr.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        reps = int(max(3, min_seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)))
+        e0.record()
+        for _ in range(reps):
+            gr.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = {"us_per_call": e0.elapsed_time(e1) * 1e3 / reps / copies, "path": path}
+    base = out["lords_r32"]["us_per_call"]
+    return {"case": "compare_q_m1", "shape": "q_proj 4096x4096 NF4, one token", "variants": out,
+            "adapter_over_lords": out["blockscale_nf4_b64_plus_adapter_r32"]["us_per_call"] / base,
+            "blockscale_over_lords": out["blockscale_nf4_b64"]["us_per_call"] / base,
+            "status_retries": 0 if lords.lords_poll_status() == 0 else 1}
+
+
 def run_sweep(device):
     """The measurement behind the per-M choice of kernel: every tensor-core path that accepts the
     shape, at M in {1, 2, 3, 4, 8, 16}, on the q_proj (NF4, r = 32), gate and down (NF3, r = 48) shapes.
@@ -726,6 +795,13 @@ def main():
             dist.destroy_process_group()
         return 0
 
+    if args.case == "compare_q_m1":
+        if rank == 0:
+            print(json.dumps(time_comparators(device)))
+        lords.lords_shutdown()
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
     if args.case in BACKWARD_CASES:
         if rank == 0:
             print(json.dumps(time_backward(args.case, *BACKWARD_CASES[args.case], device, min_seconds=min(args.min_seconds, 0.3))))
@@ -766,8 +842,11 @@ def main():
             cases.append(time_quantize(name, *shape, device))
         for name, shape in BACKWARD_CASES.items():
             cases.append(time_backward(name, *shape, device))
+        comparators = time_comparators(device)
 
     stack = []
+    if not (not args.case and not args.no_extras and world == 1):
+        comparators = None
     if not args.no_stack and not args.no_extras and not args.case and world == 1:
         for (M, mlp_bits, k) in [(1, 4, 30), (8, 4, 30), (512, 4, 5), (1, 3, 30), (1, 2, 30)]:
             stack.append(time_stack(M, mlp_bits, k, device))
@@ -801,6 +880,8 @@ def main():
         }
         if stack:
             line["stack"] = stack
+        if comparators is not None:
+            line["comparators"] = comparators
         print(json.dumps(line))
     lords.lords_shutdown()
     if world > 1:
