@@ -112,3 +112,27 @@ def test_noalloc_entry_rejects_oversized_problems():
     ok = P(4096)   # aligned and never dereferenced: the size check comes first
     # 2 * M * m = 2 * 512 * 4096 floats > 2^20
     assert f(ok, ok, ok, ok, ctypes.cast(cb, P), 4, 512, 4096, 4096, 32, ok, None) == -9
+
+
+def test_reinitialising_on_the_same_device_keeps_every_path_working():
+    """lords_shutdown followed by lords_init: the per-device launch attributes and occupancy figures are
+    kept, the device buffers are new; every kernel path still runs and agrees with the oracle."""
+    import torch
+    from paper_2601_22716_b200 import binding as lords
+    torch.cuda.set_device(0)
+    cases = [(gen.make_layer(512, 1024, 32, 1, bits=4, seed=51), "decode"),
+             (gen.make_layer(384, 1024, 32, 8, bits=4, seed=52), "decode16"),
+             (gen.make_layer(256, 512, 16, 64, bits=4, seed=53), "umma")]
+    uploaded = [_upload(lay, lords, torch) for lay, _ in cases]
+    for round_ in range(2):
+        lords.lords_init(0, 0)
+        try:
+            for (lay, path), (packed, q, B, A, x) in zip(cases, uploaded):
+                y = torch.full((lay.M, lay.m), 0x7FC0, dtype=torch.int16, device="cuda:0")
+                lords.lords_linear_forward_bits(x, q, B, A, lay.codebook, lay.bits, lay.M, lay.m, lay.n, lay.r, y)
+                assert lords.lords_last_path() == path, (round_, path)
+                torch.cuda.synchronize()
+                assert lords.lords_poll_status() == 0
+                _check_bf16_against_oracle(y.cpu().numpy().view(np.uint16), lay, packed)
+        finally:
+            lords.lords_shutdown()
