@@ -248,6 +248,17 @@ __global__ void __launch_bounds__(kThreadsQ, 3) lords_quantize_kernel(const __gr
 #pragma unroll
         for (int c = 0; c < 16; ++c) lv[c] = SORTED ? p.mids[c] : p.levels[c];
         const size_t qpitch = (size_t)p.n * BITS / 8;
+        // the row's 32 weights of a half step are requested one half step ahead, so that their way
+        // from HBM overlaps the search of the half step before
+        uint4 wv[4], wn[4];
+        auto load_w = [&](uint4 (&dst)[4], int it, int h) {
+            if (i < p.m && it < total) {
+                const uint4 *wp = reinterpret_cast<const uint4 *>(p.W + (size_t)i * p.n + (size_t)(st_a + it) * kColsQ + h * 32);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) dst[v] = __ldg(wp + v);
+            }
+        };
+        load_w(wv, 0, 0);
         for (int it = 0; it < total; ++it) {
             const int sd = it % kSDQ;
             const int col0 = (st_a + it) * kColsQ;
@@ -257,13 +268,7 @@ __global__ void __launch_bounds__(kThreadsQ, 3) lords_quantize_kernel(const __gr
             for (int h = 0; h < 2; ++h) {
                 uint32_t s[32];
                 tmem_ld_32x32(lane_addr + (uint32_t)(sd * kColsQ + h * 32), s);
-                // the row's 32 weights of these columns meanwhile
-                uint4 wv[4];
-                if (i < p.m) {
-                    const uint4 *wp = reinterpret_cast<const uint4 *>(p.W + (size_t)i * p.n + col0 + h * 32);
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) wv[v] = __ldg(wp + v);
-                }
+                load_w(wn, h == 0 ? it : it + 1, h == 0 ? 1 : 0);
                 tmem_wait_ld();
                 if (h == 1) {
                     // S is in registers: the buffer may be refilled
@@ -291,6 +296,8 @@ __global__ void __launch_bounds__(kThreadsQ, 3) lords_quantize_kernel(const __gr
                     }
                     store_codes<BITS>(p.Q + (size_t)i * qpitch + (size_t)(col0 + h * 32) * BITS / 8, codes);
                 }
+#pragma unroll
+                for (int v = 0; v < 4; ++v) wv[v] = wn[v];
             }
         }
     }

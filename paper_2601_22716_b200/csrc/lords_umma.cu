@@ -107,8 +107,10 @@ __device__ __forceinline__ void dequant_chunk(uint32_t qrow, int row, int c, uin
         for (int wi = 0; wi < 4; ++wi)
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
-                const uint32_t sh = b == 0 ? (w[wi] << 7) : (w[wi] >> (8 * b - 7));
-                lv[wi * 4 + b] = lds_u32(lut_lane + (sh & 0x7F80u));
+                // byte b of the word is the code pair: one byte permute isolates it, one multiply-add makes
+                // the address of its entry (entries are 128 bytes apart)
+                const uint32_t pair = __byte_perm(w[wi], 0u, 0x4440u | (uint32_t)b);
+                lv[wi * 4 + b] = lds_u32(lut_lane + pair * 128u);
             }
     } else if constexpr (BITS == 2) {
         // 32-byte rows: chunk c is the 64-bit group at byte 8c; pair p sits at bit 4p of it
