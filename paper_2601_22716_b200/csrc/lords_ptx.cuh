@@ -117,8 +117,6 @@ __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("grid
 // Returns when the previous kernel of the stream has finished and its writes are visible.
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
-
 // ---- proxies / fences -------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem()
 {
@@ -156,22 +154,6 @@ __device__ __forceinline__ void tmem_relinquish()
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
 {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-
-// The same three for a CTA pair (cta_group::2): one warp of EACH of the two CTAs executes them, and
-// every tcgen05 instruction of such a kernel names cta_group::2.
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_result, uint32_t cols)
-{
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_result), "r"(cols)
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish_pair()
-{
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 
 // 32 lanes x 32 consecutive 32-bit columns: thread l of the warp receives lane (base_lane + l).
@@ -266,10 +248,6 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t ra
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster_f32(uint32_t cluster_addr, float v)
-{
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
-}
 // Asynchronous 4-byte store into the shared memory of a CTA of the cluster; its completion is
 // counted in bytes on an mbarrier of that same CTA, which also makes the value visible to whoever
 // waits on the barrier: no release fence on the storing side.
@@ -281,13 +259,6 @@ __device__ __forceinline__ void st_async_cluster_f32(uint32_t cluster_addr, floa
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-// Arrival on an mbarrier of another CTA of the cluster without a cluster-scope release: for hand-offs
-// whose data does not travel through generic memory (tensor memory written with tcgen05.st and fenced
-// with tcgen05 fences; shared memory of the arriving CTA itself, fenced for the async proxy).
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar)
-{
-    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
 {
@@ -381,40 +352,6 @@ __device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, ui
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// CTA-pair forms (cta_group::2), issued by one thread of the pair's even-ranked CTA.
-// D[tmem, 256 rows: 128 lanes in each CTA] (+)= A[tmem of each CTA] * B[smem: rows 0..N/2-1 in the even
-// CTA, N/2..N-1 in the odd one, at the same shared-memory offset]
-__device__ __forceinline__ void umma_pair_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                                 uint32_t accumulate)
-{
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n"
-        "}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// Arrive once on the barrier at the same shared-memory offset in every CTA of `cta_mask` (bit = rank
-// in the cluster) when every MMA issued so far by this thread has completed.
-__device__ __forceinline__ void umma_pair_commit(uint32_t bar, uint16_t cta_mask)
-{
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(cta_mask) : "memory");
-}
-
-// Two fp32 products in one instruction: {a.x * b.x, a.y * b.y}, round to nearest even.
-__device__ __forceinline__ float2 mul_f32x2(float2 a, float2 b)
-{
-    unsigned long long ua, ub, ud;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(ua) : "f"(a.x), "f"(a.y));
-    asm("mov.b64 %0, {%1, %2};" : "=l"(ub) : "f"(b.x), "f"(b.y));
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(ud) : "l"(ua), "l"(ub));
-    float2 d;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(ud));
-    return d;
 }
 
 }  // namespace ptx
