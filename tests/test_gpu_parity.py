@@ -409,6 +409,45 @@ def test_status_word_round_trip_and_recovery(lords):
     assert np.array_equal(y32, y32b) and np.array_equal(ybf, ybfb)
 
 
+def test_many_back_to_back_launches_of_the_two_half_kernel_leave_no_status(lords):
+    """The 3-bit gate shape runs the two-half variant of the M <= 2 kernel, whose rings are three
+    stages deep while its converter groups take the k-steps alternately.  Several thousand dependent
+    launches over distinct weight copies (replayed from a CUDA graph, as a model's layers are) must
+    leave the status word clear and reproduce the first result bit for bit: a barrier that two groups
+    share by parity alone would show up here as a recorded give-up."""
+    import torch
+    lay = gen.make_layer(14336, 4096, 48, 1, bits=3, seed=91)
+    dl = DeviceLayer(lay)
+    copies = 6
+    qs = [dl.q] + [torch.roll(dl.q, l, 0).contiguous() for l in range(1, copies)]
+    ys = [torch.zeros((1, lay.m), dtype=torch.int16, device="cuda:0") for _ in range(copies)]
+
+    def one_round():
+        for q, y in zip(qs, ys):
+            lords.lords_linear_forward_bits(dl.x, q, dl.B, dl.A, lay.codebook, 3, 1, lay.m, lay.n, lay.r, y)
+
+    one_round()
+    torch.cuda.synchronize()
+    assert lords.lords_last_path() == "decode"
+    first = [y.clone() for y in ys]
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        one_round()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(20):
+            one_round()
+    for _ in range(40):                      # 40 x 20 x 6 = 4800 launches
+        g.replay()
+    torch.cuda.synchronize()
+    assert lords.lords_poll_status() == 0
+    for y, f in zip(ys, first):
+        assert torch.equal(y, f)
+
+
 def test_host_buffer_entry_point_matches_device_entry(lords):
     import torch
     lay = gen.make_layer(512, 1024, 16, 4, bits=4, seed=12)
