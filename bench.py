@@ -556,13 +556,18 @@ def time_backward(name, m, n, r, bits, M, device, min_seconds=0.3):
     peaks = measured_peaks()
     flops = 2.0 * M * m * n
     tf_dx = flops / (us_dx * 1e-6) / 1e12
-    tf_f = (flops + 4.0 * m * n * r) / (us_f * 1e-6) / 1e12      # g^T x formed once (one CTA per tile of W), plus the two folds
+    # CUDA-core work of the factor gradients: the two folds and the level multiply; with the schedules that
+    # form g^T x on the CUDA cores as well, that product too (once: one CTA per tile of W)
+    alu_flops = 4.0 * m * n * r + m * n + (0.0 if path_f == "backward_tensor" else flops)
+    tf_f = alu_flops / (us_f * 1e-6) / 1e12
     return {"case": name, "path": f"{path_dx}+{path_f}", "us_per_call": us_dx + us_f, "gbs": None, "tflops": None,
             "copies": 1, "rounds": reps_dx, "steps": 1, "status_retries": 0 if status == 0 else 1,
             "input_gradient": {"us": us_dx, "path": path_dx, "tflops": tf_dx,
                                "roofline": {"bound": "tensor", "achieved": tf_dx, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                                             "frac": tf_dx / peaks["bf16_tflops"], "peak_kind": "burst", "traffic": None}},
-            "factor_gradients": {"us": us_f, "path": path_f, "tflops": tf_f},
+            "factor_gradients": {"us": us_f, "path": path_f, "alu_tflops": tf_f,
+                                 "tile_product_tflops": flops / (us_f * 1e-6) / 1e12,
+                                 "tile_product_on": "tensor cores" if path_f == "backward_tensor" else "CUDA cores"},
             "roofline": {"bound": "alu", "achieved": tf_f, "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s",
                          "frac": tf_f / FP32_ALU_TFLOPS, "peak_source": "148 SMs x 128 fp32 lanes x 2 flops x 1.965 GHz",
                          "traffic": NCU_TRAFFIC_BYTES.get(name), "us_per_launch": us_f}}

@@ -21,15 +21,24 @@
 //          holds the contributions (4 r (m n / 64 + n m / 64) bytes).
 //   walk:  one CTA per 64 rows (dB) or 64 columns (dA) walks over the other dimension and keeps its
 //          sums in registers.  No scratch memory, g^T x formed once per gradient.
+//   tensor: the first schedule with the tile product g^T x on the tensor cores (tcgen05, bf16 operands
+//          straight from g and x by TMA, fp32 accumulator in TMEM) and only the level multiply and
+//          the two folds on the CUDA cores.  Taken when the row pitches suit TMA (m, n multiples of 8).
 // Either way every output element is summed in a fixed order without atomics: runs are bit-identical.
-// Bound: fp32 ALU, m n M fused multiply-adds for the tile product (twice with the second schedule).
+// Bound: fp32 ALU, m n M fused multiply-adds for the tile product (twice with the walk), or, with the
+// tensor schedule, the 2 m n r multiply-adds of the folds.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "lords_internal.h"
+#include "lords_ptx.cuh"
+#include "lords_tc_common.cuh"
 
 namespace lords {
 
 namespace {
+
+using namespace ptx;
 
 __device__ __forceinline__ float bf16f(uint16_t h) { return __uint_as_float((uint32_t)h << 16); }
 
@@ -295,6 +304,192 @@ __global__ void __launch_bounds__(kBwThreads) lords_backward_tile_kernel(const B
     }
 }
 
+// Schedule "tensor": CTA (jt, it) handles rows it * 128 .. and columns jt * 64 .. of W.
+//   G[128 x 64] = sum_t g[t][i] x[t][j]:  both operands are MN-major in shared memory (a row of the tile
+//   is one token: 64 consecutive rows or columns of W), K = 16 tokens per MMA, 64 tokens per stage.
+// Warps 0..7: epilogue (level multiply, folds); 8: TMEM allocation and MMA issue; 9: TMA producer.
+constexpr int kTcRows = 128, kTcCols = 64, kTcTok = 64, kTcStages = 3;
+constexpr int kTcThreads = 320;
+constexpr int kTcGAtom = kTcTok * 128;                        // 64 tokens x 64 rows of W, bf16
+constexpr int kTcStage = 2 * kTcGAtom + kTcTok * 128;         // g: two atoms, x: one
+constexpr uint32_t kTcTmemCols = 64;
+
+struct alignas(64) BwTcParams {
+    CUtensorMap tm_g;     // bf16 [M][m], box {64, 64}, 128-byte swizzle (tokens past M read as zero)
+    CUtensorMap tm_x;     // bf16 [M][n], box {64, 64}, 128-byte swizzle
+    BwParams b;
+    float *part_dB;       // [n / 64 tiles][m][r4]
+    float *part_dA;       // [m / 128 tiles][r4][n]
+    int *status;
+};
+
+__host__ __device__ constexpr int bw_tc_smem(int r4)
+{
+    // the epilogue's buffers (dS tile, the two factor slices) reuse the stages once the MMAs are done
+    const int stages = kTcStages * kTcStage;
+    const int epi = kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 2 + r4 * (kTcRows + 2) * 2;
+    return 1024 + (stages > epi ? stages : epi) + 256;
+}
+
+__global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __grid_constant__ BwTcParams p)
+{
+    extern __shared__ uint8_t tc_smem_raw[];
+    const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
+    uint8_t *base_ptr = tc_smem_raw + (base - smem_u32(tc_smem_raw));
+    const int r4 = (p.b.r + 3) & ~3;
+    const int stages_bytes = kTcStages * kTcStage;
+    const int epi_bytes = kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 2 + r4 * (kTcRows + 2) * 2;
+    const uint32_t bars = base + (uint32_t)(stages_bytes > epi_bytes ? stages_bytes : epi_bytes);
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * kTcStages, bar_acc = bar_empty + 8 * kTcStages;
+    const uint32_t tmem_slot = bar_acc + 8;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int jt = blockIdx.x, it = blockIdx.y;
+    const int i0 = it * kTcRows, j0 = jt * kTcCols;
+    const int chunks = (p.b.M + kTcTok - 1) / kTcTok;
+    const int *status = p.status;
+    bool failed = false;
+
+    if (tid == 0) {
+        for (int s = 0; s < kTcStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_acc, 1);
+        fence_mbar_init();
+    }
+    if (warp == 8) {
+        tmem_alloc(tmem_slot, kTcTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+
+    if (warp == 9) {
+        if (lane == 0) {
+            tma_prefetch_desc(&p.tm_g);
+            tma_prefetch_desc(&p.tm_x);
+            for (int c = 0; c < chunks; ++c) {
+                const int s = c % kTcStages;
+                if (c >= kTcStages && !mbar_wait(bar_empty + 8 * s, (uint32_t)((c / kTcStages - 1) & 1), status, 41)) { failed = true; break; }
+                const uint32_t bar = bar_full + 8 * s, st0 = base + (uint32_t)(s * kTcStage);
+                mbar_expect_tx(bar, (uint32_t)kTcStage);
+                tma_load_2d(st0, &p.tm_g, i0, c * kTcTok, bar);
+                tma_load_2d(st0 + kTcGAtom, &p.tm_g, i0 + 64, c * kTcTok, bar);
+                tma_load_2d(st0 + 2 * kTcGAtom, &p.tm_x, j0, c * kTcTok, bar);
+            }
+        }
+    } else if (warp == 8) {
+        constexpr uint32_t idesc = umma_idesc_f16(1, 1, 1, kTcRows, kTcCols);     // bf16, both operands MN-major
+        const uint32_t a_hi = (uint32_t)(umma_desc_sw128(0, 1024, (uint32_t)kTcGAtom) >> 32);
+        const uint32_t a_lo0 = (uint32_t)umma_desc_sw128(0, 1024, (uint32_t)kTcGAtom) | ((base & 0x3FFFFu) >> 4);
+        const uint32_t b_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
+        const uint32_t b_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | (((base + 2 * kTcGAtom) & 0x3FFFFu) >> 4);
+        for (int c = 0; c < chunks; ++c) {
+            const int s = c % kTcStages;
+            if (!mbar_wait(bar_full + 8 * s, (uint32_t)((c / kTcStages) & 1), status, 42)) { failed = true; break; }
+            tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t off = (uint32_t)((s * kTcStage) >> 4);
+#pragma unroll
+                for (int k = 0; k < kTcTok / 16; ++k)      // 16 tokens = 16 rows of 128 bytes
+                    umma_f16_ss(tmem_base, umma_desc_pack(a_lo0 + off + k * 128, a_hi), umma_desc_pack(b_lo0 + off + k * 128, b_hi),
+                                idesc, (c > 0 || k > 0) ? 1u : 0u);
+                umma_commit(bar_empty + 8 * s);
+                if (c == chunks - 1) umma_commit(bar_acc);
+            }
+            __syncwarp();
+        }
+    } else {
+        // ---- epilogue: thread = (row quadrant q, column half ch): row i0 + q * 32 + lane, 32 columns
+        const int q = warp & 3, ch = warp >> 2;
+        const int ri = q * 32 + lane, i = i0 + ri;
+        // rows of the dS tile are 66 floats apart (pairs of columns are read as one 8-byte word), rows
+        // of the factor slices 33 and 65 words (neighbouring ranks fall into different banks)
+        float (*ds)[kTcCols + 2] = reinterpret_cast<float (*)[kTcCols + 2]>(base_ptr);
+        uint16_t (*fa)[kTcCols + 2] = reinterpret_cast<uint16_t (*)[kTcCols + 2]>(base_ptr + kTcRows * (kTcCols + 2) * 4);
+        uint16_t (*fb)[kTcRows + 2] =
+            reinterpret_cast<uint16_t (*)[kTcRows + 2]>(base_ptr + kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 2);
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, 0, status, 43));
+        if (!ok) failed = true;
+        tc_fence_after_sync();
+        uint32_t gacc[32];
+        if (ok) {
+            tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ch * 32), gacc);
+            tmem_wait_ld();
+        }
+        // every MMA has completed (the accumulator barrier), so every stage has been read: the stages'
+        // memory now holds the dS tile and the factor slices
+        const size_t row_bytes = (size_t)p.b.n * p.b.bits / 8;
+#pragma unroll
+        for (int cidx = 0; cidx < 32; ++cidx) {
+            const int j = j0 + ch * 32 + cidx;
+            float v = 0.0f;
+            if (ok && i < p.b.m && j < p.b.n) v = __uint_as_float(gacc[cidx]) * p.b.levels[read_code(p.b.q, row_bytes, i, j, p.b.bits)];
+            ds[ri][ch * 32 + cidx] = v;
+        }
+        const int et = tid;                                       // 0 .. 255
+        for (int e = et; e < r4 * kTcCols; e += 256) {            // A[k][j0 ..]
+            const int k = e / kTcCols, cidx = e % kTcCols;
+            fa[k][cidx] = (k < p.b.r && j0 + cidx < p.b.n) ? p.b.A[(size_t)k * p.b.n + j0 + cidx] : (uint16_t)0;
+        }
+        for (int e = et; e < r4 * kTcRows; e += 256) {            // B[i0 ..][k] stored [k][i]
+            const int k = e / kTcRows, cidx = e % kTcRows;
+            fb[k][cidx] = (k < p.b.r && i0 + cidx < p.b.m) ? p.b.B[(size_t)(i0 + cidx) * p.b.r + k] : (uint16_t)0;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // The folds, four ranks per thread so that a value of dS is read once for four products; the
+        // factors are read as pairs of bf16.  Each output is one thread's sum in index order.
+        if (p.part_dB) {
+            float *out = p.part_dB + ((size_t)jt * p.b.m + i0) * r4;
+            for (int u = et; u < (r4 / 4) * kTcRows; u += 256) {          // dB[ii][k0 .. k0 + 3] = sum_j dS[ii][j] A[k][j]
+                const int ii = u % kTcRows, k0 = (u / kTcRows) * 4;
+                float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 4
+                for (int jp = 0; jp < kTcCols / 2; ++jp) {
+                    const float2 d = *reinterpret_cast<const float2 *>(&ds[ii][2 * jp]);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint32_t w = *reinterpret_cast<const uint32_t *>(&fa[k0 + kk][2 * jp]);
+                        acc[kk] = fmaf(d.x, __uint_as_float(w << 16), acc[kk]);
+                        acc[kk] = fmaf(d.y, __uint_as_float(w & 0xFFFF0000u), acc[kk]);
+                    }
+                }
+                if (i0 + ii < p.b.m)
+                    *reinterpret_cast<float4 *>(&out[(size_t)ii * r4 + k0]) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            }
+        }
+        if (p.part_dA) {
+            float *out = p.part_dA + (size_t)it * r4 * p.b.n + j0;
+            for (int u = et; u < (r4 / 4) * kTcCols; u += 256) {          // dA[k0 .. k0 + 3][j] = sum_i B[i][k] dS[i][j]
+                const int j = u % kTcCols, k0 = (u / kTcCols) * 4;
+                float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 4
+                for (int ip = 0; ip < kTcRows / 2; ++ip) {
+                    const float d0 = ds[2 * ip][j], d1 = ds[2 * ip + 1][j];
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint32_t w = *reinterpret_cast<const uint32_t *>(&fb[k0 + kk][2 * ip]);
+                        acc[kk] = fmaf(__uint_as_float(w << 16), d0, acc[kk]);
+                        acc[kk] = fmaf(__uint_as_float(w & 0xFFFF0000u), d1, acc[kk]);
+                    }
+                }
+                if (j0 + j < p.b.n)
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) out[(size_t)(k0 + kk) * p.b.n + j] = acc[kk];
+            }
+        }
+    }
+
+    if (failed) atomicExch(p.status, LORDS_ERR_TIMEOUT);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 8) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTcTmemCols);
+    }
+}
+
 // out[e] = sum over tiles t (in order) of part[t * stride + pos(e)]: dB (rows = m, inner = r, inner4 = r4)
 // or dA (rows = r, inner = inner4 = n).
 __global__ void lords_backward_reduce_kernel(const float *__restrict__ part, float *__restrict__ out, int tiles, size_t stride,
@@ -342,6 +537,46 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
     // schedule "tiles" when the workspace holds the tiles' contributions
     const int r4 = (r + 3) & ~3, it_n = (m + kT - 1) / kT, jt_n = (n + kT - 1) / kT;
     const size_t need_b = dB ? (size_t)jt_n * m * r4 * sizeof(float) : 0, need_a = dA ? (size_t)it_n * r4 * n * sizeof(float) : 0;
+    // schedule "tensor": the same with 128 x 64 tiles and the tile product on the tensor cores
+    {
+        const int it_t = (m + kTcRows - 1) / kTcRows, jt_t = (n + kTcCols - 1) / kTcCols;
+        const size_t nb = dB ? (size_t)jt_t * m * r4 * sizeof(float) : 0, na = dA ? (size_t)it_t * r4 * n * sizeof(float) : 0;
+        if (st.forced_path == 0 && m % 8 == 0 && n % 8 == 0 && it_t <= 65535 && nb + na + 256 <= st.workspace_bytes) {
+            BwTcParams k;
+            k.b = p;
+            k.part_dB = dB ? reinterpret_cast<float *>(st.workspace) : nullptr;
+            k.part_dA = dA ? reinterpret_cast<float *>(st.workspace + ((nb + 255) & ~(size_t)255)) : nullptr;
+            k.status = st.status_word;
+            if (!make_map_2d(&k.tm_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, g, (uint64_t)m, (uint64_t)M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+                !make_map_2d(&k.tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, (uint64_t)n, (uint64_t)M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B))
+                return LORDS_ERR_CUDA;
+            const int smem = bw_tc_smem(r4);
+            static int attr_set[kMaxDevices] = {};
+            const int dev = device_slot(st);
+            if (attr_set[dev] < smem) {
+                LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_backward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bw_tc_smem(kRMaxBw)));
+                attr_set[dev] = bw_tc_smem(kRMaxBw);
+            }
+            lords_backward_tc_kernel<<<dim3((unsigned)jt_t, (unsigned)it_t), kTcThreads, smem, stream>>>(k);
+            LORDS_CUDA_TRY(cudaGetLastError());
+            ++launches;
+            if (dB) {
+                const size_t total = (size_t)m * r;
+                lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(k.part_dB, dB, jt_t, (size_t)m * r4, m, r, r4);
+                LORDS_CUDA_TRY(cudaGetLastError());
+                ++launches;
+            }
+            if (dA) {
+                const size_t total = (size_t)r * n;
+                lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(k.part_dA, dA, it_t, (size_t)r4 * n, r, n, n);
+                LORDS_CUDA_TRY(cudaGetLastError());
+                ++launches;
+            }
+            st.last_launches = launches;
+            st.last_path = "backward_tensor";
+            return LORDS_OK;
+        }
+    }
     if (it_n <= 65535 && need_b + need_a + 256 <= st.workspace_bytes && st.forced_path != 1) {
         float *part_b = dB ? reinterpret_cast<float *>(st.workspace) : nullptr;
         float *part_a = dA ? reinterpret_cast<float *>(st.workspace + ((need_b + 255) & ~(size_t)255)) : nullptr;

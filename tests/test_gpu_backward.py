@@ -92,9 +92,12 @@ def test_backward_against_the_oracle(lords, bits, m, n, r, M, mixed, path):
     lords.lords_linear_backward_input(gd, qt, Bd, Ad, lay.codebook, bits, M, m, n, r, dxbf)
     assert lords.lords_last_path() == path
     check_against_oracle(dx32.cpu().numpy(), dxbf.cpu().numpy().view(np.uint16), dx64)
-    # both schedules of the factor gradients: one CTA per tile of W with the contributions summed by a
-    # second kernel (taken when the workspace holds them), and the walk that needs no scratch memory
-    for option, schedule, launches in (("auto", "backward_tiles", 3), ("simt", "backward_walk", 2)):
+    # the three schedules of the factor gradients: the tile product on the tensor cores (taken when the row
+    # pitches of g and x suit TMA), one CTA per tile of W on the CUDA cores -- both with the tiles'
+    # contributions summed by a second kernel --, and the walk that needs no scratch memory.  (Any forced
+    # tensor-core forward path switches the tensor schedule off, "simt" leaves only the walk.)
+    first = "backward_tensor" if m % 8 == 0 and n % 8 == 0 else "backward_tiles"
+    for option, schedule, launches in (("auto", first, 3), ("decode", "backward_tiles", 3), ("simt", "backward_walk", 2)):
         dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
         dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
         lords.lords_set_option("path", option)
@@ -129,7 +132,7 @@ def test_backward_integer_case_is_bit_exact(lords, bits, m, n, r, M):
     lords.lords_linear_backward_input_f32(gd, qt, Bd, Ad, lay.codebook, bits, M, m, n, r, dx32)
     torch.cuda.synchronize()
     assert np.array_equal(dx32.cpu().numpy().astype(np.float64), dx64)
-    for option in ("auto", "simt"):
+    for option in ("auto", "decode", "simt"):
         dB.fill_(float("nan")); dA.fill_(float("nan"))
         lords.lords_set_option("path", option)
         try:
@@ -153,7 +156,7 @@ def test_backward_factors_one_at_a_time_and_bad_arguments(lords):
     dB = torch.zeros((128, 8), dtype=torch.float32, device="cuda:0")
     dA = torch.zeros((8, 128), dtype=torch.float32, device="cuda:0")
     lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, 4, 2, 128, 128, 8, dB, None)
-    assert lords.lords_last_launch_count() == 2        # the tile kernel and one sum
+    assert lords.lords_last_path() == "backward_tensor" and lords.lords_last_launch_count() == 2    # the tile kernel and one sum
     lords.lords_linear_backward_factors(gd, xd, q, Bd, Ad, lay.codebook, 4, 2, 128, 128, 8, None, dA)
     torch.cuda.synchronize()
     assert error_metrics(dB.cpu().numpy(), dB64)[0] <= FACTOR_NORMWISE_TOL
