@@ -196,8 +196,12 @@ int lords_quantize_codes(const void *W, const void *B, const void *A, const floa
  *   is seen, so the first call of a given size must not be made during stream capture.
  *   dx: device, bf16 [M][n] (or float [M][n] for _f32).
  * lords_linear_backward_factors: dB (device, float [m][r]) and dA (device, float [r][n]); either may
- *   be NULL.  fp32 on the CUDA cores, every element summed by one thread in a fixed order (runs are
- *   bit-identical).  x: device, bf16 [M][n].  Any bits in {2,3,4}, r <= LORDS_R_MAX.
+ *   be NULL.  The product g^T x is formed tile by tile on the tensor cores (bf16 operands as given,
+ *   fp32 accumulation) when m and n are multiples of 8, else on the CUDA cores; the level multiply
+ *   and the contractions with A and B are fp32 on the CUDA cores.  Every element is summed in a
+ *   fixed order (runs are bit-identical).  The tiles' contributions go through the lords_init
+ *   workspace; without room there a slower schedule without scratch memory runs.
+ *   x: device, bf16 [M][n].  Any bits in {2,3,4}, r <= LORDS_R_MAX.
  * All enqueue on `stream` and return without synchronising; all need lords_init.
  */
 int lords_transpose_codes(const uint8_t *Qpacked, int bits, int m, int n, uint8_t *Qt_packed, void *stream);
