@@ -690,7 +690,7 @@ template <int BITS, int NTOK, int H> int choose_cluster(int dev, int tiles, int 
 
 template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem &p, const State &st, cudaStream_t stream)
 {
-    const int dev = device_slot(st), forced_cs = st.forced_splitk, forced_halves = 0;
+    const int dev = device_slot(st), forced_cs = st.forced_splitk;
     const int qrow = DCfg<BITS, 1>::QROW;
     k.ksteps = (p.n + kStep - 1) / kStep;
     int rc = DecodeVariant<BITS, NTOK, 1>::prepare(dev);
@@ -701,7 +701,7 @@ template <int BITS, int NTOK> int launch_bits_tok(DecodeParams &k, const Problem
     double cost1 = 0, cost2 = 0;
     const int cs1 = choose_cluster<BITS, NTOK, 1>(dev, tiles1, k.ksteps, forced_cs, cost1);
     const int cs2 = choose_cluster<BITS, NTOK, 2>(dev, tiles2, k.ksteps, forced_cs, cost2);
-    const bool two = forced_halves > 0 ? forced_halves == 2 : cost2 < cost1;
+    const bool two = cost2 < cost1;
     const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
     if (!make_map_2d(&k.tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, p.q, row_bytes, (uint64_t)p.m, (uint32_t)qrow,
                      two ? 256u : 128u, BITS == 4 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE) ||
