@@ -30,6 +30,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <type_traits>
+
 #include "lords_internal.h"
 #include "lords_ptx.cuh"
 #include "lords_tc_common.cuh"
@@ -421,20 +423,49 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
         // every MMA has completed (the accumulator barrier), so every stage has been read: the stages'
         // memory now holds the dS tile and the factor slices
         const size_t row_bytes = (size_t)p.b.n * p.b.bits / 8;
+        const int jc = j0 + ch * 32, bits = p.b.bits;
+        // the thread's 32 codes are `bits` consecutive 32-bit words of its row when the group lies
+        // inside the row and the row pitch keeps it word-aligned; otherwise code by code
+        const bool whole = ok && i < p.b.m && jc + 32 <= p.b.n && (row_bytes & 3) == 0;
+        uint32_t cw[5] = {0u, 0u, 0u, 0u, 0u};
+        if (whole) {
+            const uint32_t *src = reinterpret_cast<const uint32_t *>(p.b.q + (size_t)i * row_bytes + (size_t)jc * bits / 8);
 #pragma unroll
-        for (int cidx = 0; cidx < 32; ++cidx) {
-            const int j = j0 + ch * 32 + cidx;
-            float v = 0.0f;
-            if (ok && i < p.b.m && j < p.b.n) v = __uint_as_float(gacc[cidx]) * p.b.levels[read_code(p.b.q, row_bytes, i, j, p.b.bits)];
-            ds[ri][ch * 32 + cidx] = v;
+            for (int w = 0; w < 4; ++w)
+                if (w < bits) cw[w] = __ldg(src + w);
+        }
+        if (whole) {
+            // the positions of the codes inside the words are compile-time constants for each width
+            auto levels_of = [&](auto width) {
+                constexpr int W = decltype(width)::value;
+#pragma unroll
+                for (int cidx = 0; cidx < 32; ++cidx) {
+                    constexpr uint32_t mask = (1u << W) - 1u;
+                    const int bit = cidx * W, w = bit >> 5, sh = bit & 31;
+                    uint32_t code = cw[w] >> sh;
+                    if (sh + W > 32) code |= cw[w + 1] << (32 - sh);
+                    ds[ri][ch * 32 + cidx] = __uint_as_float(gacc[cidx]) * p.b.levels[code & mask];
+                }
+            };
+            if (bits == 4) levels_of(std::integral_constant<int, 4>{});
+            else if (bits == 3) levels_of(std::integral_constant<int, 3>{});
+            else levels_of(std::integral_constant<int, 2>{});
+        } else {
+#pragma unroll
+            for (int cidx = 0; cidx < 32; ++cidx) {
+                const int j = jc + cidx;
+                float v = 0.0f;
+                if (ok && i < p.b.m && j < p.b.n) v = __uint_as_float(gacc[cidx]) * p.b.levels[read_code(p.b.q, row_bytes, i, j, bits)];
+                ds[ri][ch * 32 + cidx] = v;
+            }
         }
         const int et = tid;                                       // 0 .. 255
         for (int e = et; e < r4 * kTcCols; e += 256) {            // A[k][j0 ..]
             const int k = e / kTcCols, cidx = e % kTcCols;
             fa[k][cidx] = (k < p.b.r && j0 + cidx < p.b.n) ? p.b.A[(size_t)k * p.b.n + j0 + cidx] : (uint16_t)0;
         }
-        for (int e = et; e < r4 * kTcRows; e += 256) {            // B[i0 ..][k] stored [k][i]
-            const int k = e / kTcRows, cidx = e % kTcRows;
+        for (int e = et; e < r4 * kTcRows; e += 256) {            // B[i0 ..][k] stored [k][i]; neighbouring threads read one row of B
+            const int cidx = e / r4, k = e % r4;
             fb[k][cidx] = (k < p.b.r && i0 + cidx < p.b.m) ? p.b.B[(size_t)(i0 + cidx) * p.b.r + k] : (uint16_t)0;
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
