@@ -329,7 +329,7 @@ __host__ __device__ constexpr int bw_tc_smem(int r4)
 {
     // the epilogue's buffers (dS tile, the two factor slices) reuse the stages once the MMAs are done
     const int stages = kTcStages * kTcStage;
-    const int epi = kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 2 + r4 * (kTcRows + 2) * 2;
+    const int epi = kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 4 + r4 * (kTcRows + 2) * 4;
     return 1024 + (stages > epi ? stages : epi) + 256;
 }
 
@@ -340,7 +340,7 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
     uint8_t *base_ptr = tc_smem_raw + (base - smem_u32(tc_smem_raw));
     const int r4 = (p.b.r + 3) & ~3;
     const int stages_bytes = kTcStages * kTcStage;
-    const int epi_bytes = kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 2 + r4 * (kTcRows + 2) * 2;
+    const int epi_bytes = kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 4 + r4 * (kTcRows + 2) * 4;
     const uint32_t bars = base + (uint32_t)(stages_bytes > epi_bytes ? stages_bytes : epi_bytes);
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kTcStages, bar_acc = bar_empty + 8 * kTcStages;
     const uint32_t tmem_slot = bar_acc + 8;
@@ -406,12 +406,12 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
         // ---- epilogue: thread = (row quadrant q, column half ch): row i0 + q * 32 + lane, 32 columns
         const int q = warp & 3, ch = warp >> 2;
         const int ri = q * 32 + lane, i = i0 + ri;
-        // rows of the dS tile are 66 floats apart (pairs of columns are read as one 8-byte word), rows
-        // of the factor slices 33 and 65 words (neighbouring ranks fall into different banks)
+        // rows of the dS tile and of the factor slices (widened to fp32) are an even number of floats
+        // apart: pairs of neighbouring values are read as one 8-byte word
         float (*ds)[kTcCols + 2] = reinterpret_cast<float (*)[kTcCols + 2]>(base_ptr);
-        uint16_t (*fa)[kTcCols + 2] = reinterpret_cast<uint16_t (*)[kTcCols + 2]>(base_ptr + kTcRows * (kTcCols + 2) * 4);
-        uint16_t (*fb)[kTcRows + 2] =
-            reinterpret_cast<uint16_t (*)[kTcRows + 2]>(base_ptr + kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 2);
+        float (*fa)[kTcCols + 2] = reinterpret_cast<float (*)[kTcCols + 2]>(base_ptr + kTcRows * (kTcCols + 2) * 4);
+        float (*fb)[kTcRows + 2] =
+            reinterpret_cast<float (*)[kTcRows + 2]>(base_ptr + kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 4);
         const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, 0, status, 43));
         if (!ok) failed = true;
         tc_fence_after_sync();
@@ -462,15 +462,14 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
         const int et = tid;                                       // 0 .. 255
         for (int e = et; e < r4 * kTcCols; e += 256) {            // A[k][j0 ..]
             const int k = e / kTcCols, cidx = e % kTcCols;
-            fa[k][cidx] = (k < p.b.r && j0 + cidx < p.b.n) ? p.b.A[(size_t)k * p.b.n + j0 + cidx] : (uint16_t)0;
+            fa[k][cidx] = (k < p.b.r && j0 + cidx < p.b.n) ? bf16f(p.b.A[(size_t)k * p.b.n + j0 + cidx]) : 0.0f;
         }
         for (int e = et; e < r4 * kTcRows; e += 256) {            // B[i0 ..][k] stored [k][i]; neighbouring threads read one row of B
             const int cidx = e / r4, k = e % r4;
-            fb[k][cidx] = (k < p.b.r && i0 + cidx < p.b.m) ? p.b.B[(size_t)(i0 + cidx) * p.b.r + k] : (uint16_t)0;
+            fb[k][cidx] = (k < p.b.r && i0 + cidx < p.b.m) ? bf16f(p.b.B[(size_t)(i0 + cidx) * p.b.r + k]) : 0.0f;
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
-        // The folds, four ranks per thread so that a value of dS is read once for four products; the
-        // factors are read as pairs of bf16.  Each output is one thread's sum in index order.
+        // The folds, four ranks per thread so that a value of dS is read once for four products.  Each output is one thread's sum in index order.
         if (p.part_dB) {
             float *out = p.part_dB + ((size_t)jt * p.b.m + i0) * r4;
             for (int u = et; u < (r4 / 4) * kTcRows; u += 256) {          // dB[ii][k0 .. k0 + 3] = sum_j dS[ii][j] A[k][j]
@@ -481,9 +480,9 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
                     const float2 d = *reinterpret_cast<const float2 *>(&ds[ii][2 * jp]);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        const uint32_t w = *reinterpret_cast<const uint32_t *>(&fa[k0 + kk][2 * jp]);
-                        acc[kk] = fmaf(d.x, __uint_as_float(w << 16), acc[kk]);
-                        acc[kk] = fmaf(d.y, __uint_as_float(w & 0xFFFF0000u), acc[kk]);
+                        const float2 w = *reinterpret_cast<const float2 *>(&fa[k0 + kk][2 * jp]);
+                        acc[kk] = fmaf(d.x, w.x, acc[kk]);
+                        acc[kk] = fmaf(d.y, w.y, acc[kk]);
                     }
                 }
                 if (i0 + ii < p.b.m)
@@ -500,9 +499,9 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
                     const float d0 = ds[2 * ip][j], d1 = ds[2 * ip + 1][j];
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        const uint32_t w = *reinterpret_cast<const uint32_t *>(&fb[k0 + kk][2 * ip]);
-                        acc[kk] = fmaf(__uint_as_float(w << 16), d0, acc[kk]);
-                        acc[kk] = fmaf(__uint_as_float(w & 0xFFFF0000u), d1, acc[kk]);
+                        const float2 w = *reinterpret_cast<const float2 *>(&fb[k0 + kk][2 * ip]);
+                        acc[kk] = fmaf(w.x, d0, acc[kk]);
+                        acc[kk] = fmaf(w.y, d1, acc[kk]);
                     }
                 }
                 if (j0 + j < p.b.n)
