@@ -11,11 +11,10 @@
 // forward kernels as they are.  This file holds what that needs -- the transposition of packed codes
 // and of a bf16 matrix -- and the kernels for dB and dA.
 //
-// dB and dA run on the CUDA cores in fp32 (bf16 inputs are widened exactly).  A 64 x 64 tile of dS is
-// formed by a shared-memory-tiled product g^T x over the tokens, multiplied by the levels of the
-// tile's codes, and folded with the matching 64-column slice of A (for dB) and 64-row slice of B (for
-// dA).  Two schedules:
-//   tiles: one CTA per tile of W; it writes the tile's contributions to dB and dA into the library's
+// dB and dA: a tile of dS is formed by the product g^T x over the tokens, multiplied by the levels of
+// the tile's codes, and folded with the matching column slice of A (for dB) and row slice of B (for
+// dA); bf16 inputs are widened exactly, sums are fp32.  Three schedules:
+//   tiles: one CTA per 64 x 64 tile of W, everything on the CUDA cores; it writes the tile's contributions to dB and dA into the library's
 //          workspace, and a second kernel adds the contributions of a row (or column) of tiles in tile
 //          order.  g^T x is formed once, and the grid fills the machine.  Taken when the workspace
 //          holds the contributions (4 r (m n / 64 + n m / 64) bytes).
