@@ -836,10 +836,12 @@ def main():
             k = {"decode_q_m8": 400, "mlp3_gate_m1": 800, "mlp3_down_m1": 800, "mlp3_down_m16": 300,
                  "prefill_m2048": 60}.get(name, 20)
             k = max(3, min(args.steps, k))
-            r2 = time_case(name, k, 3, device, rank, world, None, do_e2e=False, min_seconds=0.4)
+            # every case has its clocks sampled while it is timed (the prefill case runs under the power cap)
+            r2 = time_case(name, k, 3, device, rank, world, ClockSampler(local) if rank == 0 else None, do_e2e=False,
+                           min_seconds=0.4)
             r2.pop("_lay")
             cases.append({"case": name, "path": r2["path"], "us_per_call": r2["us_per_call"],
-                          "gbs": r2["gbs"], "tflops": r2["tflops"], "roofline": r2["roofline"],
+                          "gbs": r2["gbs"], "tflops": r2["tflops"], "roofline": r2["roofline"], "clocks": r2["clocks"],
                           "copies": r2["copies"], "rounds": r2["rounds"], "steps": k, "status_retries": r2["status_retries"]})
 
     if not args.case and not args.no_extras and world == 1:
