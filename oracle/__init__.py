@@ -52,6 +52,8 @@ def _load():
         lib.lords_oracle_quantize.argtypes = [p, p, p, p, ci, i64, i64, i64, p, p, p, p]
         lib.lords_oracle_backward.restype = ci
         lib.lords_oracle_backward.argtypes = [p, p, p, p, p, p, ci, i64, i64, i64, i64, p, p, p]
+        lib.lords_oracle_backward_qat.restype = ci
+        lib.lords_oracle_backward_qat.argtypes = [p, p, p, p, p, p, p, ci, i64, i64, i64, i64, p, p, p]
         lib.lords_oracle_equivalent_rank.restype = i64
         lib.lords_oracle_equivalent_rank.argtypes = [i64, i64, i64]
         _lib = lib
@@ -185,6 +187,26 @@ def backward(g, x, qpacked, B, A, codebook, bits: int):
     if rc != 0:
         raise ValueError(f"oracle backward failed: {rc}")
     return dx, dB, dA
+
+
+def backward_qat(g, x, W, qpacked, B, A, codebook, bits: int):
+    """Straight-through gradients of quantisation-aware training (Eq. 4-5): (dW [m, n], dB [m, r], dA [r, n]), fp64.
+
+    dW = g^T x (Eq. 4); dS = dW * (L[Q] - W / S) (Eq. 5), zero where S is zero; dB = dS A^T, dA = B^T dS."""
+    g = _c(g, np.uint16); x = _c(x, np.uint16); W = _c(W, np.uint16); B = _c(B, np.uint16); A = _c(A, np.uint16)
+    qpacked = _c(qpacked, np.uint8); codebook = _c(codebook, np.float32)
+    M, n = x.shape
+    m, r = B.shape
+    assert g.shape == (M, m) and W.shape == (m, n) and A.shape == (r, n) and codebook.size == 2**bits
+    assert qpacked.size == packed_bytes(m, n, bits)
+    dW = np.empty((m, n), dtype=np.float64)
+    dB = np.empty((m, r), dtype=np.float64)
+    dA = np.empty((r, n), dtype=np.float64)
+    rc = _load().lords_oracle_backward_qat(_ptr(g), _ptr(x), _ptr(W), _ptr(qpacked), _ptr(B), _ptr(A), _ptr(codebook), bits,
+                                           M, m, n, r, _ptr(dW), _ptr(dB), _ptr(dA))
+    if rc != 0:
+        raise ValueError(f"oracle QAT backward failed: {rc}")
+    return dW, dB, dA
 
 
 def adapter_forward(x, qpacked, s, blk: int, A_l, B_l, codebook, bits: int) -> np.ndarray:

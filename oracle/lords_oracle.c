@@ -41,6 +41,12 @@
  * the tests take such differences on sampled entries, and check <g, y> identities that follow from
  * linearity (sum(dx (.) x) = sum(dB (.) B) = sum(dA (.) A) = sum(g (.) y)).
  *
+ * The gradients of quantisation-aware training with the straight-through estimator (Eq. 4-5) are in
+ * lords_oracle_backward_qat.  Pins: dL/dW against a library matmul; a weight that its codes represent
+ * exactly (W = L[Q] (.) S) has Q - W (/) S = 0, so dB = dA = 0; dL/dS differs from the fine-tuning
+ * case above only by the term -dL/dW^ (.) (W (/) S), checked with the pinned fine-tuning gradients
+ * and an array-wise quotient; linearity in g.
+ *
  * The step before the path, the quantisation step of Alg. 1 (step 2.1), is stated here too
  * (lords_oracle_quantize): Q_ij = argmin over the levels v of (S_ij v - W_ij)^2 with S = BA, every
  * level tried in turn in fp64.  The paper does not say which level wins a tie: the lowest code does.
@@ -350,6 +356,58 @@ int lords_oracle_backward(const uint16_t *g, const uint16_t *x, const uint8_t *q
             }
         if (dA)
             for (int64_t k = 0; k < r; ++k) {                                   /* dA_kj += B_ik dS_ij */
+                double b = bf16_to_f64(B[i * r + k]);
+                for (int64_t j = 0; j < n; ++j) dA[k * n + j] += b * dS_row[j];
+            }
+    }
+    free(S_row);
+    free(dS_row);
+    return ORACLE_OK;
+}
+
+/*
+ * Backward of quantisation-aware training (Sec. 3.3, Eq. 4-5): the fake-quantised weight is
+ * W^ = Round(W (/) S) (.) S with S = B A, and with the straight-through estimator
+ *     dL/dW = dL/dW^                                  (Eq. 4)
+ *     dL/dS = dL/dW^ (.) (Q - W (/) S)                (Eq. 5),   Q = Round(W (/) S) = the level L[code]
+ * and then dB = dL/dS A^T, dA = B^T dL/dS as for any function of S = B A.  Here dL/dW^ = g^T x for
+ * the layer y = x W^T, the codes are the given ones (the rounding has been done), and an element
+ * whose S is exactly zero, where the quotient is undefined, gets dL/dS = 0.
+ *   W   : bf16 [m][n], the latent full-precision weight
+ *   dW  : m x n doubles (may be NULL), dB : m x r (may be NULL), dA : r x n (may be NULL)
+ */
+int lords_oracle_backward_qat(const uint16_t *g, const uint16_t *x, const uint16_t *W, const uint8_t *qpacked,
+                              const uint16_t *B, const uint16_t *A, const float *codebook, int bits, int64_t M,
+                              int64_t m, int64_t n, int64_t r, double *dW, double *dB, double *dA)
+{
+    if (!g || !x || !W || !qpacked || !B || !A || !codebook || M < 1 || m < 1 || n < 1 || r < 1 || !group_ok(n, bits))
+        return ORACLE_ERR_ARG;
+    int64_t row_bytes = n * bits / 8;
+    double *S_row = (double *)malloc(sizeof(double) * (size_t)n);
+    double *dS_row = (double *)malloc(sizeof(double) * (size_t)n);
+    if (!S_row || !dS_row) {
+        free(S_row); free(dS_row);
+        return ORACLE_ERR_NOMEM;
+    }
+    if (dA) for (int64_t e = 0; e < r * n; ++e) dA[e] = 0.0;
+    for (int64_t i = 0; i < m; ++i) {
+        const uint8_t *qrow = qpacked + i * row_bytes;
+        scale_row(B, A, n, r, i, S_row);
+        for (int64_t j = 0; j < n; ++j) {
+            double dWhat = 0.0;                                                 /* dL/dW^_ij = sum_t g_ti x_tj */
+            for (int64_t t = 0; t < M; ++t) dWhat += bf16_to_f64(g[t * m + i]) * bf16_to_f64(x[t * n + j]);
+            if (dW) dW[i * n + j] = dWhat;                                      /* Eq. 4 */
+            double level = (double)codebook[read_code(qrow, j, bits)];
+            dS_row[j] = S_row[j] != 0.0 ? dWhat * (level - bf16_to_f64(W[i * n + j]) / S_row[j]) : 0.0;   /* Eq. 5 */
+        }
+        if (dB)
+            for (int64_t k = 0; k < r; ++k) {
+                double acc = 0.0;
+                for (int64_t j = 0; j < n; ++j) acc += dS_row[j] * bf16_to_f64(A[k * n + j]);
+                dB[i * r + k] = acc;
+            }
+        if (dA)
+            for (int64_t k = 0; k < r; ++k) {
                 double b = bf16_to_f64(B[i * r + k]);
                 for (int64_t j = 0; j < n; ++j) dA[k * n + j] += b * dS_row[j];
             }

@@ -404,3 +404,55 @@ def test_adapter_comparator_against_brute_force():
     zero = np.zeros_like(Al)
     assert np.array_equal(oracle.adapter_forward(lay.x, qp, s, blk, zero, Bl, lay.codebook, bits),
                           oracle.forward(lay.x, qp, lay.B, lay.A, lay.codebook, bits))
+
+
+# ---- straight-through gradients of quantisation-aware training (Eq. 4-5) --------------------------------
+
+def test_qat_backward_pins():
+    import torch
+    m, n, r, M, bits = 24, 64, 5, 3, 4
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=31, mixed_sign=True)
+    packed = oracle.pack_codes(lay.codes, bits)
+    g = gen.make_layer(m, 64, 1, M, bits=4, seed=6).x[:, :m].copy()
+    Wb = gen.make_weight(m, n, seed=7, sigma=0.02)
+    dW, dB, dA = oracle.backward_qat(g, lay.x, Wb, packed, lay.B, lay.A, lay.codebook, bits)
+    gf, xf, Wf, Bf, Af = _f64(g), _f64(lay.x), _f64(Wb), _f64(lay.B), _f64(lay.A)
+    # Eq. 4: dL/dW is dL/dW^ = g^T x, a library matmul
+    assert np.allclose(dW, gf.T @ xf, rtol=1e-13, atol=1e-13)
+    # Eq. 5 against the fine-tuning gradients (pinned above): dS_qat = dS_peft - dW^ (.) (W / S)
+    _, dB_p, dA_p = oracle.backward(g, lay.x, packed, lay.B, lay.A, lay.codebook, bits)
+    S = Bf @ Af
+    assert (S != 0).all()
+    extra = dW * (Wf / S)
+    assert np.allclose(dB, dB_p - extra @ Af.T, rtol=1e-10, atol=1e-10 * np.abs(dB_p).max())
+    assert np.allclose(dA, dA_p - Bf.T @ extra, rtol=1e-10, atol=1e-10 * np.abs(dA_p).max())
+    # a weight that its codes represent exactly has Q - W / S = 0: no gradient reaches S
+    What = oracle.dequant_rows(packed, lay.B, lay.A, lay.codebook, bits)
+    Wexact = gen.bf16_bits(torch.from_numpy(What.astype(np.float32)))
+    if np.array_equal(gen.bf16_to_f32(Wexact).astype(np.float64), What):     # only when W^ is bf16-representable
+        _, dB0, dA0 = oracle.backward_qat(g, lay.x, Wexact, packed, lay.B, lay.A, lay.codebook, bits)
+        assert np.abs(dB0).max() <= 1e-12 and np.abs(dA0).max() <= 1e-12
+    # linear in g
+    g2 = gen.make_layer(m, 64, 1, M, bits=4, seed=8).x[:, :m].copy()
+    gsum = gen.bf16_bits(torch.from_numpy((gen.bf16_to_f32(g) * 2.0).astype(np.float32)))      # 2 g is exact in bf16
+    dW2, dB2, dA2 = oracle.backward_qat(gsum, lay.x, Wb, packed, lay.B, lay.A, lay.codebook, bits)
+    assert np.allclose(dW2, 2 * dW, rtol=1e-13) and np.allclose(dB2, 2 * dB, rtol=1e-12, atol=1e-15) and np.allclose(dA2, 2 * dA, rtol=1e-12, atol=1e-15)
+    del g2
+
+
+def test_qat_backward_exactly_representable_weight_and_zero_scale():
+    """Integers: W = L[Q] * S exactly, so dB = dA = 0; rows with S = 0 contribute nothing either."""
+    import torch
+    lay = gen.make_integer_layer(32, 64, 4, 2, bits=4, seed=3)
+    packed = oracle.pack_codes(lay.codes, 4)
+    S = _f64(lay.B) @ _f64(lay.A)
+    W = lay.codebook.astype(np.float64)[lay.codes] * S
+    Bz = lay.B.copy(); Bz[::5, :] = 0                       # S = 0 in every fifth row
+    Wb = gen.bf16_bits(torch.from_numpy(W.astype(np.float32)))
+    g = gen.bf16_bits(torch.randint(-2, 3, (2, 32), generator=torch.Generator().manual_seed(1)).float())
+    dW, dB, dA = oracle.backward_qat(g, lay.x, Wb, packed, lay.B, lay.A, lay.codebook, 4)
+    assert np.array_equal(dB, np.zeros_like(dB)) and np.array_equal(dA, np.zeros_like(dA))
+    assert np.array_equal(dW, _f64(g).T @ _f64(lay.x))
+    dWz, dBz, dAz = oracle.backward_qat(g, lay.x, Wb, packed, Bz, lay.A, lay.codebook, 4)
+    assert np.isfinite(dBz).all() and np.isfinite(dAz).all()
+    assert np.array_equal(dBz[::5], np.zeros_like(dBz[::5]))
