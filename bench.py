@@ -552,6 +552,10 @@ def time_backward(name, m, n, r, bits, M, device, min_seconds=0.3):
 
     us_dx, path_dx, reps_dx = timed(lambda: lords.lords_linear_backward_input(g, qt, B, A, lay.codebook, bits, M, m, n, r, dx))
     us_f, path_f, reps_f = timed(lambda: lords.lords_linear_backward_factors(g, x, q, B, A, lay.codebook, bits, M, m, n, r, dB, dA))
+    # the straight-through gradients of quantisation-aware training (Eq. 4-5) on the same layer: dW, dB, dA
+    Wd = torch.from_numpy(gen.make_weight(m, n, seed=2).view(np.int16)).to(device)
+    dW = torch.zeros((m, n), dtype=torch.float32, device=device)
+    us_q, path_q, _ = timed(lambda: lords.lords_linear_backward_qat(g, x, Wd, q, B, A, lay.codebook, bits, M, m, n, r, dW, dB, dA))
     status = lords.lords_poll_status()
     peaks = measured_peaks()
     flops = 2.0 * M * m * n
@@ -568,6 +572,7 @@ def time_backward(name, m, n, r, bits, M, device, min_seconds=0.3):
             "factor_gradients": {"us": us_f, "path": path_f, "alu_tflops": tf_f,
                                  "tile_product_tflops": flops / (us_f * 1e-6) / 1e12,
                                  "tile_product_on": "tensor cores" if path_f == "backward_tensor" else "CUDA cores"},
+            "qat_gradients": {"us": us_q, "path": path_q},
             "roofline": {"bound": "alu", "achieved": tf_f, "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s",
                          "frac": tf_f / FP32_ALU_TFLOPS, "peak_source": "148 SMs x 128 fp32 lanes x 2 flops x 1.965 GHz",
                          "traffic": NCU_TRAFFIC_BYTES.get(name), "us_per_launch": us_f}}

@@ -214,6 +214,23 @@ int lords_linear_backward_factors(const void *dy, const void *x, const uint8_t *
                                   void *stream);
 
 /*
+ * Gradients of quantisation-aware training with the straight-through estimator (Sec. 3.3, Eq. 4-5):
+ * the fake-quantised weight is W^ = Round(W (/) S) (.) S, S = B A, the codes are those of the current
+ * rounding (lords_quantize_codes), and with g = dL/dy
+ *     dL/dW = dL/dW^ = g^T x                              (Eq. 4),
+ *     dL/dS = dL/dW^ (.) (L[Q] - W (/) S)                  (Eq. 5; 0 where S is exactly 0),
+ *     dB = dL/dS A^T,   dA = B^T dL/dS.
+ *   W  : device, bf16 [m][n], the latent full-precision weight
+ *   dW : device, float [m][n] or NULL;  dB : device, float [m][r] or NULL;  dA : device, float [r][n] or NULL
+ * Runs on the tensor-core schedule of lords_linear_backward_factors only: m and n multiples of 8 and
+ * room in the lords_init workspace for the tiles' contributions, else LORDS_ERR_UNSUPPORTED.  The
+ * quotient and S are formed in fp32.  Enqueues on `stream` and returns without synchronising.
+ */
+int lords_linear_backward_qat(const void *dy, const void *x, const void *W, const uint8_t *Qpacked, const void *B, const void *A,
+                              const float *codebook, int bits, int M, int m, int n, int r, float *dW, float *dB, float *dA,
+                              void *stream);
+
+/*
  * Comparators for the paper's efficiency claims (Sec. 4.4, Table 6), on the same GPU and the same packed
  * codes: a block-scaled layer (Eq. 2), and that layer with an additive low-rank adapter that cannot be
  * merged into the quantised weights (Sec. 3.4).

@@ -53,6 +53,7 @@ def _load():
         "lords_linear_backward_input": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_backward_input_f32": (ci, [p, p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_linear_backward_factors": (ci, [p, p, p, p, p, p, ci, ci, ci, ci, ci, p, p, p]),
+        "lords_linear_backward_qat": (ci, [p, p, p, p, p, p, p, ci, ci, ci, ci, ci, p, p, p, p]),
         "lords_blockscale_forward": (ci, [p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_blockscale_forward_f32": (ci, [p, p, p, p, ci, ci, ci, ci, ci, p, p]),
         "lords_adapter_forward": (ci, [p, p, p, p, p, p, ci, ci, ci, ci, ci, ci, p, p]),
@@ -83,7 +84,7 @@ def exported_symbols():
             "lords_linear_forward", "lords_linear_forward_bits", "lords_linear_forward_f32",
             "lords_linear_forward_host", "lords_linear_forward_noalloc", "lords_quantize_codes", "lords_transpose_codes",
             "lords_linear_backward_input", "lords_linear_backward_input_f32", "lords_linear_backward_factors",
-            "lords_blockscale_forward", "lords_blockscale_forward_f32", "lords_adapter_forward", "lords_adapter_forward_f32", "lords_poll_status", "lords_read_status_detail", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
+            "lords_linear_backward_qat", "lords_blockscale_forward", "lords_blockscale_forward_f32", "lords_adapter_forward", "lords_adapter_forward_f32", "lords_poll_status", "lords_read_status_detail", "lords_last_cuda_error", "lords_set_option", "lords_last_path",
             "lords_last_launch_count"]
 
 
@@ -231,6 +232,15 @@ def lords_linear_backward_factors(dy, x, Qpacked, B, A, codebook, bits, M, m, n,
                                                  cb.ctypes.data, bits, M, m, n, r,
                                                  None if dB is None else dB.data_ptr(), None if dA is None else dA.data_ptr(),
                                                  _stream_ptr(stream)), "lords_linear_backward_factors")
+
+
+def lords_linear_backward_qat(dy, x, W, Qpacked, B, A, codebook, bits, M, m, n, r, dW, dB, dA, stream=None) -> None:
+    """Straight-through gradients of quantisation-aware training (Eq. 4-5); any of dW, dB, dA may be None."""
+    cb = _cb_ptr(codebook, bits)
+    ptr = lambda t: None if t is None else t.data_ptr()
+    _check(_load().lords_linear_backward_qat(dy.data_ptr(), x.data_ptr(), W.data_ptr(), Qpacked.data_ptr(), B.data_ptr(),
+                                             A.data_ptr(), cb.ctypes.data, bits, M, m, n, r, ptr(dW), ptr(dB), ptr(dA),
+                                             _stream_ptr(stream)), "lords_linear_backward_qat")
 
 
 def lords_blockscale_forward(x, Qpacked, scales, codebook, bits, blk, M, m, n, y, stream=None, f32=False) -> None:

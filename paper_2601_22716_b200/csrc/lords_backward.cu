@@ -322,6 +322,9 @@ struct alignas(64) BwTcParams {
     float *part_dB;       // [n / 64 tiles][m][r4]
     float *part_dA;       // [m / 128 tiles][r4][n]
     int *status;
+    // quantisation-aware training (Eq. 4-5): the latent weight and, optionally, where dL/dW goes
+    const uint16_t *W;    // bf16 [m][n]
+    float *dW;            // float [m][n] or null
 };
 
 __host__ __device__ constexpr int bw_tc_smem(int r4)
@@ -332,6 +335,9 @@ __host__ __device__ constexpr int bw_tc_smem(int r4)
     return 1024 + (stages > epi ? stages : epi) + 256;
 }
 
+// QAT: the tile of g^T x is dL/dW^ itself (Eq. 4: stored as dL/dW if asked for), and the factor of
+// dL/dS is Q - W (/) S instead of Q (Eq. 5), with S = B A rebuilt per element from the factor slices.
+template <bool QAT>
 __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __grid_constant__ BwTcParams p)
 {
     extern __shared__ uint8_t tc_smem_raw[];
@@ -420,7 +426,19 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
             tmem_wait_ld();
         }
         // every MMA has completed (the accumulator barrier), so every stage has been read: the stages'
-        // memory now holds the dS tile and the factor slices
+        // memory now holds the factor slices and the dS tile
+        const int et = tid;                                       // 0 .. 255
+        auto load_slices = [&]() {
+            for (int e = et; e < r4 * kTcCols; e += 256) {            // A[k][j0 ..]
+                const int k = e / kTcCols, cidx = e % kTcCols;
+                fa[k][cidx] = (k < p.b.r && j0 + cidx < p.b.n) ? bf16f(p.b.A[(size_t)k * p.b.n + j0 + cidx]) : 0.0f;
+            }
+            for (int e = et; e < r4 * kTcRows; e += 256) {            // B[i0 ..][k] stored [k][i]; neighbouring threads read one row of B
+                const int cidx = e / r4, k = e % r4;
+                fb[k][cidx] = (k < p.b.r && i0 + cidx < p.b.m) ? bf16f(p.b.B[(size_t)(i0 + cidx) * p.b.r + k]) : 0.0f;
+            }
+        };
+        if constexpr (QAT) load_slices();                         // S is rebuilt from them below
         const size_t row_bytes = (size_t)p.b.n * p.b.bits / 8;
         const int jc = j0 + ch * 32, bits = p.b.bits;
         // the thread's 32 codes are `bits` consecutive 32-bit words of its row when the group lies
@@ -433,6 +451,36 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
             for (int w = 0; w < 4; ++w)
                 if (w < bits) cw[w] = __ldg(src + w);
         }
+        // QAT: W / S per element (0 where S is 0, and the level is dropped there too: no gradient)
+        float quot[QAT ? 32 : 1];
+        bool live[QAT ? 32 : 1];
+        if constexpr (QAT) {
+            if (p.dW && ok && i < p.b.m) {                        // Eq. 4: dL/dW = dL/dW^
+#pragma unroll
+                for (int cidx = 0; cidx < 32; ++cidx)
+                    if (jc + cidx < p.b.n) p.dW[(size_t)i * p.b.n + jc + cidx] = __uint_as_float(gacc[cidx]);
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");        // the factor slices are in place
+            float sv[32];
+#pragma unroll
+            for (int cidx = 0; cidx < 32; ++cidx) sv[cidx] = 0.0f;
+            for (int k = 0; k < p.b.r; ++k) {
+                const float bk = fb[k][ri];
+#pragma unroll
+                for (int cidx = 0; cidx < 32; ++cidx) sv[cidx] = fmaf(bk, fa[k][ch * 32 + cidx], sv[cidx]);
+            }
+#pragma unroll
+            for (int cidx = 0; cidx < 32; ++cidx) {
+                const int j = jc + cidx;
+                const float w = (i < p.b.m && j < p.b.n) ? bf16f(p.W[(size_t)i * p.b.n + j]) : 0.0f;
+                live[cidx] = sv[cidx] != 0.0f;
+                quot[cidx] = live[cidx] ? w / sv[cidx] : 0.0f;
+            }
+        }
+        auto factor = [&](int cidx, float level) -> float {
+            if constexpr (QAT) return live[cidx] ? level - quot[cidx] : 0.0f;
+            else return level;
+        };
         if (whole) {
             // the positions of the codes inside the words are compile-time constants for each width
             auto levels_of = [&](auto width) {
@@ -443,7 +491,7 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
                     const int bit = cidx * W, w = bit >> 5, sh = bit & 31;
                     uint32_t code = cw[w] >> sh;
                     if (sh + W > 32) code |= cw[w + 1] << (32 - sh);
-                    ds[ri][ch * 32 + cidx] = __uint_as_float(gacc[cidx]) * p.b.levels[code & mask];
+                    ds[ri][ch * 32 + cidx] = __uint_as_float(gacc[cidx]) * factor(cidx, p.b.levels[code & mask]);
                 }
             };
             if (bits == 4) levels_of(std::integral_constant<int, 4>{});
@@ -454,19 +502,12 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
             for (int cidx = 0; cidx < 32; ++cidx) {
                 const int j = jc + cidx;
                 float v = 0.0f;
-                if (ok && i < p.b.m && j < p.b.n) v = __uint_as_float(gacc[cidx]) * p.b.levels[read_code(p.b.q, row_bytes, i, j, bits)];
+                if (ok && i < p.b.m && j < p.b.n)
+                    v = __uint_as_float(gacc[cidx]) * factor(cidx, p.b.levels[read_code(p.b.q, row_bytes, i, j, bits)]);
                 ds[ri][ch * 32 + cidx] = v;
             }
         }
-        const int et = tid;                                       // 0 .. 255
-        for (int e = et; e < r4 * kTcCols; e += 256) {            // A[k][j0 ..]
-            const int k = e / kTcCols, cidx = e % kTcCols;
-            fa[k][cidx] = (k < p.b.r && j0 + cidx < p.b.n) ? bf16f(p.b.A[(size_t)k * p.b.n + j0 + cidx]) : 0.0f;
-        }
-        for (int e = et; e < r4 * kTcRows; e += 256) {            // B[i0 ..][k] stored [k][i]; neighbouring threads read one row of B
-            const int cidx = e / r4, k = e % r4;
-            fb[k][cidx] = (k < p.b.r && i0 + cidx < p.b.m) ? bf16f(p.b.B[(size_t)(i0 + cidx) * p.b.r + k]) : 0.0f;
-        }
+        if constexpr (!QAT) load_slices();
         asm volatile("bar.sync 1, 256;" ::: "memory");
         // The folds, four ranks per thread so that a value of dS is read once for four products.  Each output is one thread's sum in index order.
         if (p.part_dB) {
@@ -552,6 +593,53 @@ int launch_transpose_bf16(const uint16_t *src, int rows, int cols, uint16_t *dst
     return LORDS_OK;
 }
 
+// The tensor schedule.  W != null: the gradients of quantisation-aware training (dW may be null).
+// LORDS_ERR_UNSUPPORTED when the shapes do not suit it or the workspace cannot hold the contributions.
+static int launch_backward_tc(const BwParams &p, const uint16_t *W, float *dW, State &st, cudaStream_t stream)
+{
+    const int m = p.m, n = p.n, r = p.r, M = p.M;
+    const int r4 = (r + 3) & ~3;
+    const int it_t = (m + kTcRows - 1) / kTcRows, jt_t = (n + kTcCols - 1) / kTcCols;
+    const size_t nb = p.dB ? (size_t)jt_t * m * r4 * sizeof(float) : 0, na = p.dA ? (size_t)it_t * r4 * n * sizeof(float) : 0;
+    if (m % 8 != 0 || n % 8 != 0 || it_t > 65535 || nb + na + 256 > st.workspace_bytes) return LORDS_ERR_UNSUPPORTED;
+    BwTcParams k;
+    k.b = p;
+    k.part_dB = p.dB ? reinterpret_cast<float *>(st.workspace) : nullptr;
+    k.part_dA = p.dA ? reinterpret_cast<float *>(st.workspace + ((nb + 255) & ~(size_t)255)) : nullptr;
+    k.status = st.status_word;
+    k.W = W; k.dW = dW;
+    if (!make_map_2d(&k.tm_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.g, (uint64_t)m, (uint64_t)M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&k.tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.x, (uint64_t)n, (uint64_t)M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B))
+        return LORDS_ERR_CUDA;
+    const int smem = bw_tc_smem(r4);
+    static bool attr_set[kMaxDevices] = {};
+    const int dev = device_slot(st);
+    if (!attr_set[dev]) {
+        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_backward_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bw_tc_smem(kRMaxBw)));
+        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_backward_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bw_tc_smem(kRMaxBw)));
+        attr_set[dev] = true;
+    }
+    if (W) lords_backward_tc_kernel<true><<<dim3((unsigned)jt_t, (unsigned)it_t), kTcThreads, smem, stream>>>(k);
+    else lords_backward_tc_kernel<false><<<dim3((unsigned)jt_t, (unsigned)it_t), kTcThreads, smem, stream>>>(k);
+    LORDS_CUDA_TRY(cudaGetLastError());
+    int launches = 1;
+    if (p.dB) {
+        const size_t total = (size_t)m * r;
+        lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(k.part_dB, p.dB, jt_t, (size_t)m * r4, m, r, r4);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        ++launches;
+    }
+    if (p.dA) {
+        const size_t total = (size_t)r * n;
+        lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(k.part_dA, p.dA, it_t, (size_t)r4 * n, r, n, n);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        ++launches;
+    }
+    st.last_launches = launches;
+    st.last_path = W ? "backward_qat_tensor" : "backward_tensor";
+    return LORDS_OK;
+}
+
 int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t *q, const uint16_t *B, const uint16_t *A,
                             const float *levels, int bits, int M, int m, int n, int r, float *dB, float *dA,
                             State &st, cudaStream_t stream)
@@ -567,44 +655,9 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
     const int r4 = (r + 3) & ~3, it_n = (m + kT - 1) / kT, jt_n = (n + kT - 1) / kT;
     const size_t need_b = dB ? (size_t)jt_n * m * r4 * sizeof(float) : 0, need_a = dA ? (size_t)it_n * r4 * n * sizeof(float) : 0;
     // schedule "tensor": the same with 128 x 64 tiles and the tile product on the tensor cores
-    {
-        const int it_t = (m + kTcRows - 1) / kTcRows, jt_t = (n + kTcCols - 1) / kTcCols;
-        const size_t nb = dB ? (size_t)jt_t * m * r4 * sizeof(float) : 0, na = dA ? (size_t)it_t * r4 * n * sizeof(float) : 0;
-        if (st.forced_path == 0 && m % 8 == 0 && n % 8 == 0 && it_t <= 65535 && nb + na + 256 <= st.workspace_bytes) {
-            BwTcParams k;
-            k.b = p;
-            k.part_dB = dB ? reinterpret_cast<float *>(st.workspace) : nullptr;
-            k.part_dA = dA ? reinterpret_cast<float *>(st.workspace + ((nb + 255) & ~(size_t)255)) : nullptr;
-            k.status = st.status_word;
-            if (!make_map_2d(&k.tm_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, g, (uint64_t)m, (uint64_t)M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
-                !make_map_2d(&k.tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, (uint64_t)n, (uint64_t)M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B))
-                return LORDS_ERR_CUDA;
-            const int smem = bw_tc_smem(r4);
-            static int attr_set[kMaxDevices] = {};
-            const int dev = device_slot(st);
-            if (attr_set[dev] < smem) {
-                LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_backward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bw_tc_smem(kRMaxBw)));
-                attr_set[dev] = bw_tc_smem(kRMaxBw);
-            }
-            lords_backward_tc_kernel<<<dim3((unsigned)jt_t, (unsigned)it_t), kTcThreads, smem, stream>>>(k);
-            LORDS_CUDA_TRY(cudaGetLastError());
-            ++launches;
-            if (dB) {
-                const size_t total = (size_t)m * r;
-                lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(k.part_dB, dB, jt_t, (size_t)m * r4, m, r, r4);
-                LORDS_CUDA_TRY(cudaGetLastError());
-                ++launches;
-            }
-            if (dA) {
-                const size_t total = (size_t)r * n;
-                lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(k.part_dA, dA, it_t, (size_t)r4 * n, r, n, n);
-                LORDS_CUDA_TRY(cudaGetLastError());
-                ++launches;
-            }
-            st.last_launches = launches;
-            st.last_path = "backward_tensor";
-            return LORDS_OK;
-        }
+    if (st.forced_path == 0) {
+        const int rc = launch_backward_tc(p, nullptr, nullptr, st, stream);
+        if (rc != LORDS_ERR_UNSUPPORTED) return rc;
     }
     if (it_n <= 65535 && need_b + need_a + 256 <= st.workspace_bytes && st.forced_path != 1) {
         float *part_b = dB ? reinterpret_cast<float *>(st.workspace) : nullptr;
@@ -641,6 +694,20 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
     st.last_launches = launches;
     st.last_path = "backward_walk";
     return LORDS_OK;
+}
+
+// Straight-through gradients of quantisation-aware training (Eq. 4-5): tensor schedule only.
+int launch_backward_qat(const uint16_t *g, const uint16_t *x, const uint16_t *W, const uint8_t *q, const uint16_t *B,
+                        const uint16_t *A, const float *levels, int bits, int M, int m, int n, int r, float *dW, float *dB,
+                        float *dA, State &st, cudaStream_t stream)
+{
+    if (r > kRMaxBw) return LORDS_ERR_SHAPE;
+    BwParams p;
+    p.g = g; p.x = x; p.q = q; p.B = B; p.A = A;
+    for (int c = 0; c < 16; ++c) p.levels[c] = c < (1 << bits) ? levels[c] : 0.0f;
+    p.bits = bits; p.M = M; p.m = m; p.n = n; p.r = r;
+    p.dB = dB; p.dA = dA;
+    return launch_backward_tc(p, W, dW, st, stream);
 }
 
 }  // namespace lords

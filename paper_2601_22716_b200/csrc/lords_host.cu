@@ -420,6 +420,22 @@ int lords_linear_backward_factors(const void *dy, const void *x, const uint8_t *
                                    n, r, dB, dA, st, static_cast<cudaStream_t>(stream));
 }
 
+int lords_linear_backward_qat(const void *dy, const void *x, const void *W, const uint8_t *Qpacked, const void *B, const void *A,
+                              const float *codebook, int bits, int M, int m, int n, int r, float *dW, float *dB, float *dA,
+                              void *stream)
+{
+    if (!dy || !x || !W || !Qpacked || !B || !A || !codebook || (!dW && !dB && !dA)) return LORDS_ERR_NULL;
+    const int g = pack_group(bits);
+    if (g == 0) return LORDS_ERR_BITS;
+    if (M < 1 || M > LORDS_M_MAX || m < 1 || n < 1 || n % g != 0 || r < 1 || r > LORDS_R_MAX) return LORDS_ERR_SHAPE;
+    if (!aligned16(dy) || !aligned16(x) || !aligned16(W) || (dW && !aligned16(dW))) return LORDS_ERR_ALIGN;
+    State &st = state();
+    if (!st.initialised) return LORDS_ERR_NOT_INIT;
+    return launch_backward_qat(static_cast<const uint16_t *>(dy), static_cast<const uint16_t *>(x), static_cast<const uint16_t *>(W),
+                               Qpacked, static_cast<const uint16_t *>(B), static_cast<const uint16_t *>(A), codebook, bits, M, m, n, r,
+                               dW, dB, dA, st, static_cast<cudaStream_t>(stream));
+}
+
 static int blockscale_common(const void *x, const uint8_t *q, const void *scales, const float *cb, int bits, int blk, int M,
                              int m, int n, void *y, int y_f32, void *stream)
 {

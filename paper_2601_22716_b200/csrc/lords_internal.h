@@ -83,6 +83,12 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
                             const float *levels, int bits, int M, int m, int n, int r, float *dB, float *dA,
                             State &st, cudaStream_t stream);
 
+// Straight-through gradients of quantisation-aware training (Eq. 4-5); LORDS_ERR_UNSUPPORTED outside the
+// rules of the tensor-core schedule.
+int launch_backward_qat(const uint16_t *g, const uint16_t *x, const uint16_t *W, const uint8_t *q, const uint16_t *B,
+                        const uint16_t *A, const float *levels, int bits, int M, int m, int n, int r, float *dW, float *dB,
+                        float *dA, State &st, cudaStream_t stream);
+
 // Comparators (Sec. 4.4, Table 6): the block-scale instantiation of the 16-token decode kernel (Eq. 2) and
 // the two extra launches of an additive low-rank adapter on top of it.
 int launch_blockscale16(const Problem &p, const uint16_t *scales, int blk, State &st, cudaStream_t stream);

@@ -167,3 +167,78 @@ def test_backward_factors_one_at_a_time_and_bad_arguments(lords):
     with pytest.raises(lords.LordsError) as ei:        # m = 127 is not a multiple of the 4-bit pack group
         lords.lords_transpose_codes(q, 4, 127, 128, torch.empty(128 * 64, dtype=torch.uint8, device="cuda:0"))
     assert ei.value.status == -2
+
+
+# ---- straight-through gradients of quantisation-aware training (Eq. 4-5) --------------------------------
+# dW is the tile product itself (fp32 accumulation of exactly widened bf16 products: as dB, dA above).  dS
+# carries the factor L[Q] - W / S with S (r products) and the quotient in fp32: its rounding error is a few
+# 2^-24 of the two terms, far below the fp32 summation error of the folds, so the same tolerances hold
+# (measured: 1e-7 to 3e-7 normwise).
+QAT_NORMWISE_TOL = FACTOR_NORMWISE_TOL
+QAT_ELEMENT_TOL = FACTOR_ELEMENT_TOL
+
+
+@pytest.mark.parametrize("bits,m,n,r,M,mixed", [(4, 512, 384, 32, 64, False), (3, 256, 544, 48, 8, True), (2, 320, 256, 6, 5, False),
+                                                (4, 136, 200, 12, 130, True)])
+def test_qat_backward_against_the_oracle(lords, bits, m, n, r, M, mixed):
+    import torch
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=m + 3 * n + r, mixed_sign=mixed)
+    Wb = gen.make_weight(m, n, seed=m + r, sigma=0.05 * (r / 32.0))
+    codes = oracle.quantize(Wb, lay.B, lay.A, lay.codebook, bits)      # the codes of the current rounding
+    packed = oracle.pack_codes(codes, bits)
+    g = _grad_out(M, m, n)
+    dW64, dB64, dA64 = oracle.backward_qat(g, lay.x, Wb, packed, lay.B, lay.A, lay.codebook, bits)
+    q = torch.from_numpy(packed).to("cuda:0")
+    dW = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda:0")
+    dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
+    dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
+    lords.lords_linear_backward_qat(_dev(g), _dev(lay.x), _dev(Wb), q, _dev(lay.B), _dev(lay.A), lay.codebook, bits,
+                                    M, m, n, r, dW, dB, dA)
+    assert lords.lords_last_path() == "backward_qat_tensor" and lords.lords_last_launch_count() == 3
+    torch.cuda.synchronize()
+    assert lords.lords_poll_status() == 0
+    nw, el = error_metrics(dW.cpu().numpy(), dW64)
+    assert nw <= FACTOR_NORMWISE_TOL and el <= FACTOR_ELEMENT_TOL, ("dW", nw, el)
+    for name, got, want in (("dB", dB.cpu().numpy(), dB64), ("dA", dA.cpu().numpy(), dA64)):
+        assert np.isfinite(got).all(), name
+        nw, el = error_metrics(got, want)
+        print(f"qat {name} bits={bits} m={m} n={n} r={r} M={M}: normwise={nw:.2e} element={el:.2e}")
+        assert nw <= QAT_NORMWISE_TOL and el <= QAT_ELEMENT_TOL, (name, nw, el)
+
+
+def test_qat_backward_exactly_representable_weight_is_exact(lords):
+    """Integers: W = L[Q] S exactly, so the factor L[Q] - W / S is exactly zero and no gradient reaches B or
+    A; rows whose S is zero contribute nothing; dW is the exact integer product."""
+    import torch
+    m, n, r, M = 256, 384, 8, 3
+    lay = gen.make_integer_layer(m, n, r, M, bits=4, seed=13)
+    Bz = lay.B.copy(); Bz[::9, :] = 0
+    S = gen.bf16_to_f32(Bz).astype(np.float64) @ gen.bf16_to_f32(lay.A).astype(np.float64)
+    W = lay.codebook.astype(np.float64)[lay.codes] * S
+    Wb = gen.bf16_bits(torch.from_numpy(W.astype(np.float32)))
+    assert np.array_equal(gen.bf16_to_f32(Wb).astype(np.float64), W)
+    packed = oracle.pack_codes(lay.codes, 4)
+    g = _grad_out(M, m, 5, integer=True)
+    dW64, dB64, dA64 = oracle.backward_qat(g, lay.x, Wb, packed, Bz, lay.A, lay.codebook, 4)
+    assert not dB64.any() and not dA64.any()
+    q = torch.from_numpy(packed).to("cuda:0")
+    dW = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda:0")
+    dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
+    dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
+    lords.lords_linear_backward_qat(_dev(g), _dev(lay.x), _dev(Wb), q, _dev(Bz), _dev(lay.A), lay.codebook, 4, M, m, n, r, dW, dB, dA)
+    torch.cuda.synchronize()
+    assert lords.lords_poll_status() == 0
+    assert np.array_equal(dW.cpu().numpy().astype(np.float64), dW64)
+    assert not dB.cpu().numpy().any() and not dA.cpu().numpy().any()
+
+
+def test_qat_backward_declines_shapes_outside_the_tensor_schedule(lords):
+    import torch
+    lay = gen.make_layer(36, 64, 4, 2, bits=4, seed=2)                 # m = 36 is not a multiple of 8
+    q = torch.from_numpy(oracle.pack_codes(lay.codes, 4)).to("cuda:0")
+    Wb = gen.make_weight(36, 64, seed=1)
+    dB = torch.zeros((36, 4), dtype=torch.float32, device="cuda:0")
+    with pytest.raises(lords.LordsError) as ei:
+        lords.lords_linear_backward_qat(_dev(_grad_out(2, 36, 1)), _dev(lay.x), _dev(Wb), q, _dev(lay.B), _dev(lay.A),
+                                        lay.codebook, 4, 2, 36, 64, 4, None, dB, None)
+    assert ei.value.status == -11
