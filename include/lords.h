@@ -19,6 +19,12 @@
  * Note the paper writes W in R^{n x m}; this interface uses m for out-features and
  * n for in-features (the reduction axis).
  *
+ * Around that layer the library also has, each documented at its declaration: the quantisation
+ * step that produces the codes (Alg. 1 step 2.1), the layer's backward for multiplicative
+ * fine-tuning of B and A (Sec. 3.4) and for quantisation-aware training (Eq. 4-5), and two
+ * comparators for the paper's efficiency table (a block-scaled layer, Eq. 2, and that layer with an
+ * additive adapter).
+ *
  * Conventions
  *   - every function returns an int status: LORDS_OK (0) or a negative LORDS_ERR_*;
  *     nothing throws, exits or traps.  Size-returning calls return a negative
