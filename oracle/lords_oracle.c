@@ -264,7 +264,9 @@ int64_t lords_oracle_equivalent_rank(int64_t rows, int64_t cols, int64_t blk)
  *   codes_out  : m*n bytes, one code per byte
  *   runner_out : (may be NULL) the best code among the others (lowest code on ties)
  *   gap_out    : (may be NULL) |S L[runner] - W| - |S L[best] - W| >= 0: by how much the choice was clear
- *   mag_out    : (may be NULL) |S| * max|L| + |W|: the magnitude the gap is to be compared with
+ *   mag_out    : (may be NULL) (sum_k |B_ik A_kj|) * max|L| + |W|: the magnitude the gap is to be compared with
+ *                (a sum of r products rounds in proportion to the sum of their absolute values, which
+ *                under cancellation is much larger than |S| itself)
  */
 int lords_oracle_quantize(const uint16_t *W, const uint16_t *B, const uint16_t *A, const float *codebook, int bits,
                           int64_t m, int64_t n, int64_t r, uint8_t *codes_out, uint8_t *runner_out, double *gap_out,
@@ -303,7 +305,11 @@ int lords_oracle_quantize(const uint16_t *W, const uint16_t *B, const uint16_t *
             codes_out[i * n + j] = (uint8_t)best;
             if (runner_out) runner_out[i * n + j] = (uint8_t)runner;
             if (gap_out) gap_out[i * n + j] = sqrt(e_runner) - sqrt(e_best);
-            if (mag_out) mag_out[i * n + j] = fabs(S_row[j]) * lmax + fabs(w);
+            if (mag_out) {
+                double sabs = 0.0;
+                for (int64_t k = 0; k < r; ++k) sabs += fabs(bf16_to_f64(B[i * r + k]) * bf16_to_f64(A[k * n + j]));
+                mag_out[i * n + j] = sabs * lmax + fabs(w);
+            }
         }
         free(S_row);
     }

@@ -1,10 +1,10 @@
 """GPU quantisation step (Alg. 1, step 2.1) against the fp64 oracle, through the C ABI.
 
-The kernel accumulates S = B A in fp32 and tries the levels in fp32; the oracle does both in fp64.  A
-weight whose two nearest levels are equally far to within fp32 rounding may therefore get either of the
-two.  The test asserts that the codes are equal wherever the oracle's choice was clear by more than
-that rounding distance, that every other difference is the oracle's runner-up code, and that such near
-ties are rare; then that the packed codes, fed to the forward path, reproduce the oracle's forward of
+The kernel accumulates S = B A in fp32 and decides in fp32; the oracle does both in fp64.  A weight whose
+two nearest levels are equally far to within fp32 rounding (of a sum of r products: proportional to
+the sum of their absolute values) may therefore get either of the two.  The test asserts that the codes are equal wherever the oracle's choice was clear by more than
+that rounding distance, that every other code is as good as the oracle's to within that distance, and
+that such near ties are rare; then that the packed codes, fed to the forward path, reproduce the oracle's forward of
 the oracle's codes up to the forward tolerances."""
 import dataclasses
 
@@ -52,13 +52,21 @@ def _check_codes(lords, Q, Wb, lay):
     packed = Q.cpu().numpy().reshape(lay.m, -1)
     got = oracle.unpack_codes(packed, lay.m, lay.n, lay.bits)          # the oracle's own reader of the layout
     want, runner, gap, mag = oracle.quantize(Wb, lay.B, lay.A, lay.codebook, lay.bits, details=True)
-    # fp32 accumulation of r products and one fused multiply-add: a few (r + 2) * 2^-24 of the magnitude
+    # fp32 accumulation of r products and one fused multiply-add: a few (r + 2) * 2^-24 of the magnitude,
+    # which is that of the sum of the ABSOLUTE products B_ik A_kj (times the largest level) plus |W|:
+    # with factors of mixed sign S cancels, and its rounding error does not
     slack = 8.0 * (lay.r + 2) * 2.0 ** -24 * mag
     clear = gap > slack
     assert np.array_equal(got[clear], want[clear]), "codes differ where the choice was clear"
     near = ~clear
-    assert np.all((got[near] == want[near]) | (got[near] == runner[near])), "a near tie went to a third level"
-    assert near.mean() < 2e-3, f"too many near ties: {near.mean():.2e}"
+    # a near tie may go to any level that is as good as the best one to within the slack (with a scale
+    # near zero several levels are)
+    S = gen.bf16_to_f32(lay.B).astype(np.float64) @ gen.bf16_to_f32(lay.A).astype(np.float64)
+    Wf = gen.bf16_to_f32(Wb).astype(np.float64)
+    L = lay.codebook.astype(np.float64)
+    excess = np.abs(S * L[got] - Wf) - np.abs(S * L[want] - Wf)
+    assert np.all(excess <= slack), "a near tie went to a level that is clearly worse"
+    assert near.mean() < 1e-3 + 3e-5 * lay.r, f"too many near ties: {near.mean():.2e}"       # the slack grows with r
     return want
 
 
@@ -78,7 +86,8 @@ def test_quantize_tensor_core_path(lords, bits, m, n, r, mixed):
     _check_codes(lords, Q, Wb, lay)
 
 
-@pytest.mark.parametrize("bits,m,n,r", [(4, 70, 66, 5), (3, 33, 96, 100), (2, 64, 132, 3), (4, 200, 512, 128)])
+@pytest.mark.parametrize("bits,m,n,r", [(4, 70, 66, 5), (3, 33, 96, 100), (2, 64, 132, 3), (4, 200, 512, 128),
+                                        (4, 520, 2048, 128)])      # the last one: many ranks of mixed sign, S cancels heavily
 def test_quantize_cuda_core_path(lords, bits, m, n, r):
     lay = gen.make_layer(m, n, r, 1, bits=bits, seed=m + n, mixed_sign=True)
     Wb = gen.make_weight(m, n, seed=m, sigma=0.05 * (r / 32.0))
