@@ -374,7 +374,7 @@ template <int BITS, bool SORTED> int launch_quantize_tc(QuantParams &k, const St
 int launch_quantize(const void *W, const void *B, const void *A, const float *levels, int bits, int m, int n, int r,
                     uint8_t *Q, State &st, cudaStream_t stream)
 {
-    const bool tc = r <= kRMaxQ && n % kColsQ == 0 && (long long)((m + kRowsQ - 1) / kRowsQ) <= 2147483647LL;
+    const bool tc = r <= kRMaxQ && n % kColsQ == 0;      // the row tiles are the grid's x dimension: any int fits
     if (tc && st.forced_path != 1) {
         QuantParams k;
         k.W = static_cast<const uint16_t *>(W); k.B = static_cast<const uint16_t *>(B); k.Q = Q;
