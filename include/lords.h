@@ -228,9 +228,12 @@ int lords_linear_backward_factors(const void *dy, const void *x, const uint8_t *
  *     dB = dL/dS A^T,   dA = B^T dL/dS.
  *   W  : device, bf16 [m][n], the latent full-precision weight
  *   dW : device, float [m][n] or NULL;  dB : device, float [m][r] or NULL;  dA : device, float [r][n] or NULL
- * Runs on the tensor-core schedule of lords_linear_backward_factors only: m and n multiples of 8 and
- * room in the lords_init workspace for the tiles' contributions, else LORDS_ERR_UNSUPPORTED.  The
- * quotient and S are formed in fp32.  Enqueues on `stream` and returns without synchronising.
+ * Runs on the tensor-core schedule of lords_linear_backward_factors when m and n are multiples of 8
+ * and the lords_init workspace has room for the tiles' contributions; otherwise on the CUDA cores,
+ * one pass over W per requested factor gradient, without scratch memory (any shape the forward calls
+ * accept).  The quotient and S are formed in fp32, S summed over the rank in ascending order on both
+ * schedules.  An output that is NULL is not touched.  Enqueues on `stream` and returns without
+ * synchronising.
  */
 int lords_linear_backward_qat(const void *dy, const void *x, const void *W, const uint8_t *Qpacked, const void *B, const void *A,
                               const float *codebook, int bits, int M, int m, int n, int r, float *dW, float *dB, float *dA,

@@ -112,11 +112,18 @@ struct BwParams {
     int bits, M, m, n, r;
     float *dB;            // [m][r]
     float *dA;            // [r][n]
+    // quantisation-aware training (Eq. 4-5), schedule "walk": the latent weight (null: fine-tuning with
+    // the codes fixed) and where dL/dW goes (null: not asked for)
+    const uint16_t *W;    // bf16 [m][n]
+    float *dW;            // float [m][n]
 };
 
 // ROLE 0: dB for rows blockIdx.x * 64 ..; ROLE 1: dA for columns blockIdx.x * 64 ...
+// With p.W set the factor of dL/dS is L[Q] - W (/) S (Eq. 5; S = B A rebuilt per tile in fp32, summed over
+// the rank in ascending order; 0 where S is 0), and the launch with write_dW set also stores the tile of
+// g^T x as dL/dW (Eq. 4).
 template <int ROLE>
-__global__ void __launch_bounds__(kBwThreads) lords_backward_factors_kernel(const BwParams p)
+__global__ void __launch_bounds__(kBwThreads) lords_backward_factors_kernel(const BwParams p, const int write_dW)
 {
     __shared__ __align__(16) float gs[kTok][kT];   // g[t][i0 + ..]
     __shared__ __align__(16) float xs[kTok][kT];   // x[t][j0 + ..]
@@ -167,14 +174,47 @@ __global__ void __launch_bounds__(kBwThreads) lords_backward_factors_kernel(cons
             }
             __syncthreads();
         }
-        // ---- dS = (g^T x) (.) L[Q]
+        // ---- QAT: the tile of S = B A, by the same outer-product steps with the rank in place of the tokens
+        float sc[4][4];
+        if (p.W) {
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) sc[a][b] = 0.0f;
+            for (int k0 = 0; k0 < p.r; k0 += kTok) {
+                for (int e = tid; e < kTok * kT; e += kBwThreads) {
+                    const int k = k0 + e / kT, cidx = e % kT;
+                    gs[e / kT][cidx] = (k < p.r && i0 + cidx < p.m) ? bf16f(p.B[(size_t)(i0 + cidx) * p.r + k]) : 0.0f;
+                    xs[e / kT][cidx] = (k < p.r && j0 + cidx < p.n) ? bf16f(p.A[(size_t)k * p.n + j0 + cidx]) : 0.0f;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int t = 0; t < kTok; ++t) {
+                    const float4 b4 = *reinterpret_cast<const float4 *>(&gs[t][ty * 4]);
+                    const float4 a4 = *reinterpret_cast<const float4 *>(&xs[t][tx * 4]);
+                    const float bv[4] = {b4.x, b4.y, b4.z, b4.w}, av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) sc[a][b] = fmaf(bv[a], av[b], sc[a][b]);
+                }
+                __syncthreads();
+            }
+        }
+        // ---- dS = (g^T x) (.) L[Q]   (QAT: (.) (L[Q] - W (/) S))
 #pragma unroll
         for (int a = 0; a < 4; ++a)
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
                 const int i = i0 + ty * 4 + a, j = j0 + tx * 4 + b;
                 float lv = 0.0f;
-                if (i < p.m && j < p.n) lv = p.levels[read_code(p.q, row_bytes, i, j, p.bits)];
+                if (i < p.m && j < p.n) {
+                    lv = p.levels[read_code(p.q, row_bytes, i, j, p.bits)];
+                    if (p.W) {
+                        lv = sc[a][b] != 0.0f ? lv - bf16f(p.W[(size_t)i * p.n + j]) / sc[a][b] : 0.0f;
+                        if (write_dW) p.dW[(size_t)i * p.n + j] = c[a][b];
+                    }
+                }
                 ds[ty * 4 + a][tx * 4 + b] = c[a][b] * lv;
             }
         // ---- the factor slice that folds the tile: A[:, j0 ..] (ROLE 0) or B[i0 .., :] (ROLE 1), zero padded
@@ -213,10 +253,10 @@ __global__ void __launch_bounds__(kBwThreads) lords_backward_factors_kernel(cons
         const int e = tid + kBwThreads * a;
         if (ROLE == 0) {
             const int i = own0 + e / r4, k = e % r4;
-            if (i < p.m && k < p.r) p.dB[(size_t)i * p.r + k] = acc[a];
+            if (p.dB && i < p.m && k < p.r) p.dB[(size_t)i * p.r + k] = acc[a];
         } else {
             const int k = e / kT, j = own0 + e % kT;
-            if (k < p.r && j < p.n) p.dA[(size_t)k * p.n + j] = acc[a];
+            if (p.dA && k < p.r && j < p.n) p.dA[(size_t)k * p.n + j] = acc[a];
         }
     }
 }
@@ -650,6 +690,7 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
     for (int c = 0; c < 16; ++c) p.levels[c] = c < (1 << bits) ? levels[c] : 0.0f;
     p.bits = bits; p.M = M; p.m = m; p.n = n; p.r = r;
     p.dB = dB; p.dA = dA;
+    p.W = nullptr; p.dW = nullptr;
     int launches = 0;
     // schedule "tiles" when the workspace holds the tiles' contributions
     const int r4 = (r + 3) & ~3, it_n = (m + kT - 1) / kT, jt_n = (n + kT - 1) / kT;
@@ -682,12 +723,12 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
         return LORDS_OK;
     }
     if (dB) {
-        lords_backward_factors_kernel<0><<<(unsigned)((m + kT - 1) / kT), kBwThreads, 0, stream>>>(p);
+        lords_backward_factors_kernel<0><<<(unsigned)((m + kT - 1) / kT), kBwThreads, 0, stream>>>(p, 0);
         LORDS_CUDA_TRY(cudaGetLastError());
         ++launches;
     }
     if (dA) {
-        lords_backward_factors_kernel<1><<<(unsigned)((n + kT - 1) / kT), kBwThreads, 0, stream>>>(p);
+        lords_backward_factors_kernel<1><<<(unsigned)((n + kT - 1) / kT), kBwThreads, 0, stream>>>(p, 0);
         LORDS_CUDA_TRY(cudaGetLastError());
         ++launches;
     }
@@ -696,7 +737,9 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
     return LORDS_OK;
 }
 
-// Straight-through gradients of quantisation-aware training (Eq. 4-5): tensor schedule only.
+// Straight-through gradients of quantisation-aware training (Eq. 4-5): the tensor schedule where the shapes
+// and the workspace allow it, else the walk (any shape, no scratch memory; g^T x is formed once per
+// requested factor gradient).
 int launch_backward_qat(const uint16_t *g, const uint16_t *x, const uint16_t *W, const uint8_t *q, const uint16_t *B,
                         const uint16_t *A, const float *levels, int bits, int M, int m, int n, int r, float *dW, float *dB,
                         float *dA, State &st, cudaStream_t stream)
@@ -707,7 +750,27 @@ int launch_backward_qat(const uint16_t *g, const uint16_t *x, const uint16_t *W,
     for (int c = 0; c < 16; ++c) p.levels[c] = c < (1 << bits) ? levels[c] : 0.0f;
     p.bits = bits; p.M = M; p.m = m; p.n = n; p.r = r;
     p.dB = dB; p.dA = dA;
-    return launch_backward_tc(p, W, dW, st, stream);
+    p.W = nullptr; p.dW = nullptr;                       // the tensor schedule takes them as arguments
+    if (st.forced_path == 0) {
+        const int rc = launch_backward_tc(p, W, dW, st, stream);
+        if (rc != LORDS_ERR_UNSUPPORTED) return rc;
+    }
+    p.W = W; p.dW = dW;
+    int launches = 0;
+    const bool rows_pass = dB || !dA;                    // dL/dW alone is written by the row pass
+    if (rows_pass) {
+        lords_backward_factors_kernel<0><<<(unsigned)((m + kT - 1) / kT), kBwThreads, 0, stream>>>(p, dW ? 1 : 0);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        ++launches;
+    }
+    if (dA) {
+        lords_backward_factors_kernel<1><<<(unsigned)((n + kT - 1) / kT), kBwThreads, 0, stream>>>(p, dW && !rows_pass ? 1 : 0);
+        LORDS_CUDA_TRY(cudaGetLastError());
+        ++launches;
+    }
+    st.last_launches = launches;
+    st.last_path = "backward_qat_walk";
+    return LORDS_OK;
 }
 
 }  // namespace lords

@@ -189,21 +189,28 @@ def test_qat_backward_against_the_oracle(lords, bits, m, n, r, M, mixed):
     g = _grad_out(M, m, n)
     dW64, dB64, dA64 = oracle.backward_qat(g, lay.x, Wb, packed, lay.B, lay.A, lay.codebook, bits)
     q = torch.from_numpy(packed).to("cuda:0")
-    dW = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda:0")
-    dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
-    dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
-    lords.lords_linear_backward_qat(_dev(g), _dev(lay.x), _dev(Wb), q, _dev(lay.B), _dev(lay.A), lay.codebook, bits,
-                                    M, m, n, r, dW, dB, dA)
-    assert lords.lords_last_path() == "backward_qat_tensor" and lords.lords_last_launch_count() == 3
-    torch.cuda.synchronize()
-    assert lords.lords_poll_status() == 0
-    nw, el = error_metrics(dW.cpu().numpy(), dW64)
-    assert nw <= FACTOR_NORMWISE_TOL and el <= FACTOR_ELEMENT_TOL, ("dW", nw, el)
-    for name, got, want in (("dB", dB.cpu().numpy(), dB64), ("dA", dA.cpu().numpy(), dA64)):
-        assert np.isfinite(got).all(), name
-        nw, el = error_metrics(got, want)
-        print(f"qat {name} bits={bits} m={m} n={n} r={r} M={M}: normwise={nw:.2e} element={el:.2e}")
-        assert nw <= QAT_NORMWISE_TOL and el <= QAT_ELEMENT_TOL, (name, nw, el)
+    # both schedules: the tile product on the tensor cores, and the walk on the CUDA cores that any forced
+    # forward path other than "auto" selects (no scratch memory, one launch per factor gradient)
+    for option, schedule, launches in (("auto", "backward_qat_tensor", 3), ("simt", "backward_qat_walk", 2)):
+        dW = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda:0")
+        dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
+        dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
+        lords.lords_set_option("path", option)
+        try:
+            lords.lords_linear_backward_qat(_dev(g), _dev(lay.x), _dev(Wb), q, _dev(lay.B), _dev(lay.A), lay.codebook, bits,
+                                            M, m, n, r, dW, dB, dA)
+        finally:
+            lords.lords_set_option("path", "auto")
+        assert lords.lords_last_path() == schedule and lords.lords_last_launch_count() == launches
+        torch.cuda.synchronize()
+        assert lords.lords_poll_status() == 0
+        nw, el = error_metrics(dW.cpu().numpy(), dW64)
+        assert nw <= FACTOR_NORMWISE_TOL and el <= FACTOR_ELEMENT_TOL, (schedule, "dW", nw, el)
+        for name, got, want in (("dB", dB.cpu().numpy(), dB64), ("dA", dA.cpu().numpy(), dA64)):
+            assert np.isfinite(got).all(), (schedule, name)
+            nw, el = error_metrics(got, want)
+            print(f"qat {schedule} {name} bits={bits} m={m} n={n} r={r} M={M}: normwise={nw:.2e} element={el:.2e}")
+            assert nw <= QAT_NORMWISE_TOL and el <= QAT_ELEMENT_TOL, (schedule, name, nw, el)
 
 
 def test_qat_backward_exactly_representable_weight_is_exact(lords):
@@ -232,13 +239,33 @@ def test_qat_backward_exactly_representable_weight_is_exact(lords):
     assert not dB.cpu().numpy().any() and not dA.cpu().numpy().any()
 
 
-def test_qat_backward_declines_shapes_outside_the_tensor_schedule(lords):
+@pytest.mark.parametrize("bits,m,n,r,M,ask", [(4, 36, 64, 4, 2, "WBA"), (3, 75, 96, 7, 19, "WBA"), (2, 130, 68, 33, 1, "BA"),
+                                              (4, 100, 70, 17, 5, "W"), (4, 61, 130, 3, 33, "WA"), (3, 67, 64, 128, 4, "B")])
+def test_qat_backward_walk_takes_shapes_outside_the_tensor_schedule(lords, bits, m, n, r, M, ask):
+    """Row or column counts that are not multiples of 8 (the row pitches of g and x do not suit TMA): the
+    walk runs, with any subset of the three gradients asked for; what is not asked for is not touched."""
     import torch
-    lay = gen.make_layer(36, 64, 4, 2, bits=4, seed=2)                 # m = 36 is not a multiple of 8
-    q = torch.from_numpy(oracle.pack_codes(lay.codes, 4)).to("cuda:0")
-    Wb = gen.make_weight(36, 64, seed=1)
-    dB = torch.zeros((36, 4), dtype=torch.float32, device="cuda:0")
-    with pytest.raises(lords.LordsError) as ei:
-        lords.lords_linear_backward_qat(_dev(_grad_out(2, 36, 1)), _dev(lay.x), _dev(Wb), q, _dev(lay.B), _dev(lay.A),
-                                        lay.codebook, 4, 2, 36, 64, 4, None, dB, None)
-    assert ei.value.status == -11
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=5 * m + n + r, mixed_sign=(r % 2 == 1))
+    Wb = gen.make_weight(m, n, seed=m + r, sigma=0.05 * (r / 32.0))
+    codes = oracle.quantize(Wb, lay.B, lay.A, lay.codebook, bits)
+    packed = oracle.pack_codes(codes, bits)
+    g = _grad_out(M, m, n + 1)
+    want = dict(zip("WBA", oracle.backward_qat(g, lay.x, Wb, packed, lay.B, lay.A, lay.codebook, bits)))
+    q = torch.from_numpy(packed).to("cuda:0")
+    shapes = {"W": (m, n), "B": (m, r), "A": (r, n)}
+    out = {k: torch.full(shapes[k], float("nan"), dtype=torch.float32, device="cuda:0") for k in "WBA"}
+    args = [out[k] if k in ask else None for k in "WBA"]
+    lords.lords_linear_backward_qat(_dev(g), _dev(lay.x), _dev(Wb), q, _dev(lay.B), _dev(lay.A), lay.codebook, bits,
+                                    M, m, n, r, *args)
+    launches = (1 if ("B" in ask or "A" not in ask) else 0) + (1 if "A" in ask else 0)
+    assert lords.lords_last_path() == "backward_qat_walk" and lords.lords_last_launch_count() == launches
+    torch.cuda.synchronize()
+    assert lords.lords_poll_status() == 0
+    for k in "WBA":
+        got = out[k].cpu().numpy()
+        if k not in ask:
+            assert np.isnan(got).all(), k
+            continue
+        assert np.isfinite(got).all(), k
+        nw, el = error_metrics(got, want[k])
+        assert nw <= QAT_NORMWISE_TOL and el <= QAT_ELEMENT_TOL, (k, nw, el)
