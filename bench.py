@@ -374,37 +374,61 @@ def time_case(case, steps, warmup, device, rank, world, sampler=None, do_e2e=Tru
 STACK_LAYERS = ["q", "k", "v", "o", "gate", "up", "down"]
 
 
-def time_stack(M, mlp_bits, steps, device):
+def time_stack(M, mlp_bits, steps, device, qkv_one_call=False, gate_up_one_call=False):
     """Full Llama-3-8B linear stack: 32 layers x {q, k, v, o, gate, up, down}, one forward call per
     module (224 calls) from one CUDA graph.  Attention modules are NF4 (r = 32; r = 16 for k/v); the
     MLP modules are NF4 r = 32, NF3 r = 48 or NF2 r = 32 (the NF4/NF2 layer mix of the paper's low-bit setting).  Each of the 224 modules has its own weights (3.5 GB
-    at 4 bits: far beyond L2) and its own activations."""
+    at 4 bits: far beyond L2) and its own activations.
+
+    qkv_one_call / gate_up_one_call: the projections of a block that read the same activations go through
+    one call as one layer (rows and ranks concatenated, B block-diagonal: packing.concat_layers) -- 160 or
+    128 calls; bytes and flops are still counted per original module."""
+    import dataclasses
+
     import numpy as np
     import torch
     from paper_2601_22716_b200 import binding as lords
     from paper_2601_22716_b200 import inputs as gen
+    from paper_2601_22716_b200 import packing
 
-    protos = {}
+    lays = {}
     for idx, name in enumerate(STACK_LAYERS):
         m, n = gen.LLAMA3_8B_SHAPES[name]
         mlp = name in ("gate", "up", "down")
         bits = mlp_bits if mlp else 4
         r = (48 if bits == 3 else 32) if mlp else (16 if name in ("k", "v") else 32)
-        lay = gen.make_layer(m, n, r, M, bits=bits, seed=idx)
-        packed = lords.lords_pack_codes(lay.codes, bits)
+        lays[name] = gen.make_layer(m, n, r, M, bits=bits, seed=idx)
+    byt = flo = 0
+    for lay in lays.values():
+        c = dict(m=lay.m, n=lay.n, bits=lay.bits, r=lay.r, M=M)
+        byt += 32 * algorithmic_bytes(c)
+        flo += 32 * useful_flops(c)
+    modules = list(STACK_LAYERS)
+    groups = []
+    if qkv_one_call:
+        groups.append(("qkv", ("q", "k", "v")))
+    if gate_up_one_call:
+        groups.append(("gate_up", ("gate", "up")))
+    for joined, names in groups:
+        parts = [lays.pop(k) for k in names]
+        codes, Bc, Ac = packing.concat_layers([p.codes for p in parts], [p.B for p in parts], [p.A for p in parts])
+        lays[joined] = dataclasses.replace(parts[0], m=codes.shape[0], r=Ac.shape[0], codes=codes, B=Bc, A=Ac)
+        at = modules.index(names[0])
+        modules = modules[:at] + [joined] + modules[at + len(names):]
+    protos = {}
+    for name in modules:
+        lay = lays[name]
+        packed = lords.lords_pack_codes(lay.codes, lay.bits)
         protos[name] = (lay, torch.from_numpy(packed).to(device), torch.from_numpy(lay.B.view(np.int16)).to(device),
                         torch.from_numpy(lay.A.view(np.int16)).to(device), torch.from_numpy(lay.x.view(np.int16)).to(device))
-    calls, byt, flo = [], 0, 0
+    calls = []
     for layer in range(32):
-        for name in STACK_LAYERS:
+        for name in modules:
             lay, q0, B0, A0, x0 = protos[name]
             q = q0 if layer == 0 else torch.roll(q0, layer, 0).contiguous()
             B = B0 if layer == 0 else torch.roll(B0, layer, 0).contiguous()
             y = torch.zeros((M, lay.m), dtype=torch.int16, device=device)
             calls.append((lay, q, B, A0.clone(), x0.clone(), y))
-            c = dict(m=lay.m, n=lay.n, bits=lay.bits, r=lay.r, M=M)
-            byt += algorithmic_bytes(c)
-            flo += useful_flops(c)
 
     def one_pass():
         for lay, q, B, A, x, y in calls:
@@ -442,7 +466,8 @@ def time_stack(M, mlp_bits, steps, device):
             raise RuntimeError(f"device status {status} during the M = {M} stack, twice")
     peaks = measured_peaks()
     gbs, tfs = byt / (ms * 1e-3) / 1e9, flo / (ms * 1e-3) / 1e12
-    return {"case": f"stack_m{M}_mlp{mlp_bits}bit", "ms_per_pass": ms, "ms_per_token": ms / M, "calls": len(calls),
+    return {"case": f"stack_m{M}_mlp{mlp_bits}bit" + ("_qkv_one_call" if qkv_one_call else "") + ("_gate_up_one_call" if gate_up_one_call else ""),
+            "ms_per_pass": ms, "ms_per_token": ms / M, "calls": len(calls),
             "algorithmic_bytes": byt, "gbs": gbs, "tflops": tfs, "frac_hbm": gbs / peaks["hbm_gbs"],
             "frac_tensor": tfs / peaks["bf16_tflops"], "steps": steps, "status_retries": status_retries}
 
@@ -860,8 +885,10 @@ def main():
     if not (not args.case and not args.no_extras and world == 1):
         comparators = None
     if not args.no_stack and not args.no_extras and not args.case and world == 1:
-        for (M, mlp_bits, k) in [(1, 4, 30), (8, 4, 30), (512, 4, 5), (1, 3, 30), (1, 2, 30)]:
-            stack.append(time_stack(M, mlp_bits, k, device))
+        # the last line: the projections that share their input (q, k, v; gate, up) each as one call
+        for (M, mlp_bits, k, joined) in [(1, 4, 30, False), (8, 4, 30, False), (512, 4, 5, False), (1, 3, 30, False), (1, 2, 30, False),
+                                         (1, 4, 30, True)]:
+            stack.append(time_stack(M, mlp_bits, k, device, qkv_one_call=joined, gate_up_one_call=joined))
             torch.cuda.empty_cache()
 
     if rank == 0:

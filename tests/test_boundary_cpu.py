@@ -126,3 +126,26 @@ def test_measurement_options_are_validated():
         assert ei.value.status == -10
     for key, value in [("path", "auto"), ("splitk", "0"), ("bn", "0")]:
         lords.lords_set_option(key, value)
+
+
+def test_concat_layers_is_the_concatenation_of_the_layers_outputs():
+    """Host logic of packing.concat_layers, checked with the oracle: the combined layer (rows and ranks
+    stacked, B block-diagonal) gives exactly the layers' outputs side by side -- the zero blocks of B add
+    exact zeros to every scale -- and malformed input is refused."""
+    from paper_2601_22716_b200 import inputs as gen
+    from paper_2601_22716_b200 import packing
+    shapes = [(96, 5), (32, 16), (40, 3)]
+    lays = [gen.make_layer(m, 128, r, 3, bits=4, seed=10 + i, mixed_sign=(i == 1)) for i, (m, r) in enumerate(shapes)]
+    x = lays[0].x
+    codes, B, A = packing.concat_layers([l.codes for l in lays], [l.B for l in lays], [l.A for l in lays])
+    assert codes.shape == (168, 128) and B.shape == (168, 24) and A.shape == (24, 128)
+    assert not B[:96, 5:].any() and not B[96:128, :5].any() and not B[96:128, 21:].any() and not B[128:, :21].any()
+    y = oracle.forward(x, oracle.pack_codes(codes, 4), B, A, lays[0].codebook, 4)
+    parts = [oracle.forward(x, oracle.pack_codes(l.codes, 4), l.B, l.A, l.codebook, 4) for l in lays]
+    assert np.array_equal(y, np.concatenate(parts, axis=1))
+    with pytest.raises(ValueError):
+        packing.concat_layers([lays[0].codes], [lays[0].B, lays[1].B], [lays[0].A])
+    with pytest.raises(ValueError):
+        packing.concat_layers([lays[0].codes, lays[1].codes[:, :64]], [lays[0].B, lays[1].B], [lays[0].A, lays[1].A[:, :64]])
+    with pytest.raises(ValueError):
+        packing.concat_layers([lays[0].codes], [lays[1].B], [lays[0].A])

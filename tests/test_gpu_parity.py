@@ -469,3 +469,28 @@ def test_four_bit_entry_point_and_launch_count(lords):
     assert np.array_equal(y.cpu().numpy().view(np.uint16), ybf)
     assert lords.lords_last_launch_count() >= 1
     assert lords.lords_last_path() in ("simt", "decode", "decode16", "umma")
+
+
+@pytest.mark.parametrize("M", [1, 8])
+def test_qkv_as_one_layer_full_size(lords, M):
+    """The q, k and v projections of a Llama-3-8B block (NF4, r = 32 / 16 / 16) as one 6144 x 4096 layer
+    of rank 64 with a block-diagonal B (packing.concat_layers): against the oracle on stratified rows,
+    and against the three separate calls."""
+    import dataclasses
+    import torch
+    from paper_2601_22716_b200 import packing
+    parts = [gen.make_layer(m, 4096, r, M, bits=4, seed=40 + i) for i, (m, r) in enumerate([(4096, 32), (1024, 16), (1024, 16)])]
+    codes, B, A = packing.concat_layers([p.codes for p in parts], [p.B for p in parts], [p.A for p in parts])
+    lay = dataclasses.replace(parts[0], m=6144, r=64, codes=codes, B=B, A=A)
+    dl, y32, ybf = _run(lords, lay, "auto")
+    # rank 64: one token fits the reassociated decode kernel (M * r <= 64); the 16-token kernel holds r <= 32
+    # at 4 bits, so eight tokens go to the scale-MMA kernel
+    assert lords.lords_last_path() == ("decode" if M == 1 else "umma")
+    rows = _sampled_rows(6144, 32, 9)
+    check_against_oracle(y32[:, rows], ybf[:, rows], _oracle(lay, dl.packed_host, rows=rows), label=f"qkv as one layer M={M}")
+    assert np.isfinite(y32).all()
+    separate = []
+    for p in parts:
+        p.x = lay.x
+        separate.append(_run(lords, p, "auto")[1])
+    assert error_metrics(y32, np.concatenate(separate, axis=1).astype(np.float64))[0] <= 1e-5
