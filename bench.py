@@ -885,10 +885,11 @@ def main():
     if not (not args.case and not args.no_extras and world == 1):
         comparators = None
     if not args.no_stack and not args.no_extras and not args.case and world == 1:
-        # the last line: the projections that share their input (q, k, v; gate, up) each as one call
-        for (M, mlp_bits, k, joined) in [(1, 4, 30, False), (8, 4, 30, False), (512, 4, 5, False), (1, 3, 30, False), (1, 2, 30, False),
-                                         (1, 4, 30, True)]:
-            stack.append(time_stack(M, mlp_bits, k, device, qkv_one_call=joined, gate_up_one_call=joined))
+        # the last two lines: projections that share their input as one call (q, k, v; at one token also gate, up)
+        for (M, mlp_bits, k, qkv, gate_up) in [(1, 4, 30, False, False), (8, 4, 30, False, False), (512, 4, 5, False, False),
+                                               (1, 3, 30, False, False), (1, 2, 30, False, False),
+                                               (1, 4, 30, True, True), (8, 4, 30, True, False)]:
+            stack.append(time_stack(M, mlp_bits, k, device, qkv_one_call=qkv, gate_up_one_call=gate_up))
             torch.cuda.empty_cache()
 
     if rank == 0:

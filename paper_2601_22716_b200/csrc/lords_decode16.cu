@@ -62,7 +62,6 @@ constexpr uint32_t kSCol = 64;
 constexpr int SD = 2;
 constexpr uint32_t kWCol = kSCol + SD * kStep;         // 320
 constexpr int WS = 3;                                  // W ring = activation ring depth
-constexpr int SA = 4;                                  // factor-tile ring depth
 // A barrier is waited on by parity alone, so whoever waits for its phase n must know that phase n - 1
 // has completed: true for a warp that waits for every phase of the barrier, and for a group (or an
 // issuer) that owns it.  Worker groups and main issuers take the k-steps alternately, and the W ring
@@ -80,6 +79,9 @@ template <int BITS, int RP> struct XCfg {
     static constexpr int QSTAGE = kRows * QROW;
     static constexpr int SQ = BITS == 4 ? 4 : 6;               // code-tile ring depth (even: one group per barrier)
     static constexpr int AATOM = RP * 128;                     // RP ranks x 64 columns bf16
+    // factor-tile ring depth (even: each of its barriers belongs to one scale issuer).  The 4-bit layout keeps
+    // this ring below the 64 KB boundary of its level table, where 64 ranks leave room for two stages.
+    static constexpr int SA = (BITS == 4 && RP == 64) ? 2 : 4;
     static constexpr int ASTAGE = 2 * AATOM;
     static constexpr int LUT_ENTRIES = BITS == 4 ? 256 : BITS == 3 ? 64 : 16;   // one entry per code pair
     // 32 lane-private copies of every entry (word = lane).  4-bit: entries 256 bytes apart, table on
@@ -197,7 +199,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         x0 = (raw + 1023u) & ~1023u;
         b_tile = x0 + WS * kXStage;
         a0 = b_tile + kBTileBytes;
-        bars = a0 + SA * C::ASTAGE;
+        bars = a0 + C::SA * C::ASTAGE;
         q0 = lut + C::LUT_BYTES;
         red0 = q0 + SQ * C::QSTAGE;
         fits = bars + C::BAR_BYTES <= lut && red0 + C::RED_BYTES <= raw + (uint32_t)C::SMEM;
@@ -207,7 +209,7 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         x0 = (red0 + C::RED_BYTES + 1023u) & ~1023u;
         b_tile = x0 + WS * kXStage;
         a0 = b_tile + kBTileBytes;
-        bars = a0 + SA * C::ASTAGE;
+        bars = a0 + C::SA * C::ASTAGE;
         fits = bars + C::BAR_BYTES <= raw + (uint32_t)C::SMEM;
     }
     const uint32_t bar_q_full = bars + 8 * C::kBarQFull, bar_q_empty = bars + 8 * C::kBarQEmpty;
@@ -342,8 +344,8 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
             }
             const uint32_t tx = (uint32_t)(2 * p.r_pad * 128);
             for (int it = 0; it < total; ++it) {
-                const int sa = it % SA;
-                if (it >= SA && !mbar_wait(bar_a_done + 8 * sa, (uint32_t)((it / SA - 1) & 1))) { failed = true; break; }
+                const int sa = it % C::SA;
+                if (it >= C::SA && !mbar_wait(bar_a_done + 8 * sa, (uint32_t)((it / C::SA - 1) & 1))) { failed = true; break; }
                 const uint32_t bar = bar_a_full + 8 * sa;
                 mbar_expect_tx(bar, tx);
 #pragma unroll
@@ -380,11 +382,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         const uint32_t a_lo0 = (uint32_t)umma_desc_sw128(0, 1024, (uint32_t)C::AATOM) | ((a0 & 0x3FFFFu) >> 4);
         const int rsteps = p.r_pad / 16;
         const int sj = warp - kScaleWarp0;
-        static_assert(SD == 2 && SA % 2 == 0, "one scale issuer per S buffer; each factor-ring barrier belongs to one of them");
+        static_assert(SD == 2 && C::SA % 2 == 0, "one scale issuer per S buffer; each factor-ring barrier belongs to one of them");
         if (b_by_tma && sj < total && !mbar_wait(bar_b_full, 0)) failed = true;
         for (int it = sj; !BLOCK && it < total && !failed; it += 2) {
-            const int sa = it % SA, sd = it % SD;
-            if (!mbar_wait(bar_a_full + 8 * sa, (uint32_t)((it / SA) & 1))) { failed = true; break; }
+            const int sa = it % C::SA, sd = it % SD;
+            if (!mbar_wait(bar_a_full + 8 * sa, (uint32_t)((it / C::SA) & 1))) { failed = true; break; }
             if (it >= SD && !mbar_wait(bar_s_empty + 8 * sd, (uint32_t)((it / SD - 1) & 1))) { failed = true; break; }
             tc_fence_after_sync();
             if (lane == 0) {
@@ -460,7 +462,6 @@ __global__ void __launch_bounds__(kThreads, 1) lords_decode16_kernel(const __gri
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         const uint32_t lut_lane = lut + 4u * (uint32_t)lane;
 
-        const bool stamper = wg == 0 && lane == 0;
         for (int it = g; it < total; it += 2) {
             const int sq = it % SQ, sd = it % SD, ws = it % WS;
             // this thread's 64 columns of S, as 32 fp16 pairs
@@ -681,14 +682,14 @@ template <int BITS, int RP, bool BLOCK = false> int launch_variant(Dec16Params &
 }  // namespace
 
 // Rules of this path: M <= 16 (with automatic dispatch one or two tokens go to the
-// reassociated decode kernel first, and come here when that one declines the rank); r <= 32 (4-bit) or <= 64 (3-bit), which is what the shared-memory layout holds;
+// reassociated decode kernel first, and come here when that one declines the rank); r <= 64, which is what the shared-memory layout holds;
 // n a multiple of 64 (2- and 4-bit) or 128 (3-bit), which makes every TMA row pitch a multiple of 16 bytes.
 // Anything else: LORDS_ERR_UNSUPPORTED.
 int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
 {
     if (p.bits < 2 || p.bits > 4) return LORDS_ERR_UNSUPPORTED;
     if (p.M > kTok) return LORDS_ERR_UNSUPPORTED;
-    if (p.r > (p.bits == 4 ? 32 : 64)) return LORDS_ERR_UNSUPPORTED;
+    if (p.r > 64) return LORDS_ERR_UNSUPPORTED;
     if (p.n % (p.bits == 3 ? 128 : 64) != 0) return LORDS_ERR_UNSUPPORTED;
 
     Dec16Params k;
@@ -701,7 +702,7 @@ int launch_decode16(const Problem &p, State &st, cudaStream_t stream)
     k.status = st.status_word;
     k.scales = nullptr; k.blk = 0; k.nblk = 0;
     int rc;
-    if (p.bits == 4) rc = launch_variant<4, 32>(k, p, st, stream);
+    if (p.bits == 4) rc = k.r_pad <= 32 ? launch_variant<4, 32>(k, p, st, stream) : launch_variant<4, 64>(k, p, st, stream);
     else if (p.bits == 3) rc = k.r_pad <= 32 ? launch_variant<3, 32>(k, p, st, stream) : launch_variant<3, 64>(k, p, st, stream);
     else rc = k.r_pad <= 32 ? launch_variant<2, 32>(k, p, st, stream) : launch_variant<2, 64>(k, p, st, stream);
     if (rc != LORDS_OK) return rc;

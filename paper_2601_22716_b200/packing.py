@@ -9,8 +9,8 @@ becomes block-diagonal, so that S = B A of Eq. 3 keeps every layer's own scales 
 
 The output of the combined layer is the concatenation of the layers' outputs.  All layers must have
 the same code width and in-features; the combined rank is the sum of the ranks.  The saving is there
-where the combined rank still fits the decode kernel of the token count (one token: rank <= 64; 2 to 16
-tokens at 4 bits: rank <= 32); beyond that the call falls to a slower path.
+where the combined rank still fits the decode kernels (rank <= 64, up to 16 tokens); beyond that the
+call falls to a slower path.
 """
 from __future__ import annotations
 

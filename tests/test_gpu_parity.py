@@ -196,6 +196,11 @@ DECODE16_SHAPES = [
     (2, 1000, 2048, 48, 16, True),
     (2, 256, 64, 12, 9, True),
     (4, 512, 1024, 15, 8, True),
+    # 4-bit codes with ranks above 32 (a two-stage factor ring)
+    (4, 384, 1024, 48, 8, True),
+    (4, 300, 2112, 64, 16, False),
+    (4, 128, 128, 33, 3, True),       # one k-step
+    (4, 1024, 4096, 64, 5, True),
 ]
 
 
@@ -208,7 +213,7 @@ def test_decode16_kernel_shapes(lords, bits, m, n, r, M, mixed):
     check_against_oracle(y32, ybf, y64)
 
 
-@pytest.mark.parametrize("bits,m,n,r,M", [(4, 700, 2048, 32, 8), (4, 256, 512, 16, 16), (3, 384, 1024, 48, 3),
+@pytest.mark.parametrize("bits,m,n,r,M", [(4, 700, 2048, 32, 8), (4, 256, 512, 16, 16), (4, 260, 1024, 64, 7), (3, 384, 1024, 48, 3),
                                           (3, 131, 384, 7, 9), (2, 300, 1024, 5, 4), (2, 256, 192, 40, 16)])
 def test_decode16_kernel_integer_case_is_bit_exact(lords, bits, m, n, r, M):
     lay = gen.make_integer_layer(m, n, r, M, bits=bits, seed=bits + m + M)
@@ -239,7 +244,7 @@ def test_decode16_kernel_cluster_split_is_deterministic(lords, cluster):
 def test_decode16_kernel_declines_what_it_cannot_run(lords):
     lords.lords_set_option("path", "decode16")
     try:
-        for lay in (gen.make_layer(256, 256, 48, 4, bits=4, seed=0),      # 4-bit with r > 32
+        for lay in (gen.make_layer(256, 256, 65, 4, bits=4, seed=0),      # r > 64
                     gen.make_layer(256, 256, 4, 17, bits=4, seed=0)):     # more than one token tile
             with pytest.raises(lords.LordsError) as ei:
                 DeviceLayer(lay).forward()
@@ -483,9 +488,8 @@ def test_qkv_as_one_layer_full_size(lords, M):
     codes, B, A = packing.concat_layers([p.codes for p in parts], [p.B for p in parts], [p.A for p in parts])
     lay = dataclasses.replace(parts[0], m=6144, r=64, codes=codes, B=B, A=A)
     dl, y32, ybf = _run(lords, lay, "auto")
-    # rank 64: one token fits the reassociated decode kernel (M * r <= 64); the 16-token kernel holds r <= 32
-    # at 4 bits, so eight tokens go to the scale-MMA kernel
-    assert lords.lords_last_path() == ("decode" if M == 1 else "umma")
+    # rank 64: one token fits the reassociated decode kernel (M * r <= 64), eight go to the 16-token kernel
+    assert lords.lords_last_path() == ("decode" if M == 1 else "decode16")
     rows = _sampled_rows(6144, 32, 9)
     check_against_oracle(y32[:, rows], ybf[:, rows], _oracle(lay, dl.packed_host, rows=rows), label=f"qkv as one layer M={M}")
     assert np.isfinite(y32).all()
