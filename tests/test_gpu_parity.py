@@ -414,26 +414,28 @@ def test_status_word_round_trip_and_recovery(lords):
     assert np.array_equal(y32, y32b) and np.array_equal(ybf, ybfb)
 
 
-def test_many_back_to_back_launches_of_the_two_half_kernel_leave_no_status(lords):
+@pytest.mark.parametrize("m,n,r,bits,M,path", [(14336, 4096, 48, 3, 1, "decode"), (6144, 4096, 64, 4, 8, "decode16")])
+def test_many_back_to_back_launches_leave_no_status(lords, m, n, r, bits, M, path):
     """The 3-bit gate shape runs the two-half variant of the M <= 2 kernel, whose rings are three
-    stages deep while its converter groups take the k-steps alternately.  Several thousand dependent
-    launches over distinct weight copies (replayed from a CUDA graph, as a model's layers are) must
-    leave the status word clear and reproduce the first result bit for bit: a barrier that two groups
-    share by parity alone would show up here as a recorded give-up."""
+    stages deep while its converter groups take the k-steps alternately; a 4-bit layer of rank 64 runs
+    the 16-token kernel with a two-stage factor ring that its two scale issuers share.  Several thousand
+    dependent launches over distinct weight copies (replayed from a CUDA graph, as a model's layers
+    are) must leave the status word clear and reproduce the first result bit for bit: a barrier that
+    two groups share by parity alone would show up here as a recorded give-up."""
     import torch
-    lay = gen.make_layer(14336, 4096, 48, 1, bits=3, seed=91)
+    lay = gen.make_layer(m, n, r, M, bits=bits, seed=91)
     dl = DeviceLayer(lay)
     copies = 6
     qs = [dl.q] + [torch.roll(dl.q, l, 0).contiguous() for l in range(1, copies)]
-    ys = [torch.zeros((1, lay.m), dtype=torch.int16, device="cuda:0") for _ in range(copies)]
+    ys = [torch.zeros((M, lay.m), dtype=torch.int16, device="cuda:0") for _ in range(copies)]
 
     def one_round():
         for q, y in zip(qs, ys):
-            lords.lords_linear_forward_bits(dl.x, q, dl.B, dl.A, lay.codebook, 3, 1, lay.m, lay.n, lay.r, y)
+            lords.lords_linear_forward_bits(dl.x, q, dl.B, dl.A, lay.codebook, bits, M, lay.m, lay.n, lay.r, y)
 
     one_round()
     torch.cuda.synchronize()
-    assert lords.lords_last_path() == "decode"
+    assert lords.lords_last_path() == path
     first = [y.clone() for y in ys]
     s = torch.cuda.Stream()
     s.wait_stream(torch.cuda.current_stream())
