@@ -130,8 +130,10 @@ __global__ void __launch_bounds__(kBwThreads) lords_backward_factors_kernel(cons
     __shared__ float ds[kT][kT + 1];               // dS tile
     __shared__ uint16_t fs[kRMaxBw][kT + 2];       // ROLE 0: A[k][j0 + ..]; ROLE 1: B[i0 + ..][k] stored [k][i]
                                                    // (rows 33 words apart: neighbouring k fall into different banks)
+    __shared__ float lv_s[16];                     // the level table (a per-thread index into the kernel parameters is replayed per distinct value)
 
     const int tid = threadIdx.x;
+    if (tid < 16) lv_s[tid] = p.levels[tid];       // read after the first __syncthreads below
     const int ty = tid >> 4, tx = tid & 15;   // 16 x 16 threads, a 4 x 4 micro-tile each
     const int own0 = blockIdx.x * kT;         // first owned row (ROLE 0) or column (ROLE 1)
     const int walk_len = ROLE == 0 ? p.n : p.m;
@@ -209,7 +211,7 @@ __global__ void __launch_bounds__(kBwThreads) lords_backward_factors_kernel(cons
                 const int i = i0 + ty * 4 + a, j = j0 + tx * 4 + b;
                 float lv = 0.0f;
                 if (i < p.m && j < p.n) {
-                    lv = p.levels[read_code(p.q, row_bytes, i, j, p.bits)];
+                    lv = lv_s[read_code(p.q, row_bytes, i, j, p.bits)];
                     if (p.W) {
                         lv = sc[a][b] != 0.0f ? lv - bf16f(p.W[(size_t)i * p.n + j]) / sc[a][b] : 0.0f;
                         if (write_dW) p.dW[(size_t)i * p.n + j] = c[a][b];
@@ -270,8 +272,10 @@ __global__ void __launch_bounds__(kBwThreads) lords_backward_tile_kernel(const B
     __shared__ __align__(16) float xs[kTok][kT];
     __shared__ float ds[kT][kT + 1];
     __shared__ uint16_t fs[kRMaxBw][kT + 2];
+    __shared__ float lv_s[16];
 
     const int tid = threadIdx.x;
+    if (tid < 16) lv_s[tid] = p.levels[tid];       // read after the first __syncthreads below
     const int ty = tid >> 4, tx = tid & 15;
     const int jt = blockIdx.x, it = blockIdx.y;
     const int i0 = it * kT, j0 = jt * kT;
@@ -309,7 +313,7 @@ __global__ void __launch_bounds__(kBwThreads) lords_backward_tile_kernel(const B
         for (int b = 0; b < 4; ++b) {
             const int i = i0 + ty * 4 + a, j = j0 + tx * 4 + b;
             float lv = 0.0f;
-            if (i < p.m && j < p.n) lv = p.levels[read_code(p.q, row_bytes, i, j, p.bits)];
+            if (i < p.m && j < p.n) lv = lv_s[read_code(p.q, row_bytes, i, j, p.bits)];
             ds[ty * 4 + a][tx * 4 + b] = c[a][b] * lv;
         }
     if (part_dB) {
@@ -354,6 +358,10 @@ constexpr int kTcThreads = 320;
 constexpr int kTcGAtom = kTcTok * 128;                        // 64 tokens x 64 rows of W, bf16
 constexpr int kTcStage = 2 * kTcGAtom + kTcTok * 128;         // g: two atoms, x: one
 constexpr uint32_t kTcTmemCols = 64;
+// epilogue buffers (floats): rows of the dS tile and of the A slice are 68 floats apart, rows of the B slice
+// (stored [rank][row]) 132: multiples of four, so that four neighbouring values are one 16-byte word, and with
+// 16-byte words of consecutive rows in different banks
+constexpr int kTcDsPitch = kTcCols + 4, kTcFbPitch = kTcRows + 4;
 
 struct alignas(64) BwTcParams {
     CUtensorMap tm_g;     // bf16 [M][m], box {64, 64}, 128-byte swizzle (tokens past M read as zero)
@@ -371,24 +379,27 @@ __host__ __device__ constexpr int bw_tc_smem(int r4)
 {
     // the epilogue's buffers (dS tile, the two factor slices) reuse the stages once the MMAs are done
     const int stages = kTcStages * kTcStage;
-    const int epi = kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 4 + r4 * (kTcRows + 2) * 4;
+    const int epi = kTcRows * kTcDsPitch * 4 + r4 * kTcDsPitch * 4 + r4 * kTcFbPitch * 4;
     return 1024 + (stages > epi ? stages : epi) + 256;
 }
 
 // QAT: the tile of g^T x is dL/dW^ itself (Eq. 4: stored as dL/dW if asked for), and the factor of
 // dL/dS is Q - W (/) S instead of Q (Eq. 5), with S = B A rebuilt per element from the factor slices.
 template <bool QAT>
-__global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __grid_constant__ BwTcParams p)
+__global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 3) lords_backward_tc_kernel(const __grid_constant__ BwTcParams p)
 {
     extern __shared__ uint8_t tc_smem_raw[];
     const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
     uint8_t *base_ptr = tc_smem_raw + (base - smem_u32(tc_smem_raw));
     const int r4 = (p.b.r + 3) & ~3;
     const int stages_bytes = kTcStages * kTcStage;
-    const int epi_bytes = kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 4 + r4 * (kTcRows + 2) * 4;
+    const int epi_bytes = kTcRows * kTcDsPitch * 4 + r4 * kTcDsPitch * 4 + r4 * kTcFbPitch * 4;
     const uint32_t bars = base + (uint32_t)(stages_bytes > epi_bytes ? stages_bytes : epi_bytes);
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kTcStages, bar_acc = bar_empty + 8 * kTcStages;
     const uint32_t tmem_slot = bar_acc + 8;
+    // the level table in shared memory (16 floats behind the barriers): a lookup by a per-thread code is one
+    // conflict-free read there, where the same lookup in the kernel parameters is replayed once per distinct code
+    float *levels_s = reinterpret_cast<float *>(base_ptr + (bars - base) + 128);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int jt = blockIdx.x, it = blockIdx.y;
@@ -402,6 +413,7 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
         mbar_init(bar_acc, 1);
         fence_mbar_init();
     }
+    if (tid >= 32 && tid < 48) levels_s[tid - 32] = p.b.levels[tid - 32];
     if (warp == 8) {
         tmem_alloc(tmem_slot, kTcTmemCols);
         tmem_relinquish();
@@ -451,12 +463,40 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
         // ---- epilogue: thread = (row quadrant q, column half ch): row i0 + q * 32 + lane, 32 columns
         const int q = warp & 3, ch = warp >> 2;
         const int ri = q * 32 + lane, i = i0 + ri;
-        // rows of the dS tile and of the factor slices (widened to fp32) are an even number of floats
-        // apart: pairs of neighbouring values are read as one 8-byte word
-        float (*ds)[kTcCols + 2] = reinterpret_cast<float (*)[kTcCols + 2]>(base_ptr);
-        float (*fa)[kTcCols + 2] = reinterpret_cast<float (*)[kTcCols + 2]>(base_ptr + kTcRows * (kTcCols + 2) * 4);
-        float (*fb)[kTcRows + 2] =
-            reinterpret_cast<float (*)[kTcRows + 2]>(base_ptr + kTcRows * (kTcCols + 2) * 4 + r4 * (kTcCols + 2) * 4);
+        // the dS tile and the factor slices (widened to fp32)
+        float (*ds)[kTcDsPitch] = reinterpret_cast<float (*)[kTcDsPitch]>(base_ptr);
+        float (*fa)[kTcDsPitch] = reinterpret_cast<float (*)[kTcDsPitch]>(base_ptr + kTcRows * kTcDsPitch * 4);
+        float (*fb)[kTcFbPitch] =
+            reinterpret_cast<float (*)[kTcFbPitch]>(base_ptr + kTcRows * kTcDsPitch * 4 + r4 * kTcDsPitch * 4);
+        // What the epilogue needs from global memory does not depend on the tile product: the thread's codes and, for
+        // ranks that are multiples of 8 up to 32 (one 16-byte piece of the A slice and two of the B slice per thread),
+        // the factor slices are requested before the wait for the accumulator and parked in registers.
+        const int et = tid;                                       // 0 .. 255
+        const size_t row_bytes = (size_t)p.b.n * p.b.bits / 8;
+        const int jc = j0 + ch * 32, bits = p.b.bits;
+        // the thread's 32 codes are `bits` consecutive 32-bit words of its row when the group lies
+        // inside the row and the row pitch keeps it word-aligned; otherwise code by code
+        const bool whole_shape = i < p.b.m && jc + 32 <= p.b.n && (row_bytes & 3) == 0;
+        uint32_t cw[5] = {0u, 0u, 0u, 0u, 0u};
+        if (whole_shape) {
+            const uint32_t *src = reinterpret_cast<const uint32_t *>(p.b.q + (size_t)i * row_bytes + (size_t)jc * bits / 8);
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+                if (w < bits) cw[w] = __ldg(src + w);
+        }
+        const bool parked = (p.b.r & 7) == 0 && r4 <= 32;
+        uint4 park_a = make_uint4(0u, 0u, 0u, 0u), park_b[2] = {park_a, park_a};
+        if (parked) {
+            const int k = et / (kTcCols / 8), c8 = 8 * (et % (kTcCols / 8));
+            if (k < p.b.r && j0 + c8 < p.b.n) park_a = __ldg(reinterpret_cast<const uint4 *>(p.b.A + (size_t)k * p.b.n + j0 + c8));
+            const int per_row = p.b.r / 8;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int e = et + 256 * h, cidx = e / per_row, k8 = 8 * (e % per_row);
+                if (e < kTcRows * per_row && i0 + cidx < p.b.m)
+                    park_b[h] = __ldg(reinterpret_cast<const uint4 *>(p.b.B + (size_t)(i0 + cidx) * p.b.r + k8));
+            }
+        }
         const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, 0, status, 43));
         if (!ok) failed = true;
         tc_fence_after_sync();
@@ -467,30 +507,57 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
         }
         // every MMA has completed (the accumulator barrier), so every stage has been read: the stages'
         // memory now holds the factor slices and the dS tile
-        const int et = tid;                                       // 0 .. 255
-        auto load_slices = [&]() {
-            for (int e = et; e < r4 * kTcCols; e += 256) {            // A[k][j0 ..]
-                const int k = e / kTcCols, cidx = e % kTcCols;
-                fa[k][cidx] = (k < p.b.r && j0 + cidx < p.b.n) ? bf16f(p.b.A[(size_t)k * p.b.n + j0 + cidx]) : 0.0f;
+        auto store_a8 = [&](int k, int c8, const uint4 &v) {
+            *reinterpret_cast<float4 *>(&fa[k][c8]) = make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u),
+                                                                  __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xFFFF0000u));
+            *reinterpret_cast<float4 *>(&fa[k][c8 + 4]) = make_float4(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xFFFF0000u),
+                                                                      __uint_as_float(v.w << 16), __uint_as_float(v.w & 0xFFFF0000u));
+        };
+        auto store_b8 = [&](int cidx, int k8, const uint4 &v) {
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                fb[k8 + 2 * h][cidx] = __uint_as_float(w[h] << 16);
+                fb[k8 + 2 * h + 1][cidx] = __uint_as_float(w[h] & 0xFFFF0000u);
             }
-            for (int e = et; e < r4 * kTcRows; e += 256) {            // B[i0 ..][k] stored [k][i]; neighbouring threads read one row of B
-                const int cidx = e / r4, k = e % r4;
-                fb[k][cidx] = (k < p.b.r && i0 + cidx < p.b.m) ? bf16f(p.b.B[(size_t)(i0 + cidx) * p.b.r + k]) : 0.0f;
+        };
+        auto load_slices = [&]() {
+            if (parked) {
+                if (et < r4 * (kTcCols / 8)) store_a8(et / (kTcCols / 8), 8 * (et % (kTcCols / 8)), park_a);
+                const int per_row = p.b.r / 8;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int e = et + 256 * h;
+                    if (e < kTcRows * per_row) store_b8(e / per_row, 8 * (e % per_row), park_b[h]);
+                }
+                return;
+            }
+            // A[k][j0 ..]: eight columns (16 bytes) per load -- n is a multiple of 8 on this schedule, so a group
+            // of eight columns is whole and aligned
+            for (int e = et; e < r4 * (kTcCols / 8); e += 256) {
+                const int k = e / (kTcCols / 8), c8 = 8 * (e % (kTcCols / 8));
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (k < p.b.r && j0 + c8 < p.b.n) v = __ldg(reinterpret_cast<const uint4 *>(p.b.A + (size_t)k * p.b.n + j0 + c8));
+                store_a8(k, c8, v);
+            }
+            // B[i0 ..][k] stored [k][i]
+            if ((p.b.r & 7) == 0) {                                   // rows of B are 16-byte multiples: eight ranks per load
+                const int per_row = p.b.r / 8;
+                for (int e = et; e < kTcRows * per_row; e += 256) {
+                    const int cidx = e / per_row, k8 = 8 * (e % per_row);
+                    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                    if (i0 + cidx < p.b.m) v = __ldg(reinterpret_cast<const uint4 *>(p.b.B + (size_t)(i0 + cidx) * p.b.r + k8));
+                    store_b8(cidx, k8, v);
+                }
+            } else {
+                for (int e = et; e < r4 * kTcRows; e += 256) {        // neighbouring threads read one row of B
+                    const int cidx = e / r4, k = e % r4;
+                    fb[k][cidx] = (k < p.b.r && i0 + cidx < p.b.m) ? bf16f(p.b.B[(size_t)(i0 + cidx) * p.b.r + k]) : 0.0f;
+                }
             }
         };
         if constexpr (QAT) load_slices();                         // S is rebuilt from them below
-        const size_t row_bytes = (size_t)p.b.n * p.b.bits / 8;
-        const int jc = j0 + ch * 32, bits = p.b.bits;
-        // the thread's 32 codes are `bits` consecutive 32-bit words of its row when the group lies
-        // inside the row and the row pitch keeps it word-aligned; otherwise code by code
-        const bool whole = ok && i < p.b.m && jc + 32 <= p.b.n && (row_bytes & 3) == 0;
-        uint32_t cw[5] = {0u, 0u, 0u, 0u, 0u};
-        if (whole) {
-            const uint32_t *src = reinterpret_cast<const uint32_t *>(p.b.q + (size_t)i * row_bytes + (size_t)jc * bits / 8);
-#pragma unroll
-            for (int w = 0; w < 4; ++w)
-                if (w < bits) cw[w] = __ldg(src + w);
-        }
+        const bool whole = ok && whole_shape;
         // QAT: W / S per element (0 where S is 0, and the level is dropped there too: no gradient)
         float quot[QAT ? 32 : 1];
         bool live[QAT ? 32 : 1];
@@ -525,13 +592,16 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
             // the positions of the codes inside the words are compile-time constants for each width
             auto levels_of = [&](auto width) {
                 constexpr int W = decltype(width)::value;
+                float dv[4];
 #pragma unroll
                 for (int cidx = 0; cidx < 32; ++cidx) {
                     constexpr uint32_t mask = (1u << W) - 1u;
                     const int bit = cidx * W, w = bit >> 5, sh = bit & 31;
                     uint32_t code = cw[w] >> sh;
                     if (sh + W > 32) code |= cw[w + 1] << (32 - sh);
-                    ds[ri][ch * 32 + cidx] = __uint_as_float(gacc[cidx]) * factor(cidx, p.b.levels[code & mask]);
+                    dv[cidx & 3] = __uint_as_float(gacc[cidx]) * factor(cidx, levels_s[code & mask]);
+                    if ((cidx & 3) == 3)
+                        *reinterpret_cast<float4 *>(&ds[ri][ch * 32 + cidx - 3]) = make_float4(dv[0], dv[1], dv[2], dv[3]);
                 }
             };
             if (bits == 4) levels_of(std::integral_constant<int, 4>{});
@@ -543,50 +613,80 @@ __global__ void __launch_bounds__(kTcThreads) lords_backward_tc_kernel(const __g
                 const int j = jc + cidx;
                 float v = 0.0f;
                 if (ok && i < p.b.m && j < p.b.n)
-                    v = __uint_as_float(gacc[cidx]) * factor(cidx, p.b.levels[read_code(p.b.q, row_bytes, i, j, bits)]);
+                    v = __uint_as_float(gacc[cidx]) * factor(cidx, levels_s[read_code(p.b.q, row_bytes, i, j, bits)]);
                 ds[ri][ch * 32 + cidx] = v;
             }
         }
         if constexpr (!QAT) load_slices();
         asm volatile("bar.sync 1, 256;" ::: "memory");
-        // The folds, four ranks per thread so that a value of dS is read once for four products.  Each output is one thread's sum in index order.
+        // The folds, register-blocked so that a 16-byte word read from shared memory feeds 16 (dB) or 8 (dA)
+        // multiply-adds.  Each output is one thread's sum in index order.
         if (p.part_dB) {
+            // dB[i][k] = sum_j dS[i][j] A[k][j]: lane = rows lane + 32 a, warp = ranks 4 kg .. 4 kg + 3 (kg = warp, warp + 8, ..)
             float *out = p.part_dB + ((size_t)jt * p.b.m + i0) * r4;
-            for (int u = et; u < (r4 / 4) * kTcRows; u += 256) {          // dB[ii][k0 .. k0 + 3] = sum_j dS[ii][j] A[k][j]
-                const int ii = u % kTcRows, k0 = (u / kTcRows) * 4;
-                float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll 4
-                for (int jp = 0; jp < kTcCols / 2; ++jp) {
-                    const float2 d = *reinterpret_cast<const float2 *>(&ds[ii][2 * jp]);
+            for (int kg = warp; kg < r4 / 4; kg += 8) {
+                const int k0 = 4 * kg;
+                float acc[4][4];
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const float2 w = *reinterpret_cast<const float2 *>(&fa[k0 + kk][2 * jp]);
-                        acc[kk] = fmaf(d.x, w.x, acc[kk]);
-                        acc[kk] = fmaf(d.y, w.y, acc[kk]);
-                    }
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0f;
+#pragma unroll 2
+                for (int j4 = 0; j4 < kTcCols / 4; ++j4) {
+                    float4 d[4], w[4];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) d[a] = *reinterpret_cast<const float4 *>(&ds[lane + 32 * a][4 * j4]);
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) w[b] = *reinterpret_cast<const float4 *>(&fa[k0 + b][4 * j4]);
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) {
+                            acc[a][b] = fmaf(d[a].x, w[b].x, acc[a][b]);
+                            acc[a][b] = fmaf(d[a].y, w[b].y, acc[a][b]);
+                            acc[a][b] = fmaf(d[a].z, w[b].z, acc[a][b]);
+                            acc[a][b] = fmaf(d[a].w, w[b].w, acc[a][b]);
+                        }
                 }
-                if (i0 + ii < p.b.m)
-                    *reinterpret_cast<float4 *>(&out[(size_t)ii * r4 + k0]) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {
+                    const int ii = lane + 32 * a;
+                    if (i0 + ii < p.b.m)
+                        *reinterpret_cast<float4 *>(&out[(size_t)ii * r4 + k0]) = make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]);
+                }
             }
         }
         if (p.part_dA) {
+            // dA[k][j] = sum_i B[i][k] dS[i][j]: lane = columns 4 (lane & 15) .. + 3 and ranks 4 kg + 2 (lane >> 4) + {0, 1}
             float *out = p.part_dA + (size_t)it * r4 * p.b.n + j0;
-            for (int u = et; u < (r4 / 4) * kTcCols; u += 256) {          // dA[k0 .. k0 + 3][j] = sum_i B[i][k] dS[i][j]
-                const int j = u % kTcCols, k0 = (u / kTcCols) * 4;
-                float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll 4
-                for (int ip = 0; ip < kTcRows / 2; ++ip) {
-                    const float d0 = ds[2 * ip][j], d1 = ds[2 * ip + 1][j];
+            const int jq = 4 * (lane & 15), kh = 2 * (lane >> 4);
+            for (int kg = warp; kg < r4 / 4; kg += 8) {
+                const int k0 = 4 * kg + kh;
+                float acc[2][4];
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const float2 w = *reinterpret_cast<const float2 *>(&fb[k0 + kk][2 * ip]);
-                        acc[kk] = fmaf(w.x, d0, acc[kk]);
-                        acc[kk] = fmaf(w.y, d1, acc[kk]);
-                    }
+                for (int b = 0; b < 2; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.0f;
+#pragma unroll 2
+                for (int i4 = 0; i4 < kTcRows / 4; ++i4) {
+                    float4 d[4];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) d[a] = *reinterpret_cast<const float4 *>(&ds[4 * i4 + a][jq]);
+                    const float4 b0 = *reinterpret_cast<const float4 *>(&fb[k0][4 * i4]);
+                    const float4 b1 = *reinterpret_cast<const float4 *>(&fb[k0 + 1][4 * i4]);
+                    const float bv[2][4] = {{b0.x, b0.y, b0.z, b0.w}, {b1.x, b1.y, b1.z, b1.w}};
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+#pragma unroll
+                        for (int b = 0; b < 2; ++b) {
+                            acc[b][0] = fmaf(bv[b][a], d[a].x, acc[b][0]);
+                            acc[b][1] = fmaf(bv[b][a], d[a].y, acc[b][1]);
+                            acc[b][2] = fmaf(bv[b][a], d[a].z, acc[b][2]);
+                            acc[b][3] = fmaf(bv[b][a], d[a].w, acc[b][3]);
+                        }
                 }
-                if (j0 + j < p.b.n)
+                if (j0 + jq < p.b.n)                 // n is a multiple of 8 on this schedule: a group of four columns is whole
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) out[(size_t)(k0 + kk) * p.b.n + j] = acc[kk];
+                    for (int b = 0; b < 2; ++b)
+                        *reinterpret_cast<float4 *>(&out[(size_t)(k0 + b) * p.b.n + jq]) = make_float4(acc[b][0], acc[b][1], acc[b][2], acc[b][3]);
             }
         }
     }
