@@ -386,7 +386,7 @@ __host__ __device__ constexpr int bw_tc_smem(int r4)
 // QAT: the tile of g^T x is dL/dW^ itself (Eq. 4: stored as dL/dW if asked for), and the factor of
 // dL/dS is Q - W (/) S instead of Q (Eq. 5), with S = B A rebuilt per element from the factor slices.
 template <bool QAT>
-__global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 3) lords_backward_tc_kernel(const __grid_constant__ BwTcParams p)
+__global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_kernel(const __grid_constant__ BwTcParams p)
 {
     extern __shared__ uint8_t tc_smem_raw[];
     const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
@@ -657,36 +657,55 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 3) lords_backward_tc_ker
             }
         }
         if (p.part_dA) {
-            // dA[k][j] = sum_i B[i][k] dS[i][j]: lane = columns 4 (lane & 15) .. + 3 and ranks 4 kg + 2 (lane >> 4) + {0, 1}
+            // dA[k][j] = sum_i B[i][k] dS[i][j]: a thread takes 4 ranks x 4 columns over one half of the tile's rows
+            // (warps 0..3: rows 0..63, warps 4..7: rows 64..127); the upper half parks its sums in shared memory
+            // (the A slice's, which the dB fold is done with after the barrier), the lower half adds them to its own.
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             float *out = p.part_dA + (size_t)it * r4 * p.b.n + j0;
-            const int jq = 4 * (lane & 15), kh = 2 * (lane >> 4);
-            for (int kg = warp; kg < r4 / 4; kg += 8) {
-                const int k0 = 4 * kg + kh;
-                float acc[2][4];
+            float *park = &fa[0][0];                                  // [r4][64] floats
+            const int half = warp >> 2, jq = 4 * (lane & 15), ibase = 64 * half;
+            const int blocks = r4 / 4;
+            for (int kb0 = 0; kb0 < blocks; kb0 += 8) {               // the same trip count for every thread
+                const int kb = kb0 + 2 * (warp & 3) + (lane >> 4);
+                const bool active = kb < blocks;
+                const int k0 = 4 * (active ? kb : 0);
+                float acc[4][4];
 #pragma unroll
-                for (int b = 0; b < 2; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.0f;
-#pragma unroll 2
-                for (int i4 = 0; i4 < kTcRows / 4; ++i4) {
-                    float4 d[4];
+                for (int b = 0; b < 4; ++b) acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.0f;
+                if (active) {
+#pragma unroll 4
+                    for (int i2 = 0; i2 < 32; ++i2) {
+                        const int ii = ibase + 2 * i2;
+                        const float4 d0 = *reinterpret_cast<const float4 *>(&ds[ii][jq]);
+                        const float4 d1 = *reinterpret_cast<const float4 *>(&ds[ii + 1][jq]);
 #pragma unroll
-                    for (int a = 0; a < 4; ++a) d[a] = *reinterpret_cast<const float4 *>(&ds[4 * i4 + a][jq]);
-                    const float4 b0 = *reinterpret_cast<const float4 *>(&fb[k0][4 * i4]);
-                    const float4 b1 = *reinterpret_cast<const float4 *>(&fb[k0 + 1][4 * i4]);
-                    const float bv[2][4] = {{b0.x, b0.y, b0.z, b0.w}, {b1.x, b1.y, b1.z, b1.w}};
-#pragma unroll
-                    for (int a = 0; a < 4; ++a)
-#pragma unroll
-                        for (int b = 0; b < 2; ++b) {
-                            acc[b][0] = fmaf(bv[b][a], d[a].x, acc[b][0]);
-                            acc[b][1] = fmaf(bv[b][a], d[a].y, acc[b][1]);
-                            acc[b][2] = fmaf(bv[b][a], d[a].z, acc[b][2]);
-                            acc[b][3] = fmaf(bv[b][a], d[a].w, acc[b][3]);
+                        for (int b = 0; b < 4; ++b) {
+                            const float2 bv = *reinterpret_cast<const float2 *>(&fb[k0 + b][ii]);
+                            acc[b][0] = fmaf(bv.x, d0.x, acc[b][0]);
+                            acc[b][1] = fmaf(bv.x, d0.y, acc[b][1]);
+                            acc[b][2] = fmaf(bv.x, d0.z, acc[b][2]);
+                            acc[b][3] = fmaf(bv.x, d0.w, acc[b][3]);
+                            acc[b][0] = fmaf(bv.y, d1.x, acc[b][0]);
+                            acc[b][1] = fmaf(bv.y, d1.y, acc[b][1]);
+                            acc[b][2] = fmaf(bv.y, d1.z, acc[b][2]);
+                            acc[b][3] = fmaf(bv.y, d1.w, acc[b][3]);
                         }
-                }
-                if (j0 + jq < p.b.n)                 // n is a multiple of 8 on this schedule: a group of four columns is whole
+                    }
+                    if (half == 1) {
 #pragma unroll
-                    for (int b = 0; b < 2; ++b)
-                        *reinterpret_cast<float4 *>(&out[(size_t)(k0 + b) * p.b.n + jq]) = make_float4(acc[b][0], acc[b][1], acc[b][2], acc[b][3]);
+                        for (int b = 0; b < 4; ++b)
+                            *reinterpret_cast<float4 *>(&park[(k0 + b) * kTcCols + jq]) = make_float4(acc[b][0], acc[b][1], acc[b][2], acc[b][3]);
+                    }
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (active && half == 0 && j0 + jq < p.b.n) {        // n is a multiple of 8 on this schedule: a group of four columns is whole
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        const float4 u = *reinterpret_cast<const float4 *>(&park[(k0 + b) * kTcCols + jq]);
+                        *reinterpret_cast<float4 *>(&out[(size_t)(k0 + b) * p.b.n + jq]) =
+                            make_float4(acc[b][0] + u.x, acc[b][1] + u.y, acc[b][2] + u.z, acc[b][3] + u.w);
+                    }
+                }
             }
         }
     }
