@@ -373,14 +373,22 @@ struct alignas(64) BwTcParams {
     // quantisation-aware training (Eq. 4-5): the latent weight and, optionally, where dL/dW goes
     const uint16_t *W;    // bf16 [m][n]
     float *dW;            // float [m][n] or null
+    // QAT with a rank that is a multiple of 8 up to 64: S = B_tile A_tile by a scale MMA (Eq. 3), as in the forward kernels
+    CUtensorMap tm_b;     // bf16 [m][r], box {64 ranks, 128 rows}, 128-byte swizzle (ranks past r read as zero)
+    CUtensorMap tm_a;     // bf16 [r][n], box {64 columns, ceil16(r) ranks}, 128-byte swizzle
+    int scale_mma;
 };
 
-__host__ __device__ constexpr int bw_tc_smem(int r4)
+constexpr int kTcBTile = kTcRows * 128;                       // scale MMA: B[128 rows][64 ranks] bf16
+constexpr int kTcATile = 64 * 128;                            // scale MMA: A[64 ranks][64 columns] bf16
+
+__host__ __device__ constexpr int bw_tc_smem(int r4, bool qat)
 {
-    // the epilogue's buffers (dS tile, the two factor slices) reuse the stages once the MMAs are done
+    // the epilogue's buffers (dS tile, the two factor slices) reuse the stages once the MMAs are done;
+    // the operand tiles of the scale MMA (QAT) lie behind the barriers, on a 1024-byte boundary of their own
     const int stages = kTcStages * kTcStage;
     const int epi = kTcRows * kTcDsPitch * 4 + r4 * kTcDsPitch * 4 + r4 * kTcFbPitch * 4;
-    return 1024 + (stages > epi ? stages : epi) + 256;
+    return 1024 + (stages > epi ? stages : epi) + 256 + (qat ? 1024 + kTcBTile + kTcATile : 0);
 }
 
 // QAT: the tile of g^T x is dL/dW^ itself (Eq. 4: stored as dL/dW if asked for), and the factor of
@@ -397,6 +405,11 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_ker
     const uint32_t bars = base + (uint32_t)(stages_bytes > epi_bytes ? stages_bytes : epi_bytes);
     const uint32_t bar_full = bars, bar_empty = bars + 8 * kTcStages, bar_acc = bar_empty + 8 * kTcStages;
     const uint32_t tmem_slot = bar_acc + 8;
+    const uint32_t bar_s_full = bar_acc + 16, bar_s_done = bar_acc + 24;     // scale MMA (QAT): operand tiles landed, S complete
+    const uint32_t s_btile = (bars + 256u + 1023u) & ~1023u, s_atile = s_btile + kTcBTile;
+    const bool scale_mma = QAT && p.scale_mma != 0;
+    constexpr uint32_t kTmemCols = QAT ? 2 * kTcTmemCols : kTcTmemCols;     // QAT: S in the columns behind the accumulator
+    const int r16 = (p.b.r + 15) & ~15;
     // the level table in shared memory (16 floats behind the barriers): a lookup by a per-thread code is one
     // conflict-free read there, where the same lookup in the kernel parameters is replayed once per distinct code
     float *levels_s = reinterpret_cast<float *>(base_ptr + (bars - base) + 128);
@@ -411,11 +424,13 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_ker
     if (tid == 0) {
         for (int s = 0; s < kTcStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         mbar_init(bar_acc, 1);
+        mbar_init(bar_s_full, 1);
+        mbar_init(bar_s_done, 1);
         fence_mbar_init();
     }
     if (tid >= 32 && tid < 48) levels_s[tid - 32] = p.b.levels[tid - 32];
     if (warp == 8) {
-        tmem_alloc(tmem_slot, kTcTmemCols);
+        tmem_alloc(tmem_slot, kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before_sync();
@@ -428,6 +443,11 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_ker
         if (lane == 0) {
             tma_prefetch_desc(&p.tm_g);
             tma_prefetch_desc(&p.tm_x);
+            if (scale_mma) {
+                mbar_expect_tx(bar_s_full, (uint32_t)(kTcBTile + r16 * 128));
+                tma_load_2d(s_btile, &p.tm_b, 0, i0, bar_s_full);
+                tma_load_2d(s_atile, &p.tm_a, j0, 0, bar_s_full);
+            }
             for (int c = 0; c < chunks; ++c) {
                 const int s = c % kTcStages;
                 if (c >= kTcStages && !mbar_wait(bar_empty + 8 * s, (uint32_t)((c / kTcStages - 1) & 1), status, 41)) { failed = true; break; }
@@ -444,7 +464,23 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_ker
         const uint32_t a_lo0 = (uint32_t)umma_desc_sw128(0, 1024, (uint32_t)kTcGAtom) | ((base & 0x3FFFFu) >> 4);
         const uint32_t b_hi = (uint32_t)(umma_desc_sw128(0, 1024, 16) >> 32);
         const uint32_t b_lo0 = (uint32_t)umma_desc_sw128(0, 1024, 16) | (((base + 2 * kTcGAtom) & 0x3FFFFu) >> 4);
-        for (int c = 0; c < chunks; ++c) {
+        if (scale_mma) {
+            // S[128 x 64] = B_tile (K-major: a row is one row of B, 16 ranks = 32 bytes) * A_tile (MN-major: a row is one
+            // rank, 16 ranks = 16 rows of 128 bytes), one MMA per 16 ranks, into the columns behind the accumulator
+            constexpr uint32_t idesc_s = umma_idesc_f16(1, 0, 1, kTcRows, kTcCols);
+            if (!mbar_wait(bar_s_full, 0, status, 44)) failed = true;
+            tc_fence_after_sync();
+            if (lane == 0 && !failed) {
+                const uint32_t sb_lo = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((s_btile & 0x3FFFFu) >> 4);
+                const uint32_t sa_lo = (uint32_t)umma_desc_sw128(0, 1024, 16) | ((s_atile & 0x3FFFFu) >> 4);
+                for (int k = 0; k < r16 / 16; ++k)
+                    umma_f16_ss(tmem_base + kTcTmemCols, umma_desc_pack(sb_lo + k * 2, b_hi), umma_desc_pack(sa_lo + k * 128, b_hi),
+                                idesc_s, k > 0 ? 1u : 0u);
+                umma_commit(bar_s_done);
+            }
+            __syncwarp();
+        }
+        for (int c = 0; c < chunks && !failed; ++c) {
             const int s = c % kTcStages;
             if (!mbar_wait(bar_full + 8 * s, (uint32_t)((c / kTcStages) & 1), status, 42)) { failed = true; break; }
             tc_fence_after_sync();
@@ -567,14 +603,25 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_ker
                 for (int cidx = 0; cidx < 32; ++cidx)
                     if (jc + cidx < p.b.n) p.dW[(size_t)i * p.b.n + jc + cidx] = __uint_as_float(gacc[cidx]);
             }
-            asm volatile("bar.sync 1, 256;" ::: "memory");        // the factor slices are in place
             float sv[32];
+            if (scale_mma) {
+                // S of the thread's row and columns from the scale MMA (complete long before the tile product)
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_s_done, 0, status, 45))) failed = true;
+                tc_fence_after_sync();
+                uint32_t sraw[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + kTcTmemCols + (uint32_t)(ch * 32), sraw);
+                tmem_wait_ld();
 #pragma unroll
-            for (int cidx = 0; cidx < 32; ++cidx) sv[cidx] = 0.0f;
-            for (int k = 0; k < p.b.r; ++k) {
-                const float bk = fb[k][ri];
+                for (int cidx = 0; cidx < 32; ++cidx) sv[cidx] = failed ? 0.0f : __uint_as_float(sraw[cidx]);
+            } else {
+                asm volatile("bar.sync 1, 256;" ::: "memory");    // the factor slices are in place
 #pragma unroll
-                for (int cidx = 0; cidx < 32; ++cidx) sv[cidx] = fmaf(bk, fa[k][ch * 32 + cidx], sv[cidx]);
+                for (int cidx = 0; cidx < 32; ++cidx) sv[cidx] = 0.0f;
+                for (int k = 0; k < p.b.r; ++k) {
+                    const float bk = fb[k][ri];
+#pragma unroll
+                    for (int cidx = 0; cidx < 32; ++cidx) sv[cidx] = fmaf(bk, fa[k][ch * 32 + cidx], sv[cidx]);
+                }
             }
 #pragma unroll
             for (int cidx = 0; cidx < 32; ++cidx) {
@@ -715,7 +762,7 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_ker
     __syncthreads();
     if (warp == 8) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, kTcTmemCols);
+        tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -770,12 +817,18 @@ static int launch_backward_tc(const BwParams &p, const uint16_t *W, float *dW, S
     if (!make_map_2d(&k.tm_g, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.g, (uint64_t)m, (uint64_t)M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_map_2d(&k.tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.x, (uint64_t)n, (uint64_t)M, 64, 64, CU_TENSOR_MAP_SWIZZLE_128B))
         return LORDS_ERR_CUDA;
-    const int smem = bw_tc_smem(r4);
+    k.scale_mma = (W && (r & 7) == 0 && r <= 64) ? 1 : 0;
+    k.tm_b = k.tm_g; k.tm_a = k.tm_g;                                      // placeholders when the scale MMA is not used
+    if (k.scale_mma &&
+        (!make_map_2d(&k.tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.B, (uint64_t)r, (uint64_t)m, 64, (uint32_t)kTcRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
+         !make_map_2d(&k.tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.A, (uint64_t)n, (uint64_t)r, 64, (uint32_t)((r + 15) & ~15), CU_TENSOR_MAP_SWIZZLE_128B)))
+        return LORDS_ERR_CUDA;
+    const int smem = bw_tc_smem(r4, W != nullptr);
     static bool attr_set[kMaxDevices] = {};
     const int dev = device_slot(st);
     if (!attr_set[dev]) {
-        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_backward_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bw_tc_smem(kRMaxBw)));
-        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_backward_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bw_tc_smem(kRMaxBw)));
+        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_backward_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bw_tc_smem(kRMaxBw, false)));
+        LORDS_CUDA_TRY(cudaFuncSetAttribute(lords_backward_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bw_tc_smem(kRMaxBw, true)));
         attr_set[dev] = true;
     }
     if (W) lords_backward_tc_kernel<true><<<dim3((unsigned)jt_t, (unsigned)it_t), kTcThreads, smem, stream>>>(k);

@@ -178,8 +178,10 @@ QAT_NORMWISE_TOL = FACTOR_NORMWISE_TOL
 QAT_ELEMENT_TOL = FACTOR_ELEMENT_TOL
 
 
+# ranks that are multiples of 8 up to 64 take S from a scale MMA on the tensor schedule, the others rebuild it on the CUDA cores
 @pytest.mark.parametrize("bits,m,n,r,M,mixed", [(4, 512, 384, 32, 64, False), (3, 256, 544, 48, 8, True), (2, 320, 256, 6, 5, False),
-                                                (4, 136, 200, 12, 130, True)])
+                                                (4, 136, 200, 12, 130, True), (4, 264, 320, 64, 16, True), (3, 384, 256, 8, 40, False),
+                                                (4, 200, 136, 24, 9, True), (4, 128, 64, 72, 3, False)])
 def test_qat_backward_against_the_oracle(lords, bits, m, n, r, M, mixed):
     import torch
     lay = gen.make_layer(m, n, r, M, bits=bits, seed=m + 3 * n + r, mixed_sign=mixed)
