@@ -394,7 +394,7 @@ __host__ __device__ constexpr int bw_tc_smem(int r4, bool qat)
 // QAT: the tile of g^T x is dL/dW^ itself (Eq. 4: stored as dL/dW if asked for), and the factor of
 // dL/dS is Q - W (/) S instead of Q (Eq. 5), with S = B A rebuilt per element from the factor slices.
 template <bool QAT>
-__global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_kernel(const __grid_constant__ BwTcParams p)
+__global__ void __launch_bounds__(kTcThreads, 2) lords_backward_tc_kernel(const __grid_constant__ BwTcParams p)
 {
     extern __shared__ uint8_t tc_smem_raw[];
     const uint32_t base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
@@ -533,6 +533,15 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_ker
                     park_b[h] = __ldg(reinterpret_cast<const uint4 *>(p.b.B + (size_t)(i0 + cidx) * p.b.r + k8));
             }
         }
+        // QAT: the thread's 32 latent weights (64 bytes of its row; n is a multiple of 8, so a group of eight is whole)
+        uint4 wq[QAT ? 4 : 1];
+        if constexpr (QAT) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                wq[v] = make_uint4(0u, 0u, 0u, 0u);
+                if (i < p.b.m && jc + 8 * v < p.b.n) wq[v] = __ldg(reinterpret_cast<const uint4 *>(p.W + (size_t)i * p.b.n + jc + 8 * v));
+            }
+        }
         const bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc, 0, status, 43));
         if (!ok) failed = true;
         tc_fence_after_sync();
@@ -600,8 +609,11 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_ker
         if constexpr (QAT) {
             if (p.dW && ok && i < p.b.m) {                        // Eq. 4: dL/dW = dL/dW^
 #pragma unroll
-                for (int cidx = 0; cidx < 32; ++cidx)
-                    if (jc + cidx < p.b.n) p.dW[(size_t)i * p.b.n + jc + cidx] = __uint_as_float(gacc[cidx]);
+                for (int c4 = 0; c4 < 32; c4 += 4)
+                    if (jc + c4 < p.b.n)
+                        *reinterpret_cast<float4 *>(p.dW + (size_t)i * p.b.n + jc + c4) =
+                            make_float4(__uint_as_float(gacc[c4]), __uint_as_float(gacc[c4 + 1]), __uint_as_float(gacc[c4 + 2]),
+                                        __uint_as_float(gacc[c4 + 3]));
             }
             float sv[32];
             if (scale_mma) {
@@ -625,8 +637,9 @@ __global__ void __launch_bounds__(kTcThreads, QAT ? 1 : 2) lords_backward_tc_ker
             }
 #pragma unroll
             for (int cidx = 0; cidx < 32; ++cidx) {
-                const int j = jc + cidx;
-                const float w = (i < p.b.m && j < p.b.n) ? bf16f(p.W[(size_t)i * p.b.n + j]) : 0.0f;
+                const uint4 &wv = wq[cidx / 8];
+                const uint32_t ww = (cidx % 8) / 2 == 0 ? wv.x : (cidx % 8) / 2 == 1 ? wv.y : (cidx % 8) / 2 == 2 ? wv.z : wv.w;
+                const float w = __uint_as_float((cidx & 1) ? (ww & 0xFFFF0000u) : (ww << 16));
                 live[cidx] = sv[cidx] != 0.0f;
                 quot[cidx] = live[cidx] ? w / sv[cidx] : 0.0f;
             }
