@@ -535,6 +535,11 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 // x bf16 -> fp16 (exact for every bf16 value inside fp16's normal range), 8 elements per thread.
 __global__ void lords_x_to_f16_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ x16, size_t n_vec)
 {
+    // Programmatic dependent launch on both sides: the kernel that consumes x16 may begin its set-up (weights
+    // only) at once; this kernel itself waits for the previous launch, which may still be writing x or
+    // reading the scratch that x16 overwrites.
+    griddep_launch_dependents();
+    griddep_wait();
     size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= n_vec) return;
     const uint4 v = x[e];
@@ -626,7 +631,9 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
     }
 
     // Pair mode (BN > 16): when the tiles need more than one wave of CTAs, idle slots of the last wave
-    // are filled by splitting that many tiles' k-range over the two CTAs of a cluster.
+    // are filled by splitting that many tiles' k-range over the two CTAs of a cluster; when the tiles
+    // fill at most half of the resident CTAs, every tile's k-range is split (a tile is a serial chain
+    // of k-steps, so half the range is half the time).
     k.whole_pairs = -1;
     k.pair_scratch = nullptr;
     int clusters = (int)tiles;
@@ -644,6 +651,11 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
                 cs = 2;
                 pair_bytes = (size_t)split * BN * BM * sizeof(float);
             }
+        } else if (resident > 0 && 2 * tiles <= resident) {
+            k.whole_pairs = 0;
+            clusters = (int)tiles;
+            cs = 2;
+            pair_bytes = (size_t)tiles * BN * BM * sizeof(float);
         }
     }
 
@@ -653,9 +665,17 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
         if (x16_bytes + pair_bytes > st.workspace_bytes) return LORDS_ERR_WORKSPACE;
         k.pair_scratch = reinterpret_cast<float *>(st.workspace + x16_bytes);
         const size_t n_vec = (size_t)p.M * p.n / 8;
-        lords_x_to_f16_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, stream>>>(
-            reinterpret_cast<const uint4 *>(p.x), reinterpret_cast<uint4 *>(st.workspace), n_vec);
-        LORDS_CUDA_TRY(cudaGetLastError());
+        cudaLaunchAttribute pre_attr[1];
+        pre_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        pre_attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t pre_cfg = cudaLaunchConfig_t{};
+        pre_cfg.gridDim = dim3((unsigned)((n_vec + 255) / 256));
+        pre_cfg.blockDim = dim3(256);
+        pre_cfg.stream = stream;
+        pre_cfg.attrs = pre_attr;
+        pre_cfg.numAttrs = 1;
+        LORDS_CUDA_TRY(cudaLaunchKernelEx(&pre_cfg, lords_x_to_f16_kernel, reinterpret_cast<const uint4 *>(p.x),
+                                          reinterpret_cast<uint4 *>(st.workspace), n_vec));
         xsrc = st.workspace;
     }
     const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
@@ -675,10 +695,15 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
 template <int BITS, int RP> int launch_bits_rank(UmmaParams &k, const Problem &p, State &st, cudaStream_t stream)
 {
     if (p.M <= 16) return launch_variant<BITS, 16, RP>(k, p, st, stream);
-    // token tile: the largest that still gives CTAs for most of the SMs
+    // token tile: the largest that still gives CTAs for most of the SMs (tiles that fill at most half of the
+    // SMs are split over two CTAs each, see launch_variant)
     const long long row_tiles = (p.m + BM - 1) / BM;
+    auto ctas = [&](int b) {
+        const long long t = row_tiles * ((p.M + b - 1) / b);
+        return (2 * t <= st.sm_count && p.n > 128) ? 2 * t : t;
+    };
     int bn = 256;
-    while (bn > 32 && (p.M <= bn / 2 || 5 * row_tiles * ((p.M + bn - 1) / bn) < 3 * (long long)st.sm_count)) bn /= 2;
+    while (bn > 32 && (p.M <= bn / 2 || 5 * ctas(bn) < 3 * (long long)st.sm_count)) bn /= 2;
     if (st.forced_bn > 0) bn = st.forced_bn;   // measurement switch
     switch (bn) {
         case 32: return launch_variant<BITS, 32, RP>(k, p, st, stream);
