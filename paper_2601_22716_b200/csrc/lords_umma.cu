@@ -462,14 +462,16 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 #pragma unroll
                             for (int c = 0; c < 16; ++c) part[(size_t)(c0 + c) * BM + row] = __uint_as_float(v[c]);
                         } else if (i < p.m) {
+                            // the partner's sums of the chunk are all requested before the first store to y (which
+                            // the compiler must assume may alias them: load and store by turns would pay the way to
+                            // L2 sixteen times)
+                            float pv[16];
+#pragma unroll
+                            for (int c = 0; c < 16; ++c) pv[c] = pair_split ? __ldcg(part + (size_t)(c0 + c) * BM + row) : 0.0f;
 #pragma unroll
                             for (int c = 0; c < 16; ++c) {
                                 const int t = tok0 + c0 + c;
-                                if (t < p.M) {
-                                    float a = __uint_as_float(v[c]);
-                                    if (pair_split) a += __ldcg(part + (size_t)(c0 + c) * BM + row);   // fixed order: first half + second half
-                                    store_out(p.y, p.y_f32, (size_t)t * p.m + i, a);
-                                }
+                                if (t < p.M) store_out(p.y, p.y_f32, (size_t)t * p.m + i, __uint_as_float(v[c]) + pv[c]);   // fixed order: first half + second half
                             }
                         }
                     }
