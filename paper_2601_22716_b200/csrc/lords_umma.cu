@@ -535,12 +535,12 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
 }
 
 // x bf16 -> fp16 (exact for every bf16 value inside fp16's normal range), 8 elements per thread.
-__global__ void lords_x_to_f16_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ x16, size_t n_vec)
+__global__ void lords_x_to_f16_kernel(const uint4 *__restrict__ x, uint4 *__restrict__ x16, size_t n_vec, int early)
 {
-    // Programmatic dependent launch on both sides: the kernel that consumes x16 may begin its set-up (weights
-    // only) at once; this kernel itself waits for the previous launch, which may still be writing x or
-    // reading the scratch that x16 overwrites.
-    griddep_launch_dependents();
+    // Programmatic dependent launch on both sides (early != 0): the kernel that consumes x16 may begin its
+    // set-up (weights only) at once; this kernel itself waits for the previous launch, which may still be
+    // writing x or reading the scratch that x16 overwrites.  (Without the launch attribute both are no-ops.)
+    if (early) griddep_launch_dependents();
     griddep_wait();
     size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= n_vec) return;
@@ -667,9 +667,13 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
         if (x16_bytes + pair_bytes > st.workspace_bytes) return LORDS_ERR_WORKSPACE;
         k.pair_scratch = reinterpret_cast<float *>(st.workspace + x16_bytes);
         const size_t n_vec = (size_t)p.M * p.n / 8;
+        // A short pre-pass overlaps the main kernel's set-up (-2 us per call at 512 tokens); next to a long one
+        // (2048 tokens x 14336 columns: 18 us at the HBM rate) the early main kernel's CTAs and weight prefetch
+        // cost more than the overlap gains (+2 us), so there the main kernel starts when the pre-pass is done.
+        const int early = (size_t)p.M * p.n <= ((size_t)8 << 20) ? 1 : 0;
         cudaLaunchAttribute pre_attr[1];
         pre_attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        pre_attr[0].val.programmaticStreamSerializationAllowed = 1;
+        pre_attr[0].val.programmaticStreamSerializationAllowed = early;
         cudaLaunchConfig_t pre_cfg = cudaLaunchConfig_t{};
         pre_cfg.gridDim = dim3((unsigned)((n_vec + 255) / 256));
         pre_cfg.blockDim = dim3(256);
@@ -677,7 +681,7 @@ template <int BITS, int BN, int RP> int launch_variant(UmmaParams &k, const Prob
         pre_cfg.attrs = pre_attr;
         pre_cfg.numAttrs = 1;
         LORDS_CUDA_TRY(cudaLaunchKernelEx(&pre_cfg, lords_x_to_f16_kernel, reinterpret_cast<const uint4 *>(p.x),
-                                          reinterpret_cast<uint4 *>(st.workspace), n_vec));
+                                          reinterpret_cast<uint4 *>(st.workspace), n_vec, early));
         xsrc = st.workspace;
     }
     const uint64_t row_bytes = (uint64_t)p.n * BITS / 8;
