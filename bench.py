@@ -81,7 +81,7 @@ NCU_TRAFFIC_BYTES = {
     "mlp3_gate_m1": 23850496,       # profiles/decode_kernel_mlp3_gate_m1_down_m1.md
     "mlp3_down_m1": 23938560,       # same
     "mlp3_down_m16": 24299520,      # profiles/decode16_kernel_decode_q_m8_down_m16.md
-    "prefill_m2048": 142835712,     # profiles/umma_kernel_prefill_m2048.md (the scale-MMA kernel; the pre-pass moves 73.7 MB more)
+    "prefill_m2048": 145443072,     # profiles/umma_kernel_prefill_m2048.md (the scale-MMA kernel; the pre-pass moves 73.7 MB more)
     "quantize_q_nf4": 34120448,     # profiles/quantize_kernel_q_nf4_gate_nf3.md (8.4 MB of codes were still in L2 at the end)
     "quantize_gate_nf3": 130577408,
     "backward_q_m512": 19691008,    # profiles/backward_tc_kernel_backward_q_m512.md (the factor-gradient kernel)
