@@ -284,18 +284,25 @@ __global__ void __launch_bounds__(kThreads, 1) lords_umma_kernel(const __grid_co
                 const int rr = tid >> 1, half = tid & 1;
                 const int i = row0 + rr;
 #pragma unroll
+                const bool vec = (p.r & 7) == 0;     // rows of B are 16-byte multiples (B itself is 16-byte aligned)
+#pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const int chunk = half * 4 + c;
-                    uint32_t w4[4];
+                    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+                    if (vec) {
+                        if (i < p.m && chunk * 8 < p.r) w = __ldg(reinterpret_cast<const uint4 *>(p.B + (size_t)i * p.r + chunk * 8));
+                    } else {
+                        uint32_t w4[4];
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int k = chunk * 8 + e * 2;
-                        const uint32_t lo = (i < p.m && k < p.r) ? p.B[(size_t)i * p.r + k] : 0u;
-                        const uint32_t hi = (i < p.m && k + 1 < p.r) ? p.B[(size_t)i * p.r + k + 1] : 0u;
-                        w4[e] = lo | (hi << 16);
+                        for (int e = 0; e < 4; ++e) {
+                            const int k = chunk * 8 + e * 2;
+                            const uint32_t lo = (i < p.m && k < p.r) ? p.B[(size_t)i * p.r + k] : 0u;
+                            const uint32_t hi = (i < p.m && k + 1 < p.r) ? p.B[(size_t)i * p.r + k + 1] : 0u;
+                            w4[e] = lo | (hi << 16);
+                        }
+                        w = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                     }
-                    sts_v4(b_tile + (rr >> 3) * 1024 + (rr & 7) * 128 + ((chunk ^ (rr & 7)) * 16),
-                           make_uint4(w4[0], w4[1], w4[2], w4[3]));
+                    sts_v4(b_tile + (rr >> 3) * 1024 + (rr & 7) * 128 + ((chunk ^ (rr & 7)) * 16), w);
                 }
             }
             fence_proxy_async_smem();
