@@ -641,7 +641,12 @@ __global__ void __launch_bounds__(kTcThreads, 2) lords_backward_tc_kernel(const 
                 const uint32_t ww = (cidx % 8) / 2 == 0 ? wv.x : (cidx % 8) / 2 == 1 ? wv.y : (cidx % 8) / 2 == 2 ? wv.z : wv.w;
                 const float w = __uint_as_float((cidx & 1) ? (ww & 0xFFFF0000u) : (ww << 16));
                 live[cidx] = sv[cidx] != 0.0f;
-                quot[cidx] = live[cidx] ? w / sv[cidx] : 0.0f;
+                // w / S by a reciprocal and one residual correction: exact whenever the quotient is representable
+                // (a weight that its code reproduces exactly gets the factor 0), a rounding error otherwise
+                const float rc = __fdividef(1.0f, sv[cidx]);
+                float qv = w * rc;
+                qv = fmaf(fmaf(-qv, sv[cidx], w), rc, qv);
+                quot[cidx] = live[cidx] ? qv : 0.0f;
             }
         }
         auto factor = [&](int cidx, float level) -> float {
