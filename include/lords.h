@@ -232,7 +232,8 @@ int lords_linear_backward_factors(const void *dy, const void *x, const uint8_t *
  * and the lords_init workspace has room for the tiles' contributions; otherwise on the CUDA cores,
  * one pass over W per requested factor gradient, without scratch memory (any shape the forward calls
  * accept).  The quotient is formed in fp32 (on the tensor-core schedule by a reciprocal with one residual
- * correction: exact when W / S is representable, else within a rounding error or two); S is accumulated in fp32 from the exact products of the
+ * correction: exact when W / S is representable, else within a rounding error or two; a non-zero |S| below
+ * the smallest normal float, 1.2e-38, is outside the supported range there); S is accumulated in fp32 from the exact products of the
  * bf16 factors (by a tensor-core scale MMA when r is a multiple of 8 up to 64 on the tensor-core
  * schedule, else in ascending order of the rank).  An output that is NULL is not touched.  Enqueues on `stream` and returns without
  * synchronising.
