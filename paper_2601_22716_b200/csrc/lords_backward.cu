@@ -80,11 +80,19 @@ __global__ void lords_transpose_codes_kernel(const uint8_t *__restrict__ Q, uint
     for (int b = 0; b < bytes; ++b) dst[b] = (uint8_t)(b < 8 ? lo >> (8 * b) : hi >> (8 * (b - 8)));
 }
 
-// ---- transposition of a bf16 matrix [rows][cols] -> [cols][rows] --------------------------------------
-__global__ void lords_transpose_bf16_kernel(const uint16_t *__restrict__ src, uint16_t *__restrict__ dst, int rows, int cols)
+// Two transpositions in one launch (the factors A and B of a layer): blocks [0, tiles0) take the first matrix,
+// the others the second.
+__global__ void lords_transpose_bf16_pair_kernel(const uint16_t *__restrict__ src0, uint16_t *__restrict__ dst0, int rows0, int cols0,
+                                                 const uint16_t *__restrict__ src1, uint16_t *__restrict__ dst1, int rows1, int cols1,
+                                                 int tiles0)
 {
     __shared__ uint16_t tile[32][33];
-    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    const bool first = (int)blockIdx.x < tiles0;
+    const uint16_t *src = first ? src0 : src1;
+    uint16_t *dst = first ? dst0 : dst1;
+    const int rows = first ? rows0 : rows1, cols = first ? cols0 : cols1;
+    const int t = first ? (int)blockIdx.x : (int)blockIdx.x - tiles0, tiles_x = (cols + 31) / 32;
+    const int c0 = (t % tiles_x) * 32, r0 = (t / tiles_x) * 32;
     for (int k = threadIdx.y; k < 32; k += blockDim.y) {
         const int rr = r0 + k, cc = c0 + threadIdx.x;
         tile[k][threadIdx.x] = (rr < rows && cc < cols) ? src[(size_t)rr * cols + cc] : (uint16_t)0;
@@ -808,11 +816,12 @@ int launch_transpose_codes(const uint8_t *Q, int m, int n, int bits, uint8_t *Qt
     return LORDS_OK;
 }
 
-int launch_transpose_bf16(const uint16_t *src, int rows, int cols, uint16_t *dst, cudaStream_t stream)
+int launch_transpose_bf16_pair(const uint16_t *src0, int rows0, int cols0, uint16_t *dst0, const uint16_t *src1, int rows1, int cols1,
+                               uint16_t *dst1, cudaStream_t stream)
 {
-    const dim3 grid((unsigned)((cols + 31) / 32), (unsigned)((rows + 31) / 32));
-    if (grid.y > 65535u) return LORDS_ERR_SHAPE;
-    lords_transpose_bf16_kernel<<<grid, dim3(32, 8), 0, stream>>>(src, dst, rows, cols);
+    const long long t0 = (long long)((cols0 + 31) / 32) * ((rows0 + 31) / 32), t1 = (long long)((cols1 + 31) / 32) * ((rows1 + 31) / 32);
+    if (t0 + t1 > 2147483647LL) return LORDS_ERR_SHAPE;
+    lords_transpose_bf16_pair_kernel<<<(unsigned)(t0 + t1), dim3(32, 8), 0, stream>>>(src0, dst0, rows0, cols0, src1, dst1, rows1, cols1, (int)t0);
     LORDS_CUDA_TRY(cudaGetLastError());
     return LORDS_OK;
 }

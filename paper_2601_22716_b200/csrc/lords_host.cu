@@ -382,13 +382,13 @@ static int backward_input_common(const void *dy, const uint8_t *Qt, const void *
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint16_t *At = reinterpret_cast<uint16_t *>(st.bw_scratch), *Bt = reinterpret_cast<uint16_t *>(st.bw_scratch + at_bytes);
-    int rc = launch_transpose_bf16(static_cast<const uint16_t *>(A), r, n, At, s);       // A [r][n] -> [n][r]
-    if (rc == LORDS_OK) rc = launch_transpose_bf16(static_cast<const uint16_t *>(B), m, r, Bt, s);   // B [m][r] -> [r][m]
+    // A [r][n] -> [n][r] and B [m][r] -> [r][m], one launch
+    int rc = launch_transpose_bf16_pair(static_cast<const uint16_t *>(A), r, n, At, static_cast<const uint16_t *>(B), m, r, Bt, s);
     if (rc != LORDS_OK) return rc;
     // the transposed layer has n out-features and m in-features; its "B" is A^T and its "A" is B^T
     rc = forward_common(dy, Qt, At, Bt, cb, bits, M, n, m, r, dx, dx_f32, stream);
     if (rc != LORDS_OK) return rc;
-    st.last_launches += 2;
+    st.last_launches += 1;
     return LORDS_OK;
 }
 

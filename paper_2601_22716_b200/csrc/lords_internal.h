@@ -78,7 +78,8 @@ int launch_quantize(const void *W, const void *B, const void *A, const float *le
 // Backward with the codes fixed (Sec. 3.4): transposition of packed codes and of a bf16 matrix (what the
 // input gradient needs to run on the forward kernels), and the gradients of B and A on the CUDA cores.
 int launch_transpose_codes(const uint8_t *Q, int m, int n, int bits, uint8_t *Qt, cudaStream_t stream);
-int launch_transpose_bf16(const uint16_t *src, int rows, int cols, uint16_t *dst, cudaStream_t stream);
+int launch_transpose_bf16_pair(const uint16_t *src0, int rows0, int cols0, uint16_t *dst0, const uint16_t *src1, int rows1, int cols1,
+                               uint16_t *dst1, cudaStream_t stream);
 int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t *q, const uint16_t *B, const uint16_t *A,
                             const float *levels, int bits, int M, int m, int n, int r, float *dB, float *dA,
                             State &st, cudaStream_t stream);
