@@ -792,17 +792,39 @@ __global__ void __launch_bounds__(kTcThreads, 2) lords_backward_tc_kernel(const 
     }
 }
 
-// out[e] = sum over tiles t (in order) of part[t * stride + pos(e)]: dB (rows = m, inner = r, inner4 = r4)
-// or dA (rows = r, inner = inner4 = n).
-__global__ void lords_backward_reduce_kernel(const float *__restrict__ part, float *__restrict__ out, int tiles, size_t stride,
-                                             int rows, int inner, int inner4)
+// out[e] = sum over tiles t (in order) of part[t * stride + pos(e)], for dB (rows = m, inner = r, inner4 = r4:
+// blocks below blocks_b) and for dA (rows = r, inner = inner4 = n: the other blocks) in one launch.
+struct ReduceJob {
+    const float *part;
+    float *out;
+    int tiles, rows, inner, inner4;
+    size_t stride;
+};
+
+__global__ void lords_backward_reduce_kernel(const ReduceJob jb, const ReduceJob ja, int blocks_b)
 {
-    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= (size_t)rows * inner) return;
-    const size_t row = e / inner, col = e % inner;
+    const bool isb = (int)blockIdx.x < blocks_b;
+    const ReduceJob &j = isb ? jb : ja;
+    const size_t e = (size_t)(isb ? blockIdx.x : blockIdx.x - blocks_b) * blockDim.x + threadIdx.x;
+    if (e >= (size_t)j.rows * j.inner) return;
+    const size_t row = e / j.inner, col = e % j.inner;
     float s = 0.0f;
-    for (int t = 0; t < tiles; ++t) s += part[(size_t)t * stride + row * inner4 + col];
-    out[e] = s;
+    for (int t = 0; t < j.tiles; ++t) s += j.part[(size_t)t * j.stride + row * j.inner4 + col];
+    j.out[e] = s;
+}
+
+// The sums of the tiles' contributions to dB ([tiles_b][m][r4]) and dA ([tiles_a][r4][n]); either may be absent.
+int launch_reduce(const float *part_b, float *dB, int tiles_b, const float *part_a, float *dA, int tiles_a, int m, int n, int r, int r4,
+                  cudaStream_t stream)
+{
+    ReduceJob jb = {part_b, dB, tiles_b, dB ? m : 0, r, r4, (size_t)m * r4};
+    ReduceJob ja = {part_a, dA, tiles_a, dA ? r : 0, n, n, (size_t)r4 * n};
+    const size_t nb = ((size_t)jb.rows * r + 255) / 256, na = ((size_t)ja.rows * n + 255) / 256;
+    if (nb + na == 0) return LORDS_OK;
+    if (nb + na > 2147483647u) return LORDS_ERR_SHAPE;
+    lords_backward_reduce_kernel<<<(unsigned)(nb + na), 256, 0, stream>>>(jb, ja, (int)nb);
+    LORDS_CUDA_TRY(cudaGetLastError());
+    return LORDS_OK;
 }
 
 }  // namespace
@@ -862,16 +884,9 @@ static int launch_backward_tc(const BwParams &p, const uint16_t *W, float *dW, S
     else lords_backward_tc_kernel<false><<<dim3((unsigned)jt_t, (unsigned)it_t), kTcThreads, smem, stream>>>(k);
     LORDS_CUDA_TRY(cudaGetLastError());
     int launches = 1;
-    if (p.dB) {
-        const size_t total = (size_t)m * r;
-        lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(k.part_dB, p.dB, jt_t, (size_t)m * r4, m, r, r4);
-        LORDS_CUDA_TRY(cudaGetLastError());
-        ++launches;
-    }
-    if (p.dA) {
-        const size_t total = (size_t)r * n;
-        lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(k.part_dA, p.dA, it_t, (size_t)r4 * n, r, n, n);
-        LORDS_CUDA_TRY(cudaGetLastError());
+    if (p.dB || p.dA) {
+        const int rc = launch_reduce(k.part_dB, p.dB, jt_t, k.part_dA, p.dA, it_t, m, n, r, r4, stream);
+        if (rc != LORDS_OK) return rc;
         ++launches;
     }
     st.last_launches = launches;
@@ -905,16 +920,9 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
         lords_backward_tile_kernel<<<dim3((unsigned)jt_n, (unsigned)it_n), kBwThreads, 0, stream>>>(p, part_b, part_a);
         LORDS_CUDA_TRY(cudaGetLastError());
         ++launches;
-        if (dB) {
-            const size_t total = (size_t)m * r;
-            lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(part_b, dB, jt_n, (size_t)m * r4, m, r, r4);
-            LORDS_CUDA_TRY(cudaGetLastError());
-            ++launches;
-        }
-        if (dA) {
-            const size_t total = (size_t)r * n;
-            lords_backward_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(part_a, dA, it_n, (size_t)r4 * n, r, n, n);
-            LORDS_CUDA_TRY(cudaGetLastError());
+        {
+            const int rc = launch_reduce(part_b, dB, jt_n, part_a, dA, it_n, m, n, r, r4, stream);
+            if (rc != LORDS_OK) return rc;
             ++launches;
         }
         st.last_launches = launches;

@@ -94,10 +94,10 @@ def test_backward_against_the_oracle(lords, bits, m, n, r, M, mixed, path):
     check_against_oracle(dx32.cpu().numpy(), dxbf.cpu().numpy().view(np.uint16), dx64)
     # the three schedules of the factor gradients: the tile product on the tensor cores (taken when the row
     # pitches of g and x suit TMA), one CTA per tile of W on the CUDA cores -- both with the tiles'
-    # contributions summed by a second kernel --, and the walk that needs no scratch memory.  (Any forced
+    # contributions summed by a second kernel (one launch for dB and dA) --, and the walk that needs no scratch memory.  (Any forced
     # tensor-core forward path switches the tensor schedule off, "simt" leaves only the walk.)
     first = "backward_tensor" if m % 8 == 0 and n % 8 == 0 else "backward_tiles"
-    for option, schedule, launches in (("auto", first, 3), ("decode", "backward_tiles", 3), ("simt", "backward_walk", 2)):
+    for option, schedule, launches in (("auto", first, 2), ("decode", "backward_tiles", 2), ("simt", "backward_walk", 2)):
         dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
         dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
         lords.lords_set_option("path", option)
@@ -193,7 +193,7 @@ def test_qat_backward_against_the_oracle(lords, bits, m, n, r, M, mixed):
     q = torch.from_numpy(packed).to("cuda:0")
     # both schedules: the tile product on the tensor cores, and the walk on the CUDA cores that any forced
     # forward path other than "auto" selects (no scratch memory, one launch per factor gradient)
-    for option, schedule, launches in (("auto", "backward_qat_tensor", 3), ("simt", "backward_qat_walk", 2)):
+    for option, schedule, launches in (("auto", "backward_qat_tensor", 2), ("simt", "backward_qat_walk", 2)):
         dW = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda:0")
         dB = torch.full((m, r), float("nan"), dtype=torch.float32, device="cuda:0")
         dA = torch.full((r, n), float("nan"), dtype=torch.float32, device="cuda:0")
