@@ -84,8 +84,8 @@ int launch_backward_factors(const uint16_t *g, const uint16_t *x, const uint8_t 
                             const float *levels, int bits, int M, int m, int n, int r, float *dB, float *dA,
                             State &st, cudaStream_t stream);
 
-// Straight-through gradients of quantisation-aware training (Eq. 4-5); LORDS_ERR_UNSUPPORTED outside the
-// rules of the tensor-core schedule.
+// Straight-through gradients of quantisation-aware training (Eq. 4-5): the tensor-core schedule where its
+// rules hold, else one pass over W per requested factor gradient on the CUDA cores.
 int launch_backward_qat(const uint16_t *g, const uint16_t *x, const uint16_t *W, const uint8_t *q, const uint16_t *B,
                         const uint16_t *A, const float *levels, int bits, int M, int m, int n, int r, float *dW, float *dB,
                         float *dA, State &st, cudaStream_t stream);
