@@ -9,7 +9,11 @@
 // dx is the forward operator of the transposed layer: W^T = L[Q^T] (.) (A^T B^T), so with a transposed
 // copy of the packed codes (made once: the codes are frozen) and the transposed factors it runs on the
 // forward kernels as they are.  This file holds what that needs -- the transposition of packed codes
-// and of a bf16 matrix -- and the kernels for dB and dA.
+// and of the two factors -- and the kernels for dB and dA.
+//
+// The same kernels give the straight-through gradients of quantisation-aware training (Sec. 3.3, Eq. 4-5):
+// the tile of g^T x is dL/dW^ = dL/dW itself, and the factor of dL/dS is L[Q] - W (/) S instead of L[Q],
+// with S = B A rebuilt per tile (by a scale MMA on the tensor schedule where the rank allows it).
 //
 // dB and dA: a tile of dS is formed by the product g^T x over the tokens, multiplied by the levels of
 // the tile's codes, and folded with the matching column slice of A (for dB) and row slice of B (for
@@ -22,7 +26,8 @@
 //          sums in registers.  No scratch memory, g^T x formed once per gradient.
 //   tensor: the first schedule with the tile product g^T x on the tensor cores (tcgen05, bf16 operands
 //          straight from g and x by TMA, fp32 accumulator in TMEM) and only the level multiply and
-//          the two folds on the CUDA cores.  Taken when the row pitches suit TMA (m, n multiples of 8).
+//          the two folds (register-blocked, operands from shared memory as 16-byte words) on the CUDA
+//          cores.  Taken when the row pitches suit TMA (m, n multiples of 8).
 // Either way every output element is summed in a fixed order without atomics: runs are bit-identical.
 // Bound: fp32 ALU, m n M fused multiply-adds for the tile product (twice with the walk), or, with the
 // tensor schedule, the 2 m n r multiply-adds of the folds.
