@@ -159,10 +159,10 @@ int lords_linear_forward_f32(const void *x, const uint8_t *Qpacked, const void *
  * and y_host (bf16 [M][m]) are HOST pointers (pinned memory recommended, otherwise the copies
  * are synchronous); the weights Qpacked, B, A stay device-resident as above.  Enqueues, on
  * `stream`, the host-to-device copy of x, the same kernels as lords_linear_forward_bits and
- * the device-to-host copy of y, and returns without synchronising.  Buffers of up to 1 MiB in
- * pinned (mapped) host memory are moved by two small kernels that access the host memory
- * directly, which saves most of the latency of two DMA copies; larger or pageable ones go
- * through cudaMemcpyAsync.  The device staging
+ * the device-to-host copy of y, and returns without synchronising.  With buffers of up to 1 MiB
+ * in pinned (mapped) host memory no DMA copy is made: a small kernel reads x from the host memory
+ * and the forward kernels store y straight into it, which saves most of the latency of two DMA
+ * copies; larger or pageable buffers go through cudaMemcpyAsync.  The device staging
  * buffers are library-owned and grow (cudaMalloc) the first time a larger M*n or M*m is seen,
  * so the first call of a given size must not be made during stream capture.
  */

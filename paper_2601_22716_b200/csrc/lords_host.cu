@@ -321,16 +321,12 @@ int lords_linear_forward_host(const void *x_host, const uint8_t *Qpacked, const 
     } else {
         LORDS_CUDA_TRY(cudaMemcpyAsync(st.stage_x, x_host, xb, cudaMemcpyHostToDevice, s));
     }
-    rc = forward_common(st.stage_x, Qpacked, B, A, codebook, bits, M, m, n, r, st.stage_y, 0, stream);
+    // direct: the kernels store y straight into the mapped host buffer (no kernel reads y back), which saves the
+    // copy-out launch
+    rc = forward_common(st.stage_x, Qpacked, B, A, codebook, bits, M, m, n, r, direct ? y_map : st.stage_y, 0, stream);
     if (rc != LORDS_OK) return rc;
-    const int kernels = st.last_launches;
-    if (direct) {
-        rc = copy16(st.stage_y, y_map, yb, s);
-        if (rc != LORDS_OK) return rc;
-        st.last_launches = kernels + 2;
-    } else {
-        LORDS_CUDA_TRY(cudaMemcpyAsync(y_host, st.stage_y, yb, cudaMemcpyDeviceToHost, s));
-    }
+    if (direct) st.last_launches += 1;
+    else LORDS_CUDA_TRY(cudaMemcpyAsync(y_host, st.stage_y, yb, cudaMemcpyDeviceToHost, s));
     return LORDS_OK;
 }
 

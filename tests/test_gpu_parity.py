@@ -455,14 +455,24 @@ def test_many_back_to_back_launches_leave_no_status(lords, m, n, r, bits, M, pat
         assert torch.equal(y, f)
 
 
-def test_host_buffer_entry_point_matches_device_entry(lords):
+@pytest.mark.parametrize("M,path", [(1, "auto"), (4, "auto"), (40, "auto"), (3, "simt"), (300, "auto")])
+def test_host_buffer_entry_point_matches_device_entry(lords, M, path):
+    """x from and y into pinned host memory (small buffers: y is stored by the kernels straight into the
+    mapped host buffer; 300 tokens: staged copies), on every kind of kernel: bit-identical to the device entry."""
     import torch
-    lay = gen.make_layer(512, 1024, 16, 4, bits=4, seed=12)
-    dl, y32, ybf = _run(lords, lay)
+    lay = gen.make_layer(520, 1024, 16, M, bits=4, seed=12 + M)
+    dl, y32, ybf = _run(lords, lay, path)
+    used = lords.lords_last_path()
     xh = torch.from_numpy(lay.x.view(np.int16)).pin_memory()
-    yh = torch.zeros((lay.M, lay.m), dtype=torch.int16).pin_memory()
-    lords.lords_linear_forward_host(xh, dl.q, dl.B, dl.A, lay.codebook, lay.bits, lay.M, lay.m, lay.n, lay.r, yh)
+    yh = torch.full((lay.M, lay.m), 0x7FC0, dtype=torch.int16).pin_memory()
+    lords.lords_set_option("path", path)
+    try:
+        lords.lords_linear_forward_host(xh, dl.q, dl.B, dl.A, lay.codebook, lay.bits, lay.M, lay.m, lay.n, lay.r, yh)
+    finally:
+        lords.lords_set_option("path", "auto")
+    assert lords.lords_last_path() == used
     torch.cuda.synchronize()
+    assert lords.lords_poll_status() == 0
     assert np.array_equal(yh.numpy().view(np.uint16), ybf)
 
 
