@@ -161,8 +161,10 @@ int lords_linear_forward_f32(const void *x, const uint8_t *Qpacked, const void *
  * `stream`, the host-to-device copy of x, the same kernels as lords_linear_forward_bits and
  * the device-to-host copy of y, and returns without synchronising.  With buffers of up to 1 MiB
  * in pinned (mapped) host memory no DMA copy is made: a small kernel reads x from the host memory
- * and the forward kernels store y straight into it, which saves most of the latency of two DMA
- * copies; larger or pageable buffers go through cudaMemcpyAsync.  The device staging
+ * (it may do so while the previous kernel in the stream is still running: x_host must not be the
+ * target of work enqueued earlier on the stream) and the forward kernels store y straight into
+ * y_host, which saves most of the latency of two DMA copies; larger or pageable buffers go through
+ * cudaMemcpyAsync.  The device staging
  * buffers are library-owned and grow (cudaMalloc) the first time a larger M*n or M*m is seen,
  * so the first call of a given size must not be made during stream capture.
  */

@@ -14,15 +14,28 @@ State &state()
     return s;
 }
 
-// Small host buffers are moved by a kernel that reads or writes the pinned host memory directly
-// (mapped into the device's address space): two DMA copies of a few KB cost about 10 us each in
-// latency, a kernel's loads and stores across the bus about 2 us.
-__global__ void lords_copy16_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, size_t n16)
-{
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) dst[i] = src[i];
-}
-
+// A small x in pinned host memory (mapped into the device's address space) is fetched by a kernel: a DMA copy
+// of a few KB costs about 10 us in latency, a kernel's loads across the bus about 2 us.  The kernel is a
+// programmatic dependent launch on both sides: it reads the host buffer (which no kernel writes) at once,
+// waits for the previous kernel in the stream -- which may still be reading the staging buffer -- and only
+// then stores; the forward kernel behind it may begin its set-up meanwhile.
 constexpr size_t kDirectHostBytes = 1u << 20;   // above this the copy engines win
+constexpr int kFetchBlocks = 64, kFetchThreads = 256;
+constexpr int kFetchPerThread = (int)(kDirectHostBytes / 16 / (kFetchBlocks * kFetchThreads));   // 4
+
+__global__ void __launch_bounds__(kFetchThreads) lords_fetch_host_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, size_t n16)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
+    uint4 v[kFetchPerThread];
+#pragma unroll
+    for (int k = 0; k < kFetchPerThread; ++k)
+        if (t + k * stride < n16) v[k] = src[t + k * stride];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#pragma unroll
+    for (int k = 0; k < kFetchPerThread; ++k)
+        if (t + k * stride < n16) dst[t + k * stride] = v[k];
+}
 
 // The device's address of a pinned, mapped host buffer; false for pageable or foreign memory.
 static bool mapped_device_pointer(const void *host, void **dev)
@@ -37,12 +50,20 @@ static bool mapped_device_pointer(const void *host, void **dev)
     return true;
 }
 
-static int copy16(const void *src, void *dst, size_t bytes, cudaStream_t s)
+static int fetch_host(const void *src, void *dst, size_t bytes, cudaStream_t s)
 {
-    const size_t n16 = bytes / 16;
-    const unsigned blocks = (unsigned)((n16 + 255) / 256 < 64 ? (n16 + 255) / 256 : 64);
-    lords_copy16_kernel<<<blocks, 256, 0, s>>>(static_cast<const uint4 *>(src), static_cast<uint4 *>(dst), n16);
-    LORDS_CUDA_TRY(cudaGetLastError());
+    const size_t n16 = bytes / 16;      // bytes <= kDirectHostBytes: at most kFetchPerThread words per thread
+    const size_t want = (n16 + kFetchThreads - 1) / kFetchThreads;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = dim3((unsigned)(want < (size_t)kFetchBlocks ? (want > 0 ? want : 1) : (size_t)kFetchBlocks));
+    cfg.blockDim = dim3(kFetchThreads);
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    LORDS_CUDA_TRY(cudaLaunchKernelEx(&cfg, lords_fetch_host_kernel, static_cast<const uint4 *>(src), static_cast<uint4 *>(dst), n16));
     return LORDS_OK;
 }
 
@@ -316,7 +337,7 @@ int lords_linear_forward_host(const void *x_host, const uint8_t *Qpacked, const 
                         mapped_device_pointer(y_host, &y_map);
     int rc;
     if (direct) {
-        rc = copy16(x_map, st.stage_x, xb, s);
+        rc = fetch_host(x_map, st.stage_x, xb, s);
         if (rc != LORDS_OK) return rc;
     } else {
         LORDS_CUDA_TRY(cudaMemcpyAsync(st.stage_x, x_host, xb, cudaMemcpyHostToDevice, s));
